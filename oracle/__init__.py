@@ -1,0 +1,206 @@
+"""CPU oracle for the per-fragment merge (TEST INFRASTRUCTURE ONLY).
+
+Thin ctypes wrapper around ``dd_oracle.c`` (plain C99, fp64, single thread).
+It is imported by the test-suite, by the smoke check and by the benchmark's
+cpu_baseline / reference legs -- never by the product package, and it imports
+nothing from it.  bf16 arrays are carried as ``numpy.uint16`` bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass, field
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "dd_oracle.c")
+_LIB = os.path.join(_HERE, "libdd_oracle.so")
+
+MAX_LEARNERS = 64
+STATUS_OK, STATUS_QUORUM_NOT_MET, STATUS_ZERO_WEIGHT, INVALID = 0, 1, 2, -1
+MERGE_AVG, MERGE_RDA = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (``-O2``, no OpenMP, no fast-math)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c99", "-fPIC", "-shared", "-Wall", "-Wextra",
+             "-ffp-contract=off", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _Record(ctypes.Structure):
+    _fields_ = [
+        ("status", ctypes.c_int32),
+        ("n_part", ctypes.c_int32),
+        ("idx", ctypes.c_uint8 * MAX_LEARNERS),
+        ("w_hat", ctypes.c_double * MAX_LEARNERS),
+        ("w_total", ctypes.c_double),
+        ("delta_sq", ctypes.c_double),
+        ("theta_sq", ctypes.c_double),
+        ("mom_sq", ctypes.c_double),
+        ("delta_m_sq", ctypes.c_double * MAX_LEARNERS),
+    ]
+
+
+@dataclass
+class Record:
+    status: int
+    n_part: int
+    idx: list = field(default_factory=list)
+    w_hat: list = field(default_factory=list)
+    w_total: float = 0.0
+    delta_sq: float = 0.0
+    theta_sq: float = 0.0
+    mom_sq: float = 0.0
+    delta_m_sq: list = field(default_factory=list)
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        u64p = ctypes.POINTER(ctypes.c_uint64)
+        lib.ddo_bf16_rne.restype = ctypes.c_uint16
+        lib.ddo_bf16_rne.argtypes = [ctypes.c_float]
+        lib.ddo_bf16_rne_array.restype = None
+        lib.ddo_bf16_rne_array.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t]
+        lib.ddo_bf16_to_f32.restype = ctypes.c_float
+        lib.ddo_bf16_to_f32.argtypes = [ctypes.c_uint16]
+        lib.ddo_participants.restype = ctypes.c_int
+        lib.ddo_participants.argtypes = [ctypes.c_uint64, u64p, ctypes.c_int, ctypes.c_int,
+                                         ctypes.POINTER(ctypes.c_uint8),
+                                         ctypes.POINTER(ctypes.c_int32)]
+        lib.ddo_weights.restype = ctypes.c_int
+        lib.ddo_weights.argtypes = [u64p, u64p, ctypes.POINTER(ctypes.c_uint8), ctypes.c_int,
+                                    ctypes.POINTER(ctypes.c_double),
+                                    ctypes.POINTER(ctypes.c_double)]
+        lib.ddo_merge_fragment.restype = ctypes.c_int
+        lib.ddo_merge_fragment.argtypes = [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.c_int,
+            ctypes.c_int, u64p, u64p, ctypes.c_uint64, ctypes.c_int, ctypes.c_float,
+            ctypes.c_float, ctypes.c_int, ctypes.c_int, ctypes.c_size_t, ctypes.c_void_p,
+            ctypes.POINTER(_Record)]
+        lib.ddo_grace_window.restype = ctypes.c_double
+        lib.ddo_grace_window.argtypes = [ctypes.c_double] * 5
+        lib.ddo_select_quorum.restype = ctypes.c_int
+        lib.ddo_select_quorum.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.c_int,
+                                          ctypes.c_int, ctypes.c_double,
+                                          ctypes.POINTER(ctypes.c_uint64),
+                                          ctypes.POINTER(ctypes.c_int32)]
+        _lib = lib
+    return _lib
+
+
+def _u64(values):
+    arr = (ctypes.c_uint64 * len(values))(*[int(x) for x in values])
+    return arr
+
+
+def bf16_rne(x) -> np.ndarray:
+    """fp32 array -> bf16 bit patterns (uint16), round-to-nearest-even."""
+    lib = _load()
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    out = np.empty(x.shape, dtype=np.uint16)
+    lib.ddo_bf16_rne_array(x.ctypes.data, out.ctypes.data, x.size)
+    return out
+
+
+def bf16_to_f32(h) -> np.ndarray:
+    """bf16 bit patterns (uint16) -> fp32 (exact)."""
+    h = np.ascontiguousarray(h, dtype=np.uint16)
+    return (h.astype(np.uint32) << 16).view(np.float32)
+
+
+def participants(mask: int, tokens, K: int):
+    """Returns (status, idx list)."""
+    lib = _load()
+    M = len(tokens)
+    idx = (ctypes.c_uint8 * MAX_LEARNERS)()
+    n_part = ctypes.c_int32(0)
+    st = lib.ddo_participants(ctypes.c_uint64(mask & (2**64 - 1)), _u64(tokens), M, K, idx,
+                              ctypes.byref(n_part))
+    if st == INVALID:
+        raise ValueError("oracle: invalid participation arguments")
+    return st, [int(idx[j]) for j in range(n_part.value)]
+
+
+def weights(tokens, steps, idx):
+    """Returns (status, w_hat list aligned with idx, w_total)."""
+    lib = _load()
+    s = len(idx)
+    idx_c = (ctypes.c_uint8 * MAX_LEARNERS)(*idx)
+    w_hat = (ctypes.c_double * MAX_LEARNERS)()
+    W = ctypes.c_double(0.0)
+    st = lib.ddo_weights(_u64(tokens), None if steps is None else _u64(steps), idx_c, s, w_hat,
+                         ctypes.byref(W))
+    if st == INVALID:
+        raise ValueError("oracle: tokens > 0 with steps == 0")
+    return st, [float(w_hat[j]) for j in range(s)], float(W.value)
+
+
+def merge_fragment(theta: np.ndarray, v: np.ndarray, learners, tokens, mask: int, K: int,
+                   eta: float, mu: float, *, steps=None, nesterov: bool = True,
+                   merge: int = MERGE_AVG, out_bf16: np.ndarray | None = None) -> Record:
+    """One syncer update of one fragment, IN PLACE on ``theta`` and ``v``.
+
+    ``theta``/``v``: contiguous float32 arrays of n elements.  ``learners``: list
+    of M arrays (all float32, or all uint16 holding bf16 bits) or ``None`` for a
+    learner whose copy is not available.  ``out_bf16``: optional uint16[n].
+    """
+    lib = _load()
+    assert theta.dtype == np.float32 and v.dtype == np.float32
+    assert theta.flags.c_contiguous and v.flags.c_contiguous and theta.shape == v.shape
+    n = theta.size
+    M = len(learners)
+    present = [a for a in learners if a is not None]
+    is_bf16 = bool(present) and present[0].dtype == np.uint16
+    ptrs = (ctypes.c_void_p * M)()
+    for m, a in enumerate(learners):
+        if a is None:
+            ptrs[m] = None
+            continue
+        assert a.dtype == (np.uint16 if is_bf16 else np.float32), "mixed learner dtypes"
+        assert a.flags.c_contiguous and a.size == n
+        ptrs[m] = a.ctypes.data
+    if out_bf16 is not None:
+        assert out_bf16.dtype == np.uint16 and out_bf16.size == n and out_bf16.flags.c_contiguous
+    rec = _Record()
+    rc = lib.ddo_merge_fragment(
+        theta.ctypes.data, v.ctypes.data, ptrs, M, int(is_bf16), _u64(tokens),
+        None if steps is None else _u64(steps), ctypes.c_uint64(mask & (2**64 - 1)), K,
+        ctypes.c_float(eta), ctypes.c_float(mu), int(nesterov), int(merge), n,
+        None if out_bf16 is None else out_bf16.ctypes.data, ctypes.byref(rec))
+    if rc != 0:
+        raise ValueError("oracle: invalid merge arguments")
+    s = rec.n_part
+    return Record(status=rec.status, n_part=s, idx=[int(rec.idx[j]) for j in range(s)],
+                  w_hat=[float(rec.w_hat[j]) for j in range(s)], w_total=float(rec.w_total),
+                  delta_sq=float(rec.delta_sq), theta_sq=float(rec.theta_sq),
+                  mom_sq=float(rec.mom_sq),
+                  delta_m_sq=[float(rec.delta_m_sq[j]) for j in range(s)])
+
+
+def grace_window(tau, xi_step, xi_quorum, xi_sync, gamma) -> float:
+    return float(_load().ddo_grace_window(tau, xi_step, xi_quorum, xi_sync, gamma))
+
+
+def select_quorum(arrival, K: int, grace: float):
+    """Returns (status, mask, n_admitted)."""
+    lib = _load()
+    M = len(arrival)
+    arr = (ctypes.c_double * M)(*[float(a) for a in arrival])
+    mask = ctypes.c_uint64(0)
+    n_adm = ctypes.c_int32(0)
+    st = lib.ddo_select_quorum(arr, M, K, float(grace), ctypes.byref(mask), ctypes.byref(n_adm))
+    if st == INVALID:
+        raise ValueError("oracle: invalid quorum arguments")
+    return st, int(mask.value), int(n_adm.value)
