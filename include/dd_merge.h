@@ -1,0 +1,181 @@
+/*
+ * dd_merge.h -- C ABI of libddmerge: the Decoupled DiLoCo syncer's per-fragment
+ * merge on one NVIDIA B200 (sm_100a).
+ *
+ * For one parameter fragment the syncer (Algorithm 2, steps 2-3) takes the copies
+ * theta_m held by the M learners, keeps the learners that reported in time
+ * (minimum quorum K and grace window, Section 3.2), weights their outer
+ * gradients Theta - theta_m by the token/step counters (the Weight display,
+ * Section 3.2), merges them (weighted direct averaging, Appendix "Merging
+ * methods") and applies the outer optimizer, SGD with Nesterov momentum (Eq. 1,
+ * Eq. 2), to the global fragment Theta and its momentum v.  The whole chain runs
+ * in one fused CUDA kernel that reads every participating operand once.
+ *
+ * Conventions common to every call
+ *   - Pointers marked [device] are device addresses on the context's GPU;
+ *     pointers marked [host] are ordinary host memory.  Every buffer is borrowed:
+ *     the library allocates only its own context workspace.
+ *   - Theta and v are float32 and are updated IN PLACE.  Learner copies are
+ *     read-only, contiguous, all float32 or all bf16 (dd_dtype).
+ *   - Device base pointers must be 16-byte aligned.  n is arbitrary.
+ *   - Calls enqueue work on the given CUDA stream (a cudaStream_t passed as
+ *     void*; NULL = the legacy default stream) and return without waiting.  Host
+ *     arrays are consumed before the call returns.
+ *   - Return value: DD_OK (0) or a negative dd_error.  Conditions that depend on
+ *     the data -- quorum not met, zero total weight -- are not errors: the call
+ *     returns DD_OK, writes dd_merge_record.status != 0 and leaves Theta and v
+ *     untouched (the syncer "keeps waiting", Algorithm 2 step 1).
+ *   - Nothing here aborts, throws, traps or spins without bound on the device.
+ */
+#ifndef DD_MERGE_H
+#define DD_MERGE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DD_MAX_LEARNERS 64
+
+typedef struct dd_ctx dd_ctx;
+
+typedef enum { DD_F32 = 0, DD_BF16 = 1 } dd_dtype;
+
+typedef enum {
+    DD_OK = 0,
+    DD_ERR_INVALID_ARG = -1,        /* null where not allowed, M / K / P out of range, non-finite lr or mu */
+    DD_ERR_ALIGNMENT = -2,          /* a device pointer is not 16-byte aligned */
+    DD_ERR_ALIAS = -3,              /* a participating learner buffer overlaps Theta, v or out_bf16 */
+    DD_ERR_TOO_MANY_LEARNERS = -4,  /* M > DD_MAX_LEARNERS */
+    DD_ERR_CUDA = -5,               /* a CUDA runtime call failed; see dd_last_cuda_error */
+    DD_ERR_TOO_LARGE = -6           /* a size exceeds what the entry point supports */
+} dd_error;
+
+/* dd_merge_record.status */
+enum {
+    DD_STATUS_OK = 0,
+    DD_STATUS_QUORUM_NOT_MET = 1,   /* fewer than max(K,1) participants; nothing written */
+    DD_STATUS_ZERO_WEIGHT = 2,      /* weights sum to zero; nothing written */
+    DD_STATUS_WAIT_LIMIT = 3        /* a bounded device-side wait gave up; fragment state is unspecified */
+};
+
+/* flags */
+enum {
+    DD_HEAVY_BALL = 1u << 0,        /* Theta' = Theta - lr v' instead of the Nesterov form */
+    DD_DIAG_PER_LEARNER = 1u << 1,  /* also ||Theta - theta_m||^2 for every participant */
+    DD_DIAG_STATE = 1u << 2         /* also ||Theta'||^2 and ||v'||^2 */
+};
+
+/*
+ * Written by the device, one per fragment; readable by the host once the stream
+ * has been synchronised.  Participants are listed in ascending learner id.
+ */
+typedef struct {
+    int32_t status;
+    int32_t n_part;                         /* |S|, S = { m : mask bit m and tokens[m] > 0 } */
+    uint8_t idx[DD_MAX_LEARNERS];           /* first n_part entries valid */
+    float   w_hat[DD_MAX_LEARNERS];         /* normalised weights, aligned with idx */
+    double  w_total;                        /* sum of the raw weights over S */
+    double  delta_sq;                       /* ||Delta||_2^2 of the merged outer gradient */
+    double  theta_sq;                       /* ||Theta'||_2^2   (DD_DIAG_STATE) */
+    double  mom_sq;                         /* ||v'||_2^2       (DD_DIAG_STATE) */
+    double  delta_m_sq[DD_MAX_LEARNERS];    /* ||Theta - theta_m||_2^2, aligned with idx (DD_DIAG_PER_LEARNER) */
+} dd_merge_record;
+
+/*
+ * Context: binds a GPU and owns a small workspace (per-CTA partial sums of the
+ * norm diagnostics, completion tickets, a ring of descriptor staging slots).
+ * One context serves one host thread at a time; calls issued through one
+ * context on DIFFERENT streams must not overlap on the GPU, because they
+ * share that workspace.  device < 0 selects the current device.
+ */
+int dd_create(dd_ctx **ctx, int device);
+int dd_destroy(dd_ctx *ctx);
+
+/*
+ * One syncer update of one fragment (Algorithm 2 steps 2-3).
+ *
+ *   S      = { m < M : bit m of quorum_mask set and tokens[m] > 0 }      (Section 3.2; Section 4:
+ *            an absent learner is a learner of weight 0)
+ *   w_m    = tokens[m] * (tokens[m] / steps[m]);  tokens[m] when steps == NULL   (Weight, Section 3.2)
+ *   w^_m   = w_m / sum_{m in S} w_m
+ *   Delta  = sum_{m in S} w^_m (Theta - theta_m)          (weighted direct averaging, Appendix)
+ *   v'     = outer_mu v + Delta
+ *   Theta' = Theta - outer_lr (Delta + outer_mu v')       (SGD with Nesterov momentum, Section 2)
+ *
+ * If |S| < max(K, 1) the record says DD_STATUS_QUORUM_NOT_MET and nothing else
+ * is written.  Buffers of learners outside S are never dereferenced (their
+ * pointers may be NULL or dangling, their contents NaN).
+ *
+ *   global, momentum  [device] float32[n], in/out
+ *   learner_ptrs      [host]   M device pointers to learner_dtype[n]
+ *   tokens, steps     [host]   uint64[M]; steps may be NULL; tokens[m] > 0 with
+ *                              steps[m] == 0 is DD_ERR_INVALID_ARG
+ *   quorum_mask       bit m = learner m reported in time (bits >= M ignored)
+ *   K                 minimum quorum, 0 <= K <= M (0 acts as 1)
+ *   out_bf16          [device] optional bf16[n]: round-to-nearest-even copy of
+ *                     Theta' (the payload broadcast back to the learners)
+ *   record            [device] optional; without it no diagnostics are computed
+ */
+int dd_merge_fragment(dd_ctx *ctx, float *global, float *momentum,
+                      const void *const *learner_ptrs, int M, dd_dtype learner_dtype,
+                      const uint64_t *tokens, const uint64_t *steps,
+                      uint64_t quorum_mask, int K, float outer_lr, float outer_mu,
+                      uint32_t flags, size_t n, void *out_bf16,
+                      dd_merge_record *record, void *cuda_stream);
+
+/*
+ * Many fragments in ONE kernel launch.  Fragments may differ in size, mask and
+ * counters (the counters are kept per learner and per fragment, Section 3.1);
+ * M, dtype, lr, mu and flags are shared.  Semantics per fragment are exactly
+ * those of dd_merge_fragment.  descs and the arrays it points to are host
+ * memory and are consumed before return.
+ */
+typedef struct {
+    float *global;                      /* [device] float32[n] in/out */
+    float *momentum;                    /* [device] float32[n] in/out */
+    void *out_bf16;                     /* [device] optional bf16[n] */
+    const void *const *learner_ptrs;    /* [host] M device pointers */
+    const uint64_t *tokens;             /* [host] uint64[M] */
+    const uint64_t *steps;              /* [host] uint64[M] or NULL */
+    uint64_t quorum_mask;
+    int32_t K;
+    uint64_t n;
+} dd_fragment_desc;
+
+int dd_merge_fragments_batched(dd_ctx *ctx, const dd_fragment_desc *descs, int P, int M,
+                               dd_dtype learner_dtype, float outer_lr, float outer_mu,
+                               uint32_t flags, dd_merge_record *records /* [device] P records or NULL */,
+                               void *cuda_stream);
+
+/*
+ * Quorum with grace window (Section 3.2, "Adaptive Quorum Window"), host only.
+ * arrival_s[m] is when learner m's report arrived (+inf = never).  The syncer
+ * may proceed at t_K, the K-th earliest arrival, and then waits grace_s longer:
+ * every learner with arrival <= t_K + grace_s is admitted.  Returns DD_OK and the
+ * mask, or DD_OK with *mask_out = 0 and *n_admitted = 0 when fewer than
+ * max(K,1) reports ever arrived.
+ */
+int dd_select_quorum(const double *arrival_s, int M, int K, double grace_s,
+                     uint64_t *mask_out, int *n_admitted);
+
+/*
+ * Largest admissible grace window: gamma * (tau * xi_step - (xi_quorum + xi_sync)),
+ * clamped at 0 (the slack equation of Section 3.2).
+ */
+double dd_grace_window(double tau, double xi_step, double xi_quorum, double xi_sync,
+                       double gamma);
+
+/* Text for a dd_error / the most recent CUDA error string seen by ctx. */
+const char *dd_status_string(int rc);
+const char *dd_last_cuda_error(const dd_ctx *ctx);
+
+/* Launch geometry chosen by the context (for reporting): CTAs, threads per CTA, elements per tile. */
+int dd_launch_geometry(const dd_ctx *ctx, dd_dtype learner_dtype, int *grid, int *block, int *tile);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DD_MERGE_H */

@@ -1,0 +1,59 @@
+// Host-only helpers of libddmerge: quorum / grace-window selection (Section 3.2,
+// "Adaptive Quorum Window") and status strings.  No CUDA here.
+#include <algorithm>
+#include <cmath>
+#include <vector>
+
+#include "dd_merge.h"
+
+extern "C" double dd_grace_window(double tau, double xi_step, double xi_quorum, double xi_sync,
+                                  double gamma)
+{
+    // xi_grace <= gamma * xi_slack with xi_slack = tau * xi_step - (xi_quorum + xi_sync);
+    // without slack the syncer proceeds as soon as the quorum is met.
+    const double slack = tau * xi_step - (xi_quorum + xi_sync);
+    return std::max(0.0, gamma * slack);
+}
+
+extern "C" int dd_select_quorum(const double *arrival_s, int M, int K, double grace_s,
+                                uint64_t *mask_out, int *n_admitted)
+{
+    if (!arrival_s || !mask_out || !n_admitted) return DD_ERR_INVALID_ARG;
+    if (M > DD_MAX_LEARNERS) return DD_ERR_TOO_MANY_LEARNERS;
+    if (M < 1 || K < 0 || K > M || !(grace_s >= 0.0)) return DD_ERR_INVALID_ARG;
+    *mask_out = 0;
+    *n_admitted = 0;
+    std::vector<double> seen;
+    seen.reserve((size_t)M);
+    for (int m = 0; m < M; ++m) {
+        if (std::isnan(arrival_s[m])) return DD_ERR_INVALID_ARG;
+        if (std::isfinite(arrival_s[m])) seen.push_back(arrival_s[m]);
+    }
+    const size_t need = (size_t)std::max(K, 1);
+    if (seen.size() < need) return DD_OK;                 // quorum never met: nobody admitted
+    // t_K: the moment the K-th report is in.  Everything that has arrived by
+    // t_K + grace takes part; ties at the deadline are admitted.
+    std::nth_element(seen.begin(), seen.begin() + (need - 1), seen.end());
+    const double deadline = seen[need - 1] + grace_s;
+    uint64_t mask = 0;
+    int count = 0;
+    for (int m = 0; m < M; ++m)
+        if (arrival_s[m] <= deadline) { mask |= 1ull << m; ++count; }
+    *mask_out = mask;
+    *n_admitted = count;
+    return DD_OK;
+}
+
+extern "C" const char *dd_status_string(int rc)
+{
+    switch (rc) {
+    case DD_OK: return "ok";
+    case DD_ERR_INVALID_ARG: return "invalid argument";
+    case DD_ERR_ALIGNMENT: return "device pointer not 16-byte aligned";
+    case DD_ERR_ALIAS: return "learner buffer overlaps the global fragment, the momentum or the bf16 output";
+    case DD_ERR_TOO_MANY_LEARNERS: return "more than DD_MAX_LEARNERS learners";
+    case DD_ERR_CUDA: return "CUDA runtime error (see dd_last_cuda_error)";
+    case DD_ERR_TOO_LARGE: return "size exceeds what this entry point supports";
+    default: return "unknown status";
+    }
+}

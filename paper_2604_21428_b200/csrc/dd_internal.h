@@ -1,0 +1,48 @@
+// Internal layout shared by the host launcher and the device code of libddmerge.
+// Not part of the public ABI.
+#pragma once
+
+#include <cstdint>
+
+#include "dd_merge.h"
+
+namespace ddm {
+
+constexpr int kThreads = 256;            // threads per CTA
+constexpr int kWarps = kThreads / 32;
+constexpr int kVec = 8;                  // elements one thread handles per step
+constexpr int kUnroll = 4;               // steps per tile
+constexpr int kTileElems = kThreads * kVec * kUnroll;   // 8192 elements per tile
+constexpr int kNumScalarDiag = 3;        // delta_sq, theta_sq, mom_sq
+
+// One fragment as the kernel sees it.  Raw counters, mask and pointers travel to
+// the device; participation and weights are derived there.
+struct alignas(16) DevFrag {
+    float *theta;
+    float *mom;
+    uint16_t *out_bf16;
+    unsigned long long n;
+    unsigned long long tile_begin;       // first flat tile index of this fragment
+    unsigned long long tile_end;         // one past its last tile (always > tile_begin)
+    unsigned long long mask;
+    int K;
+    int has_steps;
+    const void *ptrs[DD_MAX_LEARNERS];
+    unsigned long long tokens[DD_MAX_LEARNERS];
+    unsigned long long steps[DD_MAX_LEARNERS];
+};
+
+struct Common {
+    float eta;
+    float mu;
+    unsigned flags;
+    int M;
+    int P;
+    unsigned long long total_tiles;
+    dd_merge_record *records;            // device, nullable
+    double *partials;                    // [P][nq][grid] per-CTA partial sums
+    unsigned *tickets;                   // [P] completion counters, zero between calls
+    int nq;                              // quantities per fragment in `partials`
+};
+
+}  // namespace ddm

@@ -1,0 +1,386 @@
+// libddmerge: context, argument validation and launch of the fused merge kernel.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include <cuda_runtime.h>
+
+#include "dd_merge_kernel.cuh"
+
+namespace ddm {
+
+// 2 CTAs of 256 threads per SM -> up to 128 registers per thread.
+constexpr int kMinBlocksPerSM = 2;
+
+template <bool BF16, bool PL>
+__global__ void __launch_bounds__(kThreads, kMinBlocksPerSM)
+merge_single_kernel(const __grid_constant__ DevFrag frag, const __grid_constant__ Common c)
+{
+    merge_body<BF16, PL>(&frag, c);
+}
+
+template <bool BF16, bool PL>
+__global__ void __launch_bounds__(kThreads, kMinBlocksPerSM)
+merge_batched_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ Common c)
+{
+    merge_body<BF16, PL>(frags, c);
+}
+
+constexpr int kSlots = 4;   // descriptor staging ring (batched calls in flight)
+
+struct Slot {
+    DevFrag *host = nullptr;    // pinned
+    DevFrag *dev = nullptr;
+    size_t cap = 0;             // fragments
+    cudaEvent_t done = nullptr;
+    bool used = false;
+};
+
+}  // namespace ddm
+
+struct dd_ctx {
+    int device = 0;
+    int sm_count = 0;
+    int grid[2][2] = {{0, 0}, {0, 0}};        // [bf16][per-learner diag] persistent grid size
+    double *partials = nullptr;
+    size_t partials_cap = 0;                  // doubles
+    unsigned *tickets = nullptr;
+    size_t tickets_cap = 0;
+    ddm::Slot slots[ddm::kSlots];
+    int next_slot = 0;
+    char cuda_err[256] = {0};
+};
+
+namespace ddm {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard()
+    {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+static int cuda_fail(dd_ctx *ctx, cudaError_t e, const char *where)
+{
+    if (ctx) snprintf(ctx->cuda_err, sizeof ctx->cuda_err, "%s: %s", where, cudaGetErrorString(e));
+    (void)cudaGetLastError();
+    return DD_ERR_CUDA;
+}
+
+#define DD_CUDA(ctx, call)                                           \
+    do {                                                             \
+        cudaError_t e_ = (call);                                     \
+        if (e_ != cudaSuccess) return cuda_fail((ctx), e_, #call);   \
+    } while (0)
+
+template <bool BF16, bool PL>
+static cudaError_t occupancy(int *blocks)
+{
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+        blocks, merge_batched_kernel<BF16, PL>, kThreads, 0);
+    if (e != cudaSuccess) return e;
+    int b2 = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2, merge_single_kernel<BF16, PL>, kThreads, 0);
+    if (e == cudaSuccess && b2 < *blocks) *blocks = b2;
+    return e;
+}
+
+static bool overlaps(const void *a, size_t abytes, const void *b, size_t bbytes)
+{
+    if (!a || !b || abytes == 0 || bbytes == 0) return false;
+    const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+    return a0 < b0 + bbytes && b0 < a0 + abytes;
+}
+
+static bool misaligned(const void *p) { return ((uintptr_t)p & 15u) != 0; }
+
+// Validates one fragment and fills its device descriptor (tile range excluded).
+static int fill_fragment(DevFrag &d, float *global, float *momentum, void *out_bf16,
+                         const void *const *learner_ptrs, const uint64_t *tokens,
+                         const uint64_t *steps, uint64_t mask, int K, uint64_t n, int M,
+                         dd_dtype dtype)
+{
+    if (!learner_ptrs || !tokens) return DD_ERR_INVALID_ARG;
+    if (K < 0 || K > M) return DD_ERR_INVALID_ARG;
+    if (n > 0 && (!global || !momentum)) return DD_ERR_INVALID_ARG;
+    if (misaligned(global) || misaligned(momentum) || misaligned(out_bf16)) return DD_ERR_ALIGNMENT;
+    const size_t lb = (dtype == DD_BF16 ? 2u : 4u) * (size_t)n;
+    if (overlaps(global, 4 * n, momentum, 4 * n) || overlaps(global, 4 * n, out_bf16, 2 * n) ||
+        overlaps(momentum, 4 * n, out_bf16, 2 * n))
+        return DD_ERR_ALIAS;
+    std::memset(&d, 0, sizeof d);
+    d.theta = global;
+    d.mom = momentum;
+    d.out_bf16 = static_cast<uint16_t *>(out_bf16);
+    d.n = n;
+    d.mask = M >= 64 ? mask : (mask & ((1ull << M) - 1ull));
+    d.K = K;
+    d.has_steps = steps != nullptr;
+    for (int m = 0; m < M; ++m) {
+        d.tokens[m] = tokens[m];
+        d.steps[m] = steps ? steps[m] : 0;
+        d.ptrs[m] = learner_ptrs[m];
+        if (steps && tokens[m] > 0 && steps[m] == 0) return DD_ERR_INVALID_ARG;
+        const bool takes_part = ((d.mask >> m) & 1ull) && tokens[m] > 0;
+        if (takes_part && n > 0) {
+            const void *p = learner_ptrs[m];
+            if (!p) return DD_ERR_INVALID_ARG;
+            if (misaligned(p)) return DD_ERR_ALIGNMENT;
+            if (overlaps(p, lb, global, 4 * n) || overlaps(p, lb, momentum, 4 * n) ||
+                overlaps(p, lb, out_bf16, 2 * n))
+                return DD_ERR_ALIAS;
+        }
+    }
+    return DD_OK;
+}
+
+static unsigned long long tiles_of(uint64_t n)
+{
+    const unsigned long long t = (n + kTileElems - 1) / kTileElems;
+    return t ? t : 1;       // an empty fragment still owns one (empty) tile so its record is written
+}
+
+static int check_common(const dd_ctx *ctx, int M, dd_dtype dtype, float lr, float mu, uint32_t flags)
+{
+    if (!ctx) return DD_ERR_INVALID_ARG;
+    if (M > DD_MAX_LEARNERS) return DD_ERR_TOO_MANY_LEARNERS;
+    if (M < 1) return DD_ERR_INVALID_ARG;
+    if (dtype != DD_F32 && dtype != DD_BF16) return DD_ERR_INVALID_ARG;
+    if (!std::isfinite(lr) || !std::isfinite(mu)) return DD_ERR_INVALID_ARG;
+    if (flags & ~(uint32_t)(DD_HEAVY_BALL | DD_DIAG_PER_LEARNER | DD_DIAG_STATE)) return DD_ERR_INVALID_ARG;
+    return DD_OK;
+}
+
+// Grows the diagnostics workspace; growth waits for the device to drain because
+// kernels in flight may still use the old one.
+static int ensure_workspace(dd_ctx *ctx, size_t P, size_t nq, size_t grid)
+{
+    const size_t need = P * nq * grid;
+    if (need > ctx->partials_cap) {
+        DD_CUDA(ctx, cudaDeviceSynchronize());
+        if (ctx->partials) cudaFree(ctx->partials);
+        ctx->partials = nullptr;
+        ctx->partials_cap = 0;
+        DD_CUDA(ctx, cudaMalloc(&ctx->partials, need * sizeof(double)));
+        ctx->partials_cap = need;
+    }
+    if (P > ctx->tickets_cap) {
+        DD_CUDA(ctx, cudaDeviceSynchronize());
+        if (ctx->tickets) cudaFree(ctx->tickets);
+        ctx->tickets = nullptr;
+        ctx->tickets_cap = 0;
+        const size_t cap = P < 64 ? 64 : P;
+        DD_CUDA(ctx, cudaMalloc(&ctx->tickets, cap * sizeof(unsigned)));
+        DD_CUDA(ctx, cudaMemset(ctx->tickets, 0, cap * sizeof(unsigned)));
+        ctx->tickets_cap = cap;
+    }
+    return DD_OK;
+}
+
+template <bool BF16, bool PL>
+static cudaError_t launch(bool single, const DevFrag *one, const DevFrag *dev_frags,
+                          const Common &c, unsigned grid, cudaStream_t stream)
+{
+    if (single)
+        merge_single_kernel<BF16, PL><<<grid, kThreads, 0, stream>>>(*one, c);
+    else
+        merge_batched_kernel<BF16, PL><<<grid, kThreads, 0, stream>>>(dev_frags, c);
+    return cudaGetLastError();
+}
+
+static cudaError_t dispatch(bool bf16, bool pl, bool single, const DevFrag *one,
+                            const DevFrag *dev_frags, const Common &c, unsigned grid,
+                            cudaStream_t stream)
+{
+    if (bf16) return pl ? launch<true, true>(single, one, dev_frags, c, grid, stream)
+                        : launch<true, false>(single, one, dev_frags, c, grid, stream);
+    return pl ? launch<false, true>(single, one, dev_frags, c, grid, stream)
+              : launch<false, false>(single, one, dev_frags, c, grid, stream);
+}
+
+}  // namespace ddm
+
+using namespace ddm;
+
+extern "C" int dd_create(dd_ctx **out, int device)
+{
+    if (!out) return DD_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (device < 0 && cudaGetDevice(&device) != cudaSuccess) { (void)cudaGetLastError(); return DD_ERR_CUDA; }
+    dd_ctx *ctx = new (std::nothrow) dd_ctx();
+    if (!ctx) return DD_ERR_INVALID_ARG;
+    ctx->device = device;
+    DeviceGuard guard(device);
+    int rc = DD_OK;
+    cudaError_t e = guard.ok ? cudaSuccess : cudaErrorInvalidDevice;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
+    int occ[2][2] = {{0, 0}, {0, 0}};
+    if (e == cudaSuccess) e = occupancy<false, false>(&occ[0][0]);
+    if (e == cudaSuccess) e = occupancy<false, true>(&occ[0][1]);
+    if (e == cudaSuccess) e = occupancy<true, false>(&occ[1][0]);
+    if (e == cudaSuccess) e = occupancy<true, true>(&occ[1][1]);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        delete ctx;
+        return DD_ERR_CUDA;
+    }
+    for (int a = 0; a < 2; ++a)
+        for (int b = 0; b < 2; ++b) ctx->grid[a][b] = ctx->sm_count * (occ[a][b] > 0 ? occ[a][b] : 1);
+    *out = ctx;
+    return rc;
+}
+
+extern "C" int dd_destroy(dd_ctx *ctx)
+{
+    if (!ctx) return DD_OK;
+    DeviceGuard guard(ctx->device);
+    cudaDeviceSynchronize();
+    if (ctx->partials) cudaFree(ctx->partials);
+    if (ctx->tickets) cudaFree(ctx->tickets);
+    for (Slot &s : ctx->slots) {
+        if (s.host) cudaFreeHost(s.host);
+        if (s.dev) cudaFree(s.dev);
+        if (s.done) cudaEventDestroy(s.done);
+    }
+    (void)cudaGetLastError();
+    delete ctx;
+    return DD_OK;
+}
+
+extern "C" int dd_merge_fragment(dd_ctx *ctx, float *global, float *momentum,
+                                 const void *const *learner_ptrs, int M, dd_dtype learner_dtype,
+                                 const uint64_t *tokens, const uint64_t *steps,
+                                 uint64_t quorum_mask, int K, float outer_lr, float outer_mu,
+                                 uint32_t flags, size_t n, void *out_bf16,
+                                 dd_merge_record *record, void *cuda_stream)
+{
+    int rc = check_common(ctx, M, learner_dtype, outer_lr, outer_mu, flags);
+    if (rc != DD_OK) return rc;
+    DevFrag frag;
+    rc = fill_fragment(frag, global, momentum, out_bf16, learner_ptrs, tokens, steps, quorum_mask, K,
+                       n, M, learner_dtype);
+    if (rc != DD_OK) return rc;
+    if (n == 0 && record == nullptr) return DD_OK;
+    frag.tile_begin = 0;
+    frag.tile_end = tiles_of(n);
+
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
+    const bool bf16 = learner_dtype == DD_BF16, pl = (flags & DD_DIAG_PER_LEARNER) != 0;
+    unsigned long long g = (unsigned long long)ctx->grid[bf16][pl];
+    if (g > frag.tile_end) g = frag.tile_end;
+    Common c;
+    c.eta = outer_lr;
+    c.mu = outer_mu;
+    c.flags = flags;
+    c.M = M;
+    c.P = 1;
+    c.total_tiles = frag.tile_end;
+    c.records = record;
+    c.nq = kNumScalarDiag + (pl ? M : 0);
+    if (record) {
+        rc = ensure_workspace(ctx, 1, (size_t)c.nq, (size_t)ctx->grid[bf16][pl]);
+        if (rc != DD_OK) return rc;
+    }
+    c.partials = ctx->partials;
+    c.tickets = ctx->tickets;
+    cudaError_t e = dispatch(bf16, pl, true, &frag, nullptr, c, (unsigned)g, (cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "merge_single_kernel launch");
+    return DD_OK;
+}
+
+extern "C" int dd_merge_fragments_batched(dd_ctx *ctx, const dd_fragment_desc *descs, int P, int M,
+                                          dd_dtype learner_dtype, float outer_lr, float outer_mu,
+                                          uint32_t flags, dd_merge_record *records,
+                                          void *cuda_stream)
+{
+    int rc = check_common(ctx, M, learner_dtype, outer_lr, outer_mu, flags);
+    if (rc != DD_OK) return rc;
+    if (P < 0 || (P > 0 && !descs)) return DD_ERR_INVALID_ARG;
+    if (P > (1 << 20)) return DD_ERR_TOO_LARGE;
+    if (P == 0) return DD_OK;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
+
+    // Take the next staging slot; wait only if a call from kSlots calls ago still owns it.
+    Slot &slot = ctx->slots[ctx->next_slot];
+    if (slot.used) DD_CUDA(ctx, cudaEventSynchronize(slot.done));
+    if (!slot.done) DD_CUDA(ctx, cudaEventCreateWithFlags(&slot.done, cudaEventDisableTiming));
+    if ((size_t)P > slot.cap) {
+        if (slot.host) cudaFreeHost(slot.host);
+        if (slot.dev) cudaFree(slot.dev);
+        slot.host = nullptr;
+        slot.dev = nullptr;
+        slot.cap = 0;
+        const size_t cap = P < 32 ? 32 : (size_t)P;
+        DD_CUDA(ctx, cudaMallocHost(&slot.host, cap * sizeof(DevFrag)));
+        DD_CUDA(ctx, cudaMalloc(&slot.dev, cap * sizeof(DevFrag)));
+        slot.cap = cap;
+    }
+
+    unsigned long long tile = 0;
+    for (int p = 0; p < P; ++p) {
+        const dd_fragment_desc &d = descs[p];
+        rc = fill_fragment(slot.host[p], d.global, d.momentum, d.out_bf16, d.learner_ptrs, d.tokens,
+                           d.steps, d.quorum_mask, d.K, d.n, M, learner_dtype);
+        if (rc != DD_OK) return rc;
+        slot.host[p].tile_begin = tile;
+        tile += tiles_of(d.n);
+        slot.host[p].tile_end = tile;
+    }
+
+    const bool bf16 = learner_dtype == DD_BF16, pl = (flags & DD_DIAG_PER_LEARNER) != 0;
+    unsigned long long g = (unsigned long long)ctx->grid[bf16][pl];
+    if (g > tile) g = tile;
+    Common c;
+    c.eta = outer_lr;
+    c.mu = outer_mu;
+    c.flags = flags;
+    c.M = M;
+    c.P = P;
+    c.total_tiles = tile;
+    c.records = records;
+    c.nq = kNumScalarDiag + (pl ? M : 0);
+    if (records) {
+        rc = ensure_workspace(ctx, (size_t)P, (size_t)c.nq, (size_t)ctx->grid[bf16][pl]);
+        if (rc != DD_OK) return rc;
+    }
+    c.partials = ctx->partials;
+    c.tickets = ctx->tickets;
+
+    DD_CUDA(ctx, cudaMemcpyAsync(slot.dev, slot.host, (size_t)P * sizeof(DevFrag),
+                                 cudaMemcpyHostToDevice, stream));
+    cudaError_t e = dispatch(bf16, pl, false, nullptr, slot.dev, c, (unsigned)g, stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "merge_batched_kernel launch");
+    DD_CUDA(ctx, cudaEventRecord(slot.done, stream));
+    slot.used = true;
+    ctx->next_slot = (ctx->next_slot + 1) % kSlots;
+    return DD_OK;
+}
+
+extern "C" const char *dd_last_cuda_error(const dd_ctx *ctx)
+{
+    return ctx ? ctx->cuda_err : "";
+}
+
+extern "C" int dd_launch_geometry(const dd_ctx *ctx, dd_dtype learner_dtype, int *grid, int *block,
+                                  int *tile)
+{
+    if (!ctx || (learner_dtype != DD_F32 && learner_dtype != DD_BF16)) return DD_ERR_INVALID_ARG;
+    if (grid) *grid = ctx->grid[learner_dtype == DD_BF16][0];
+    if (block) *block = kThreads;
+    if (tile) *tile = kTileElems;
+    return DD_OK;
+}

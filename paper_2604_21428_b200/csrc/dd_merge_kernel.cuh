@@ -1,0 +1,446 @@
+// Fused per-fragment merge kernel (sm_100a): participation -> weights -> outer
+// gradients -> weighted reduce -> outer optimizer step -> norm diagnostics, one
+// pass over HBM.  Algorithm 2 steps 2-3 with the Weight function of Section 3.2
+// and the weighted direct-averaging merge of the "Merging methods" appendix.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "dd_internal.h"
+
+namespace ddm {
+
+struct Smem {
+    const void *ptr[DD_MAX_LEARNERS];    // participant j's buffer (compacted)
+    double wraw[DD_MAX_LEARNERS];        // raw weights, participant order
+    float w[DD_MAX_LEARNERS];            // normalised weights, participant order
+    unsigned char idx[DD_MAX_LEARNERS];  // participant j's learner id
+    float *theta;
+    float *mom;
+    uint16_t *out_bf16;
+    unsigned long long n;
+    unsigned long long tile_begin;
+    unsigned long long tile_end;
+    int n_part;
+    int status;
+    int frag;
+    int is_last;
+    double red[kWarps][kNumScalarDiag];
+    double dm[kWarps][DD_MAX_LEARNERS];  // per-warp per-participant ||Theta-theta_m||^2 partials
+};
+
+// ---- memory access helpers ---------------------------------------------------
+
+// Read-once streaming loads: evict-first so 30+ GB of learner data does not
+// push the (rewritten) state lines out of L2 before they are stored.
+__device__ __forceinline__ uint4 ld_stream16(const void *p)
+{
+    return __ldcs(reinterpret_cast<const uint4 *>(p));
+}
+
+__device__ __forceinline__ void st_stream16(void *p, uint4 v)
+{
+    __stcs(reinterpret_cast<uint4 *>(p), v);
+}
+
+// 8 consecutive floats starting at element 8*vi; `valid` < 8 only for the ragged
+// last step of a fragment (missing elements read as 0).
+__device__ __forceinline__ void load_f32x8(const float *base, unsigned long long vi, int valid,
+                                           float (&x)[8])
+{
+    if (valid == 8) {
+        const uint4 *p = reinterpret_cast<const uint4 *>(base) + 2 * vi;
+        uint4 a = ld_stream16(p), b = ld_stream16(p + 1);
+        x[0] = __uint_as_float(a.x); x[1] = __uint_as_float(a.y);
+        x[2] = __uint_as_float(a.z); x[3] = __uint_as_float(a.w);
+        x[4] = __uint_as_float(b.x); x[5] = __uint_as_float(b.y);
+        x[6] = __uint_as_float(b.z); x[7] = __uint_as_float(b.w);
+    } else {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) x[k] = k < valid ? base[8 * vi + k] : 0.0f;
+    }
+}
+
+__device__ __forceinline__ void store_f32x8(float *base, unsigned long long vi, int valid,
+                                            const float (&x)[8])
+{
+    if (valid == 8) {
+        uint4 *p = reinterpret_cast<uint4 *>(base) + 2 * vi;
+        st_stream16(p, make_uint4(__float_as_uint(x[0]), __float_as_uint(x[1]),
+                                  __float_as_uint(x[2]), __float_as_uint(x[3])));
+        st_stream16(p + 1, make_uint4(__float_as_uint(x[4]), __float_as_uint(x[5]),
+                                      __float_as_uint(x[6]), __float_as_uint(x[7])));
+    } else {
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            if (k < valid) base[8 * vi + k] = x[k];
+    }
+}
+
+// 8 consecutive bf16 as four 32-bit words (element 2k in the low half of word k).
+__device__ __forceinline__ uint4 load_bf16x8(const void *base, unsigned long long vi, int valid)
+{
+    if (valid == 8) return ld_stream16(reinterpret_cast<const uint4 *>(base) + vi);
+    const uint16_t *p = reinterpret_cast<const uint16_t *>(base) + 8 * vi;
+    unsigned h[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) h[k] = k < valid ? p[k] : 0u;
+    return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16),
+                      h[6] | (h[7] << 16));
+}
+
+__device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi)
+{
+    __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);     // cvt.rn.bf16x2.f32: .x = lo half
+    return *reinterpret_cast<unsigned *>(&b);
+}
+
+__device__ __forceinline__ void store_bf16x8(uint16_t *base, unsigned long long vi, int valid,
+                                             const float (&x)[8])
+{
+    uint4 v = make_uint4(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3]),
+                         pack_bf16x2(x[4], x[5]), pack_bf16x2(x[6], x[7]));
+    if (valid == 8) {
+        st_stream16(reinterpret_cast<uint4 *>(base) + vi, v);
+    } else {
+        const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            if (k < valid) base[8 * vi + k] = (uint16_t)(w[k >> 1] >> ((k & 1) * 16));
+    }
+}
+
+__device__ __forceinline__ double warp_sum(double x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+__device__ __forceinline__ float warp_sum(float x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+// ---- step 1-2: participation and weights, by warp 0 ---------------------------
+//
+// S = { m : mask bit m and tokens[m] > 0 } in ascending order (ballot + popc gives
+// each member its rank), quorum test |S| >= max(K,1), w = tokens (or
+// tokens^2/steps), w_hat = w / sum_S w.  Integer work is exact; the token sum is
+// an order-free uint64 butterfly, the tokens^2/steps sum is taken in rank order.
+__device__ __forceinline__ void load_header(const DevFrag *f, int p, unsigned long long tile,
+                                            const Common &c, Smem &sm)
+{
+    const int lane = threadIdx.x;                 // called by warp 0 only
+    const unsigned lt = (1u << lane) - 1u;
+    const int M = c.M;
+    const unsigned long long mask = f->mask;
+    const int m0 = lane, m1 = lane + 32;
+    const unsigned long long tok0 = m0 < M ? f->tokens[m0] : 0ull;
+    const unsigned long long tok1 = m1 < M ? f->tokens[m1] : 0ull;
+    const bool p0 = m0 < M && ((mask >> m0) & 1ull) && tok0 > 0;
+    const bool p1 = m1 < M && ((mask >> m1) & 1ull) && tok1 > 0;
+    const unsigned b0 = __ballot_sync(0xffffffffu, p0);
+    const unsigned b1 = __ballot_sync(0xffffffffu, p1);
+    const int c0 = __popc(b0);
+    const int n_part = c0 + __popc(b1);
+    const int j0 = __popc(b0 & lt), j1 = c0 + __popc(b1 & lt);
+
+    double w0 = 0.0, w1 = 0.0, W;
+    if (!f->has_steps) {
+        unsigned long long sum = (p0 ? tok0 : 0ull) + (p1 ? tok1 : 0ull);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        W = (double)sum;
+        w0 = (double)tok0;
+        w1 = (double)tok1;
+    } else {
+        if (p0) { double t = (double)tok0; w0 = t * t / (double)f->steps[m0]; sm.wraw[j0] = w0; }
+        if (p1) { double t = (double)tok1; w1 = t * t / (double)f->steps[m1]; sm.wraw[j1] = w1; }
+        __syncwarp();
+        W = 0.0;
+        if (lane == 0)
+            for (int j = 0; j < n_part; ++j) W += sm.wraw[j];
+        W = __shfl_sync(0xffffffffu, W, 0);
+    }
+    const int Kmin = f->K > 1 ? f->K : 1;
+    const int status = n_part < Kmin ? DD_STATUS_QUORUM_NOT_MET
+                                     : (!(W > 0.0) ? DD_STATUS_ZERO_WEIGHT : DD_STATUS_OK);
+    if (p0) { sm.idx[j0] = (unsigned char)m0; sm.w[j0] = (float)(w0 / W); sm.ptr[j0] = f->ptrs[m0]; }
+    if (p1) { sm.idx[j1] = (unsigned char)m1; sm.w[j1] = (float)(w1 / W); sm.ptr[j1] = f->ptrs[m1]; }
+    if (lane == 0) {
+        sm.theta = f->theta;
+        sm.mom = f->mom;
+        sm.out_bf16 = f->out_bf16;
+        sm.n = f->n;
+        sm.tile_begin = f->tile_begin;
+        sm.tile_end = f->tile_end;
+        sm.n_part = n_part;
+        sm.status = status;
+        sm.frag = p;
+    }
+    for (int j = lane; j < kWarps * DD_MAX_LEARNERS; j += 32) (&sm.dm[0][0])[j] = 0.0;
+    __syncwarp();
+    // The CTA that owns the fragment's first tile publishes the header.
+    if (c.records != nullptr && tile == f->tile_begin) {
+        dd_merge_record *rec = c.records + p;
+        for (int j = lane; j < DD_MAX_LEARNERS; j += 32) {
+            const bool on = j < n_part && status == DD_STATUS_OK;
+            rec->idx[j] = j < n_part ? sm.idx[j] : (unsigned char)0;
+            rec->w_hat[j] = on ? sm.w[j] : 0.0f;
+            rec->delta_m_sq[j] = 0.0;
+        }
+        if (lane == 0) {
+            rec->status = status;
+            rec->n_part = n_part;
+            rec->w_total = status == DD_STATUS_QUORUM_NOT_MET ? 0.0 : W;
+            rec->delta_sq = 0.0;
+            rec->theta_sq = 0.0;
+            rec->mom_sq = 0.0;
+        }
+    }
+}
+
+// Smallest fragment index >= lo whose tile range ends after `tile`.
+__device__ __forceinline__ int find_frag(const DevFrag *frags, int lo, int P,
+                                         unsigned long long tile)
+{
+    int hi = P - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (tile < frags[mid].tile_end) hi = mid; else lo = mid + 1;
+    }
+    return lo;
+}
+
+// ---- steps 3-5 for 8 consecutive elements --------------------------------------
+// FULL: all 8 elements exist (the only case outside a fragment's ragged last step).
+template <bool BF16, bool PL, bool FULL>
+__device__ __forceinline__ void process_vec(Smem &sm, const Common &c, unsigned long long vi,
+                                            int valid_arg, double &a_delta, double &a_theta,
+                                            double &a_mom)
+{
+    constexpr int B = BF16 ? 8 : 4;              // learner loads issued back to back
+    const int valid = FULL ? 8 : valid_arg;
+    const int s = sm.n_part;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float T[8], V[8];
+    float2 nT[4], acc[4];
+    if (PL && valid == 0) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { T[k] = 0.0f; V[k] = 0.0f; }
+    } else {
+        load_f32x8(sm.theta, vi, valid, T);
+        load_f32x8(sm.mom, vi, valid, V);
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        nT[k] = make_float2(-T[2 * k], -T[2 * k + 1]);
+        acc[k] = make_float2(0.0f, 0.0f);
+    }
+
+    // acc = sum_j w_hat_j (theta_j - Theta) = -Delta.  The difference is formed
+    // FIRST (it is exact or nearly so when theta_j is close to Theta), then
+    // weighted: factoring Theta out of the sum would lose ~|Theta|/|Delta| ulps.
+    for (int j0 = 0; j0 < s; j0 += B) {
+        if (BF16) {
+            uint4 r[B];
+#pragma unroll
+            for (int b = 0; b < B; ++b)
+                if (j0 + b < s) {
+                    if (PL && valid == 0) r[b] = make_uint4(0u, 0u, 0u, 0u);
+                    else r[b] = load_bf16x8(sm.ptr[j0 + b], vi, valid);
+                }
+#pragma unroll
+            for (int b = 0; b < B; ++b)
+                if (j0 + b < s) {
+                    const float w = sm.w[j0 + b];
+                    const float2 w2 = make_float2(w, w);
+                    const unsigned word[4] = {r[b].x, r[b].y, r[b].z, r[b].w};
+                    float q = 0.0f;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float2 th = make_float2(__uint_as_float(word[k] << 16),
+                                                      __uint_as_float(word[k] & 0xffff0000u));
+                        const float2 d = __fadd2_rn(th, nT[k]);
+                        acc[k] = __ffma2_rn(w2, d, acc[k]);
+                        if (PL) q = fmaf(d.x, d.x, fmaf(d.y, d.y, q));
+                    }
+                    if (PL) {
+                        q = warp_sum(q);
+                        if (lane == 0) sm.dm[warp][j0 + b] += (double)q;
+                    }
+                }
+        } else {
+            float th[B][8];
+#pragma unroll
+            for (int b = 0; b < B; ++b)
+                if (j0 + b < s) {
+                    if (PL && valid == 0) {
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) th[b][k] = 0.0f;
+                    } else {
+                        load_f32x8(reinterpret_cast<const float *>(sm.ptr[j0 + b]), vi, valid, th[b]);
+                    }
+                }
+#pragma unroll
+            for (int b = 0; b < B; ++b)
+                if (j0 + b < s) {
+                    const float w = sm.w[j0 + b];
+                    const float2 w2 = make_float2(w, w);
+                    float q = 0.0f;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float2 d = __fadd2_rn(make_float2(th[b][2 * k], th[b][2 * k + 1]), nT[k]);
+                        acc[k] = __ffma2_rn(w2, d, acc[k]);
+                        if (PL) q = fmaf(d.x, d.x, fmaf(d.y, d.y, q));
+                    }
+                    if (PL) {
+                        q = warp_sum(q);
+                        if (lane == 0) sm.dm[warp][j0 + b] += (double)q;
+                    }
+                }
+        }
+    }
+    if (PL && valid == 0) return;
+
+    // Outer step: v' = mu v + Delta; Theta' = Theta - eta (Delta + mu v') (Nesterov)
+    // or Theta - eta v' (heavy ball).
+    const float eta = c.eta, mu = c.mu;
+    const bool heavy = (c.flags & DD_HEAVY_BALL) != 0;
+    float Tn[8], Vn[8];
+    float dsq = 0.0f, tsq = 0.0f, msq = 0.0f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const float a = (k & 1) ? acc[k >> 1].y : acc[k >> 1].x;
+        const float delta = -a;
+        const float vn = fmaf(mu, V[k], delta);
+        const float u = heavy ? vn : fmaf(mu, vn, delta);
+        const float tn = fmaf(-eta, u, T[k]);
+        Vn[k] = vn;
+        Tn[k] = tn;
+        if (k < valid) {
+            dsq = fmaf(delta, delta, dsq);
+            tsq = fmaf(tn, tn, tsq);
+            msq = fmaf(vn, vn, msq);
+        }
+    }
+    store_f32x8(sm.mom, vi, valid, Vn);
+    store_f32x8(sm.theta, vi, valid, Tn);
+    if (sm.out_bf16 != nullptr) store_bf16x8(sm.out_bf16, vi, valid, Tn);
+    a_delta += (double)dsq;
+    if (c.flags & DD_DIAG_STATE) { a_theta += (double)tsq; a_mom += (double)msq; }
+}
+
+// ---- step 6: per-CTA partials, ticket, fixed-order final reduce ----------------
+//
+// Wait-free: every CTA that worked on the fragment stores its partial sums,
+// fences, and draws a ticket; the CTA that draws the last ticket adds the
+// partials in a fixed order (so the result does not depend on CTA timing) and
+// re-arms the ticket for the next call.
+template <bool PL>
+__device__ __forceinline__ void flush_fragment(Smem &sm, const Common &c, double &a_delta,
+                                               double &a_theta, double &a_mom)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned G = gridDim.x;
+    const int s = sm.n_part, p = sm.frag;
+    const int nq = c.nq;
+    double r0 = warp_sum(a_delta), r1 = warp_sum(a_theta), r2 = warp_sum(a_mom);
+    if (lane == 0) { sm.red[warp][0] = r0; sm.red[warp][1] = r1; sm.red[warp][2] = r2; }
+    a_delta = a_theta = a_mom = 0.0;
+    __syncthreads();
+    double *part = c.partials + (size_t)p * nq * G;
+    if (threadIdx.x < kNumScalarDiag) {
+        double t = 0.0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) t += sm.red[w][threadIdx.x];
+        part[(size_t)threadIdx.x * G + blockIdx.x] = t;
+        __threadfence();
+    } else if (PL && threadIdx.x >= 32 && threadIdx.x < 32 + s) {
+        const int j = threadIdx.x - 32;
+        double t = 0.0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) t += sm.dm[w][j];
+        part[(size_t)(kNumScalarDiag + j) * G + blockIdx.x] = t;
+        __threadfence();
+    }
+    __syncthreads();
+    const unsigned long long ntiles = sm.tile_end - sm.tile_begin;
+    if (threadIdx.x == 0) {
+        const unsigned expected = ntiles < G ? (unsigned)ntiles : G;
+        const unsigned ticket = atomicAdd(c.tickets + p, 1u);
+        sm.is_last = ticket == expected - 1u;
+    }
+    __syncthreads();
+    if (!sm.is_last) return;
+    __threadfence();
+    dd_merge_record *rec = c.records + p;
+    const unsigned first = (unsigned)(sm.tile_begin % G);
+    const int nq_used = kNumScalarDiag + (PL ? s : 0);
+    for (int q = warp; q < nq_used; q += kWarps) {
+        double t = 0.0;
+        for (unsigned cta = lane; cta < G; cta += 32) {
+            const unsigned off = cta >= first ? cta - first : cta + G - first;
+            if (off < ntiles) t += __ldcg(part + (size_t)q * G + cta);
+        }
+        t = warp_sum(t);
+        if (lane == 0) {
+            if (q == 0) rec->delta_sq = t;
+            else if (q == 1) rec->theta_sq = t;
+            else if (q == 2) rec->mom_sq = t;
+            else rec->delta_m_sq[q - kNumScalarDiag] = t;
+        }
+    }
+    if (threadIdx.x == 0) c.tickets[p] = 0u;
+}
+
+// ---- the kernel body ----------------------------------------------------------
+template <bool BF16, bool PL>
+__device__ __forceinline__ void merge_body(const DevFrag *frags, const Common &c)
+{
+    __shared__ Smem sm;
+    const unsigned G = gridDim.x;
+    double a_delta = 0.0, a_theta = 0.0, a_mom = 0.0;
+    int cur = -1;
+    bool loaded = false;
+
+    for (unsigned long long tile = blockIdx.x; tile < c.total_tiles; tile += G) {
+        if (!loaded || tile >= sm.tile_end) {                     // CTA-uniform
+            if (loaded && c.records != nullptr && sm.status == DD_STATUS_OK)
+                flush_fragment<PL>(sm, c, a_delta, a_theta, a_mom);
+            __syncthreads();
+            if (threadIdx.x < 32) {
+                cur = find_frag(frags, cur < 0 ? 0 : cur + 1, c.P, tile);
+                load_header(frags + cur, cur, tile, c, sm);
+            }
+            __syncthreads();
+            cur = sm.frag;
+            loaded = true;
+        }
+        if (sm.status != DD_STATUS_OK) continue;
+
+        const unsigned long long n = sm.n;
+        const unsigned long long nvec = (n + kVec - 1) / kVec;
+        const int rem = (int)(n % kVec);
+        const unsigned long long base = (tile - sm.tile_begin) * (unsigned long long)(kTileElems / kVec);
+#pragma unroll 1
+        for (int u = 0; u < kUnroll; ++u) {
+            const unsigned long long vi = base + (unsigned long long)u * kThreads + threadIdx.x;
+            if (vi - (threadIdx.x & 31) >= nvec) break;           // warp-uniform
+            const bool active = vi < nvec;
+            const int valid = !active ? 0 : ((rem != 0 && vi == nvec - 1) ? rem : kVec);
+            if (__all_sync(0xffffffffu, valid == kVec))
+                process_vec<BF16, PL, true>(sm, c, vi, kVec, a_delta, a_theta, a_mom);
+            else if (PL || active)
+                process_vec<BF16, PL, false>(sm, c, vi, valid, a_delta, a_theta, a_mom);
+        }
+    }
+    if (loaded && c.records != nullptr && sm.status == DD_STATUS_OK)
+        flush_fragment<PL>(sm, c, a_delta, a_theta, a_mom);
+}
+
+}  // namespace ddm

@@ -1,0 +1,268 @@
+"""ctypes binding of libddmerge (argument marshalling only).
+
+Every step of the merge runs in the CUDA library; this module turns torch
+tensors into raw device pointers, host lists into C arrays, and the device-side
+``dd_merge_record`` back into Python values.  There is no CPU fallback: if the
+library is missing or fails to load, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass, field
+
+MAX_LEARNERS = 64
+F32, BF16 = 0, 1
+OK = 0
+ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_ALIAS, ERR_TOO_MANY_LEARNERS, ERR_CUDA, ERR_TOO_LARGE = \
+    -1, -2, -3, -4, -5, -6
+STATUS_OK, STATUS_QUORUM_NOT_MET, STATUS_ZERO_WEIGHT, STATUS_WAIT_LIMIT = 0, 1, 2, 3
+HEAVY_BALL, DIAG_PER_LEARNER, DIAG_STATE = 1, 2, 4
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libddmerge.so")
+
+EXPORTS = (
+    "dd_create", "dd_destroy", "dd_merge_fragment", "dd_merge_fragments_batched",
+    "dd_select_quorum", "dd_grace_window", "dd_status_string", "dd_last_cuda_error",
+    "dd_launch_geometry",
+)
+
+
+class CRecord(ctypes.Structure):
+    """Mirror of ``dd_merge_record``."""
+    _fields_ = [
+        ("status", ctypes.c_int32),
+        ("n_part", ctypes.c_int32),
+        ("idx", ctypes.c_uint8 * MAX_LEARNERS),
+        ("w_hat", ctypes.c_float * MAX_LEARNERS),
+        ("w_total", ctypes.c_double),
+        ("delta_sq", ctypes.c_double),
+        ("theta_sq", ctypes.c_double),
+        ("mom_sq", ctypes.c_double),
+        ("delta_m_sq", ctypes.c_double * MAX_LEARNERS),
+    ]
+
+
+class CFragmentDesc(ctypes.Structure):
+    """Mirror of ``dd_fragment_desc``."""
+    _fields_ = [
+        ("global_", ctypes.c_void_p),
+        ("momentum", ctypes.c_void_p),
+        ("out_bf16", ctypes.c_void_p),
+        ("learner_ptrs", ctypes.POINTER(ctypes.c_void_p)),
+        ("tokens", ctypes.POINTER(ctypes.c_uint64)),
+        ("steps", ctypes.POINTER(ctypes.c_uint64)),
+        ("quorum_mask", ctypes.c_uint64),
+        ("K", ctypes.c_int32),
+        ("n", ctypes.c_uint64),
+    ]
+
+
+RECORD_BYTES = ctypes.sizeof(CRecord)
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2604_21428_b200.build` "
+            "(there is no CPU fallback)")
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, u64p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_uint64)
+    lib.dd_create.restype = ctypes.c_int
+    lib.dd_create.argtypes = [ctypes.POINTER(vp), ctypes.c_int]
+    lib.dd_destroy.restype = ctypes.c_int
+    lib.dd_destroy.argtypes = [vp]
+    lib.dd_merge_fragment.restype = ctypes.c_int
+    lib.dd_merge_fragment.argtypes = [
+        vp, vp, vp, ctypes.POINTER(vp), ctypes.c_int, ctypes.c_int, u64p, u64p, ctypes.c_uint64,
+        ctypes.c_int, ctypes.c_float, ctypes.c_float, ctypes.c_uint32, ctypes.c_size_t, vp, vp, vp]
+    lib.dd_merge_fragments_batched.restype = ctypes.c_int
+    lib.dd_merge_fragments_batched.argtypes = [
+        vp, ctypes.POINTER(CFragmentDesc), ctypes.c_int, ctypes.c_int, ctypes.c_int,
+        ctypes.c_float, ctypes.c_float, ctypes.c_uint32, vp, vp]
+    lib.dd_select_quorum.restype = ctypes.c_int
+    lib.dd_select_quorum.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.c_int,
+                                     ctypes.c_double, u64p, ctypes.POINTER(ctypes.c_int)]
+    lib.dd_grace_window.restype = ctypes.c_double
+    lib.dd_grace_window.argtypes = [ctypes.c_double] * 5
+    lib.dd_status_string.restype = ctypes.c_char_p
+    lib.dd_status_string.argtypes = [ctypes.c_int]
+    lib.dd_last_cuda_error.restype = ctypes.c_char_p
+    lib.dd_last_cuda_error.argtypes = [vp]
+    lib.dd_launch_geometry.restype = ctypes.c_int
+    lib.dd_launch_geometry.argtypes = [vp, ctypes.c_int] + [ctypes.POINTER(ctypes.c_int)] * 3
+    return lib
+
+
+lib = _load()
+
+
+class DDMergeError(RuntimeError):
+    def __init__(self, rc: int, detail: str = ""):
+        self.rc = rc
+        msg = lib.dd_status_string(rc).decode()
+        super().__init__(f"libddmerge: {msg} (rc={rc})" + (f": {detail}" if detail else ""))
+
+
+@dataclass
+class Record:
+    status: int
+    n_part: int
+    idx: list = field(default_factory=list)
+    w_hat: list = field(default_factory=list)      # float32 values
+    w_total: float = 0.0
+    delta_sq: float = 0.0
+    theta_sq: float = 0.0
+    mom_sq: float = 0.0
+    delta_m_sq: list = field(default_factory=list)
+
+
+def _ptr(x) -> int | None:
+    """Device/host address of a tensor-like, or the integer itself."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    return int(x.data_ptr())
+
+
+def _u64_array(values):
+    return (ctypes.c_uint64 * len(values))(*[int(v) for v in values])
+
+
+def _stream_handle(stream) -> int | None:
+    if stream is None:
+        import torch
+        return int(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, int):
+        return stream
+    return int(stream.cuda_stream)
+
+
+def new_records(count: int, device=None):
+    """Device buffer for ``count`` records (a uint8 torch tensor)."""
+    import torch
+    return torch.zeros(count * RECORD_BYTES, dtype=torch.uint8, device=device or "cuda")
+
+
+def read_records(buf, count: int | None = None) -> list:
+    """Copies the record buffer to the host (synchronises) and parses it."""
+    raw = bytes(buf.cpu().numpy().tobytes())
+    count = len(raw) // RECORD_BYTES if count is None else count
+    out = []
+    for p in range(count):
+        r = CRecord.from_buffer_copy(raw, p * RECORD_BYTES)
+        s = max(0, min(int(r.n_part), MAX_LEARNERS))
+        out.append(Record(status=int(r.status), n_part=int(r.n_part),
+                          idx=[int(r.idx[j]) for j in range(s)],
+                          w_hat=[float(r.w_hat[j]) for j in range(s)],
+                          w_total=float(r.w_total), delta_sq=float(r.delta_sq),
+                          theta_sq=float(r.theta_sq), mom_sq=float(r.mom_sq),
+                          delta_m_sq=[float(r.delta_m_sq[j]) for j in range(s)]))
+    return out
+
+
+class Context:
+    """Owns a ``dd_ctx`` (GPU binding + diagnostics workspace)."""
+
+    def __init__(self, device: int = -1):
+        handle = ctypes.c_void_p()
+        rc = lib.dd_create(ctypes.byref(handle), int(device))
+        if rc != OK:
+            raise DDMergeError(rc, "dd_create")
+        self._h = handle
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib.dd_destroy(self._h)
+            self._h = None
+
+    def __del__(self):  # best effort
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc: int):
+        if rc != OK:
+            detail = lib.dd_last_cuda_error(self._h).decode() if rc == ERR_CUDA else ""
+            raise DDMergeError(rc, detail)
+
+    def launch_geometry(self, dtype: int = BF16):
+        g, b, t = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+        self._check(lib.dd_launch_geometry(self._h, dtype, ctypes.byref(g), ctypes.byref(b),
+                                           ctypes.byref(t)))
+        return g.value, b.value, t.value
+
+    def merge_fragment(self, global_, momentum, learners, tokens, quorum_mask: int, K: int,
+                       outer_lr: float, outer_mu: float, *, n: int | None = None,
+                       learner_dtype: int | None = None, steps=None, flags: int = 0,
+                       out_bf16=None, record=None, stream=None) -> None:
+        """``dd_merge_fragment``: ``learners`` is a list of tensors / addresses / None."""
+        M = len(learners)
+        if n is None:
+            n = int(global_.numel())
+        if learner_dtype is None:
+            learner_dtype = _infer_dtype(learners)
+        ptrs = (ctypes.c_void_p * M)(*[_ptr(t) for t in learners])
+        self._check(lib.dd_merge_fragment(
+            self._h, _ptr(global_), _ptr(momentum), ptrs, M, learner_dtype, _u64_array(tokens),
+            None if steps is None else _u64_array(steps),
+            ctypes.c_uint64(quorum_mask & (2**64 - 1)), int(K), ctypes.c_float(outer_lr),
+            ctypes.c_float(outer_mu), ctypes.c_uint32(flags), ctypes.c_size_t(n), _ptr(out_bf16),
+            _ptr(record), _stream_handle(stream)))
+
+    def merge_fragments_batched(self, fragments, M: int, learner_dtype: int, outer_lr: float,
+                                outer_mu: float, *, flags: int = 0, records=None,
+                                stream=None) -> None:
+        """``dd_merge_fragments_batched``: ``fragments`` is a list of dicts with keys
+        global_, momentum, learners, tokens, quorum_mask, K, n and optionally
+        steps, out_bf16."""
+        P = len(fragments)
+        descs = (CFragmentDesc * max(P, 1))()
+        keep = []
+        for p, f in enumerate(fragments):
+            ptrs = (ctypes.c_void_p * M)(*[_ptr(t) for t in f["learners"]])
+            tok = _u64_array(f["tokens"])
+            stp = None if f.get("steps") is None else _u64_array(f["steps"])
+            keep += [ptrs, tok, stp]
+            d = descs[p]
+            d.global_ = _ptr(f["global_"])
+            d.momentum = _ptr(f["momentum"])
+            d.out_bf16 = _ptr(f.get("out_bf16"))
+            d.learner_ptrs = ptrs
+            d.tokens = tok
+            d.steps = stp if stp is not None else ctypes.POINTER(ctypes.c_uint64)()
+            d.quorum_mask = f["quorum_mask"] & (2**64 - 1)
+            d.K = int(f["K"])
+            d.n = int(f["n"])
+        self._check(lib.dd_merge_fragments_batched(
+            self._h, descs, P, M, learner_dtype, ctypes.c_float(outer_lr),
+            ctypes.c_float(outer_mu), ctypes.c_uint32(flags), _ptr(records),
+            _stream_handle(stream)))
+
+
+def _infer_dtype(learners) -> int:
+    import torch
+    for t in learners:
+        if t is not None and not isinstance(t, int):
+            return BF16 if t.dtype == torch.bfloat16 else F32
+    return BF16
+
+
+def select_quorum(arrival_s, K: int, grace_s: float):
+    """``dd_select_quorum``: returns (mask, n_admitted)."""
+    M = len(arrival_s)
+    arr = (ctypes.c_double * M)(*[float(a) for a in arrival_s])
+    mask, n_adm = ctypes.c_uint64(0), ctypes.c_int(0)
+    rc = lib.dd_select_quorum(arr, M, int(K), float(grace_s), ctypes.byref(mask),
+                              ctypes.byref(n_adm))
+    if rc != OK:
+        raise DDMergeError(rc)
+    return int(mask.value), int(n_adm.value)
+
+
+def grace_window(tau: float, xi_step: float, xi_quorum: float, xi_sync: float,
+                 gamma: float) -> float:
+    """``dd_grace_window``."""
+    return float(lib.dd_grace_window(tau, xi_step, xi_quorum, xi_sync, gamma))

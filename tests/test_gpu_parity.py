@@ -1,0 +1,324 @@
+"""GPU-vs-oracle parity through the C ABI (element by element, same seeded inputs)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2604_21428_b200 import synth
+from parity_util import (TOL_BF16, TOL_STATE, assert_record_matches, bf16_bits_to_f32,
+                         floor_rel_err, to_torch_learner)
+
+pytestmark = pytest.mark.gpu
+
+GUARD = 64          # canary elements on both sides of every output buffer
+ETA, MU = synth.OUTER_LR, synth.OUTER_MU
+
+
+@pytest.fixture(scope="module")
+def dd():
+    from paper_2604_21428_b200 import ddmerge
+    return ddmerge
+
+
+@pytest.fixture(scope="module")
+def ctx(dd):
+    c = dd.Context(0)
+    yield c
+    c.close()
+
+
+def _guarded(host: np.ndarray, dtype, device="cuda"):
+    """Device copy of ``host`` with NaN-free canaries around it; returns (full, view)."""
+    n = host.size
+    full = torch.full((n + 2 * GUARD,), 12345.0, dtype=dtype, device=device)
+    view = full[GUARD:GUARD + n]
+    if n:
+        view.copy_(torch.from_numpy(host).to(dtype))
+    return full, view
+
+
+def _check_guard(full, n):
+    assert torch.all(full[:GUARD] == 12345.0) and torch.all(full[GUARD + n:] == 12345.0), \
+        "write outside the output buffer"
+
+
+def run_case(dd, ctx, n, M, dtype, tokens, mask, K, *, seed=0, steps=None, flags=0, merges=2,
+             use_out=True, poison_absent=False, null_absent=False, eta=ETA, mu=MU):
+    theta, v, learners = synth.fragment_cpu(n, M, dtype, seed)
+    part = [m for m in range(M) if (mask >> m) & 1 and tokens[m] > 0]
+    if poison_absent:
+        for m in range(M):
+            if m not in part:
+                learners[m] = np.full_like(learners[m], 0x7fc0 if dtype == "bf16" else np.nan)
+    o_learners = list(learners)
+    if null_absent:
+        o_learners = [a if m in part else None for m, a in enumerate(learners)]
+    d_learners = [to_torch_learner(a, "cuda") for a in o_learners]
+    t_full, t_dev = _guarded(theta, torch.float32)
+    v_full, v_dev = _guarded(v, torch.float32)
+    out_full = out_dev = None
+    if use_out:
+        out_full, out_dev = _guarded(np.zeros(n, dtype=np.float32), torch.bfloat16)
+    rec_buf = dd.new_records(1)
+    heavy = bool(flags & dd.HEAVY_BALL)
+    for k in range(merges):
+        o_out = np.zeros(n, dtype=np.uint16) if use_out else None
+        ref = oracle.merge_fragment(theta, v, o_learners, tokens, mask, K, eta, mu, steps=steps,
+                                    nesterov=not heavy, out_bf16=o_out)
+        ctx.merge_fragment(t_dev, v_dev, d_learners, tokens, mask, K, eta, mu, n=n,
+                           learner_dtype=dd.BF16 if dtype == "bf16" else dd.F32, steps=steps,
+                           flags=flags, out_bf16=out_dev, record=rec_buf)
+        torch.cuda.synchronize()
+        got = dd.read_records(rec_buf)[0]
+        assert_record_matches(got, ref, diag_state=bool(flags & dd.DIAG_STATE),
+                              per_learner=bool(flags & dd.DIAG_PER_LEARNER))
+        e_t = floor_rel_err(t_dev.cpu().numpy(), theta)
+        e_v = floor_rel_err(v_dev.cpu().numpy(), v)
+        assert e_t <= TOL_STATE and e_v <= TOL_STATE, (k, e_t, e_v)
+        if use_out and ref.status == 0:
+            e_o = floor_rel_err(bf16_bits_to_f32(out_dev), oracle.bf16_to_f32(o_out))
+            assert e_o <= TOL_BF16, e_o
+            # identical except where the fp32 state differs by an ulp across a rounding boundary
+            same = np.mean(out_dev.cpu().view(torch.int16).numpy().view(np.uint16) == o_out) if n else 1.0
+            assert same > 0.999
+        _check_guard(t_full, n)
+        _check_guard(v_full, n)
+        if use_out:
+            _check_guard(out_full, n)
+        if ref.status != 0 and use_out:
+            assert torch.all(out_dev == 0)
+    return got
+
+
+def test_tiny_config(dd, ctx):
+    w = synth.workload("tiny")
+    run_case(dd, ctx, w.fragment_sizes[0], w.M, "f32", w.tokens[0].tolist(), w.masks[0], w.K,
+             seed=w.seed, flags=dd.DIAG_STATE | dd.DIAG_PER_LEARNER)
+
+
+@pytest.mark.parametrize("n", [0, 1, 7, 8, 9, 1023, 8192, 8193, 3 * 8192 + 5, (1 << 20) + 3])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_ragged_sizes(dd, ctx, n, dtype):
+    run_case(dd, ctx, n, 5, dtype, [100, 200, 0, 400, 500], 0b11101, 2, seed=n % 97,
+             flags=dd.DIAG_STATE | dd.DIAG_PER_LEARNER)
+
+
+@pytest.mark.parametrize("flags", [0, 1, 2, 4, 7])
+def test_flag_combinations(dd, ctx, flags):
+    run_case(dd, ctx, 50_000, 8, "bf16", [5, 6, 7, 8, 9, 10, 11, 12], 0b10110111, 3, seed=3,
+             flags=flags, merges=3)
+
+
+def test_no_record_no_output(dd, ctx):
+    n, M = 40_000, 3
+    theta, v, learners = synth.fragment_cpu(n, M, "bf16", 5)
+    t_dev, v_dev = torch.from_numpy(theta).cuda(), torch.from_numpy(v).cuda()
+    d_learners = [to_torch_learner(a, "cuda") for a in learners]
+    oracle.merge_fragment(theta, v, learners, [1, 2, 3], 0b111, 1, ETA, MU)
+    ctx.merge_fragment(t_dev, v_dev, d_learners, [1, 2, 3], 0b111, 1, ETA, MU)
+    torch.cuda.synchronize()
+    assert floor_rel_err(t_dev.cpu().numpy(), theta) <= TOL_STATE
+    assert floor_rel_err(v_dev.cpu().numpy(), v) <= TOL_STATE
+
+
+def test_dense150m_shape_scaled(dd, ctx):
+    # the 8-learner / 6-participant bf16 workload, one fragment at 1/400 of its size
+    w = synth.workload("dense150m")
+    n = w.fragment_sizes[0] // 400 + 3
+    rec = run_case(dd, ctx, n, w.M, "bf16", w.tokens[0].tolist(), w.masks[0], w.K, seed=w.seed,
+                   flags=dd.DIAG_STATE | dd.DIAG_PER_LEARNER, poison_absent=True)
+    assert rec.n_part == 6
+
+
+def test_scale_shape_scaled(dd, ctx):
+    # 32 learners, 24 participants (the steady-state workload) at reduced n
+    w = synth.workload("scale500m")
+    rec = run_case(dd, ctx, 300_007, w.M, "bf16", w.tokens[0].tolist(), w.masks[0], w.K,
+                   seed=w.seed, flags=dd.DIAG_STATE, null_absent=True)
+    assert rec.n_part == 24
+
+
+def test_masked_learners_are_never_read(dd, ctx):
+    # absent learners: NaN payloads, then null pointers
+    run_case(dd, ctx, 20_001, 6, "bf16", [9, 9, 0, 9, 9, 9], 0b101011, 2, seed=8, poison_absent=True)
+    run_case(dd, ctx, 20_001, 6, "f32", [9, 9, 0, 9, 9, 9], 0b101011, 2, seed=8, null_absent=True)
+
+
+def test_single_learner_and_sixty_four(dd, ctx):
+    run_case(dd, ctx, 10_000, 1, "bf16", [7], 1, 1, seed=1, flags=6)
+    tokens = list(range(1, 65))
+    run_case(dd, ctx, 9_001, 64, "bf16", tokens, (1 << 64) - 1, 64, seed=2, flags=6, merges=1)
+    rec = run_case(dd, ctx, 9_001, 64, "bf16", tokens, 1 << 63, 1, seed=2, flags=6, merges=1,
+                   null_absent=True)
+    assert rec.idx == [63]
+    tokens[40] = 0
+    rec = run_case(dd, ctx, 9_001, 64, "f32", tokens, ((1 << 64) - 1) ^ (1 << 5), 10, seed=2,
+                   flags=6, merges=1)
+    assert rec.n_part == 62 and 40 not in rec.idx and 5 not in rec.idx
+
+
+def test_quorum_not_met_and_zero_tokens(dd, ctx):
+    rec = run_case(dd, ctx, 5_000, 4, "bf16", [1, 2, 3, 4], 0b0011, 3, seed=4)
+    assert rec.status == dd.STATUS_QUORUM_NOT_MET and rec.n_part == 2
+    rec = run_case(dd, ctx, 5_000, 4, "bf16", [0, 0, 0, 0], 0b1111, 0, seed=4)
+    assert rec.status == dd.STATUS_QUORUM_NOT_MET and rec.n_part == 0
+
+
+def test_steps_weighting(dd, ctx):
+    tokens = [40960, 8192, 123456, 99999, 5]
+    steps = [10, 1, 33, 7, 5]
+    rec = run_case(dd, ctx, 30_011, 5, "bf16", tokens, 0b11111, 5, seed=6, steps=steps, flags=6)
+    raw = [t * (t / s) for t, s in zip(tokens, steps)]
+    assert math.isclose(rec.w_total, sum(raw), rel_tol=1e-12)
+
+
+def test_lr1_mu0_gives_weighted_mean(dd, ctx):
+    run_case(dd, ctx, 12_345, 4, "f32", [1000, 3000, 2000, 500], 0b1111, 4, seed=7, eta=1.0, mu=0.0)
+
+
+def test_nan_in_participant_propagates(dd, ctx):
+    n, M = 4_096 + 17, 3
+    theta, v, learners = synth.fragment_cpu(n, M, "bf16", 12)
+    learners[1][100] = 0x7fc0          # NaN
+    learners[2][200] = 0x7f80          # +Inf
+    t_dev, v_dev = torch.from_numpy(theta).cuda(), torch.from_numpy(v).cuda()
+    d_learners = [to_torch_learner(a, "cuda") for a in learners]
+    oracle.merge_fragment(theta, v, learners, [1, 2, 3], 0b111, 1, ETA, MU)
+    ctx.merge_fragment(t_dev, v_dev, d_learners, [1, 2, 3], 0b111, 1, ETA, MU)
+    torch.cuda.synchronize()
+    assert floor_rel_err(t_dev.cpu().numpy(), theta) <= TOL_STATE
+    assert floor_rel_err(v_dev.cpu().numpy(), v) <= TOL_STATE
+    assert np.isnan(theta[100]) and np.isinf(theta[200])
+
+
+def _batched_case(dd, ctx, sizes, M, dtype, tokens, masks, K, *, seed, flags, steps=None,
+                  merges=2):
+    P = len(sizes)
+    host, dev = [], []
+    for p, n in enumerate(sizes):
+        theta, v, learners = synth.fragment_cpu(n, M, dtype, seed * 1000 + p)
+        part = [m for m in range(M) if (masks[p] >> m) & 1 and int(tokens[p][m]) > 0]
+        o_learners = [a if m in part else None for m, a in enumerate(learners)]
+        host.append((theta, v, o_learners))
+        t_full, t_dev = _guarded(theta, torch.float32)
+        v_full, v_dev = _guarded(v, torch.float32)
+        o_full, o_dev = _guarded(np.zeros(n, dtype=np.float32), torch.bfloat16)
+        dev.append(dict(t_full=t_full, v_full=v_full, o_full=o_full, global_=t_dev, momentum=v_dev,
+                        out_bf16=o_dev, learners=[to_torch_learner(a, "cuda") for a in o_learners],
+                        tokens=[int(x) for x in tokens[p]], quorum_mask=masks[p], K=K, n=n,
+                        steps=None if steps is None else [int(x) for x in steps[p]]))
+    rec_buf = dd.new_records(P)
+    heavy = bool(flags & dd.HEAVY_BALL)
+    for k in range(merges):
+        ctx.merge_fragments_batched(dev, M, dd.BF16 if dtype == "bf16" else dd.F32, ETA, MU,
+                                    flags=flags, records=rec_buf)
+        torch.cuda.synchronize()
+        recs = dd.read_records(rec_buf)
+        for p, n in enumerate(sizes):
+            theta, v, o_learners = host[p]
+            o_out = np.zeros(n, dtype=np.uint16)
+            ref = oracle.merge_fragment(theta, v, o_learners, dev[p]["tokens"], masks[p], K, ETA,
+                                        MU, steps=dev[p]["steps"], nesterov=not heavy,
+                                        out_bf16=o_out)
+            assert_record_matches(recs[p], ref, diag_state=bool(flags & dd.DIAG_STATE),
+                                  per_learner=bool(flags & dd.DIAG_PER_LEARNER))
+            assert floor_rel_err(dev[p]["global_"].cpu().numpy(), theta) <= TOL_STATE, (k, p)
+            assert floor_rel_err(dev[p]["momentum"].cpu().numpy(), v) <= TOL_STATE, (k, p)
+            if ref.status == 0:
+                assert floor_rel_err(bf16_bits_to_f32(dev[p]["out_bf16"]),
+                                     oracle.bf16_to_f32(o_out)) <= TOL_BF16
+            for key in ("t_full", "v_full", "o_full"):
+                _check_guard(dev[p][key], n)
+    return recs
+
+
+def test_batched_ragged_mixed_status(dd, ctx):
+    rng = np.random.default_rng(5)
+    sizes = [8192 * 3 + 1, 0, 17, 100_000, 8192, 250_003, 5]
+    M = 6
+    tokens = rng.integers(0, 50, size=(len(sizes), M))
+    masks = [int(rng.integers(1, 1 << M)) for _ in sizes]
+    masks[3] = 0b000011                  # 2 participants at most: below K = 3
+    tokens[3] = [5, 5, 5, 5, 5, 5]
+    recs = _batched_case(dd, ctx, sizes, M, "bf16", tokens, masks, 3, seed=9,
+                         flags=dd.DIAG_STATE | dd.DIAG_PER_LEARNER)
+    assert recs[3].status == dd.STATUS_QUORUM_NOT_MET
+    assert any(r.status == 0 for r in recs)
+
+
+def test_batched_many_small_fragments(dd, ctx):
+    # more fragments than CTAs can each own: every CTA walks across several fragments
+    rng = np.random.default_rng(6)
+    P, M = 700, 4
+    sizes = [int(x) for x in rng.integers(1, 3000, size=P)]
+    tokens = rng.integers(1, 1000, size=(P, M))
+    steps = rng.integers(1, 9, size=(P, M))
+    masks = [int(rng.integers(1, 1 << M)) for _ in range(P)]
+    _batched_case(dd, ctx, sizes, M, "f32", tokens, masks, 1, seed=10, flags=dd.DIAG_STATE,
+                  steps=steps, merges=1)
+
+
+@pytest.mark.parametrize("name,factor", [("dense150m", 1 / 256), ("dense1b3", 1 / 2048),
+                                         ("moe4b", 1 / 4096)])
+def test_batched_workload_shapes_scaled(dd, ctx, name, factor):
+    w = synth.scaled(synth.workload(name), factor)
+    recs = _batched_case(dd, ctx, w.fragment_sizes, w.M, "bf16", w.tokens, w.masks, w.K,
+                         seed=w.seed, flags=dd.DIAG_STATE, merges=2)
+    for p, r in enumerate(recs):
+        assert r.status == 0 and r.n_part == w.participants(p)
+
+
+def test_back_to_back_calls_share_context(dd, ctx):
+    # many launches without host synchronisation in between (staging ring, tickets re-armed)
+    n, M = 70_001, 4
+    theta, v, learners = synth.fragment_cpu(n, M, "bf16", 21)
+    t_dev, v_dev = torch.from_numpy(theta).cuda(), torch.from_numpy(v).cuda()
+    d_learners = [to_torch_learner(a, "cuda") for a in learners]
+    rec_buf = dd.new_records(1)
+    frag = dict(global_=t_dev, momentum=v_dev, learners=d_learners, tokens=[4, 3, 2, 1],
+                quorum_mask=0b1111, K=4, n=n)
+    for k in range(12):
+        if k % 2:
+            ctx.merge_fragment(t_dev, v_dev, d_learners, [4, 3, 2, 1], 0b1111, 4, ETA, MU,
+                               flags=dd.DIAG_STATE, record=rec_buf)
+        else:
+            ctx.merge_fragments_batched([frag], M, dd.BF16, ETA, MU, flags=dd.DIAG_STATE,
+                                        records=rec_buf)
+        ref = oracle.merge_fragment(theta, v, learners, [4, 3, 2, 1], 0b1111, 4, ETA, MU)
+    torch.cuda.synchronize()
+    assert floor_rel_err(t_dev.cpu().numpy(), theta) <= TOL_STATE
+    assert floor_rel_err(v_dev.cpu().numpy(), v) <= TOL_STATE
+    assert_record_matches(dd.read_records(rec_buf)[0], ref, per_learner=False)
+
+
+def test_argument_validation(dd, ctx):
+    n, M = 1024, 3
+    t = torch.zeros(n, device="cuda")
+    v = torch.zeros(n, device="cuda")
+    L = [torch.zeros(n, device="cuda", dtype=torch.bfloat16) for _ in range(M)]
+
+    def rc_of(fn):
+        with pytest.raises(dd.DDMergeError) as e:
+            fn()
+        return e.value.rc
+
+    good = dict(n=n, learner_dtype=dd.BF16)
+    assert rc_of(lambda: ctx.merge_fragment(t, v, L, [1, 1, 1], 7, 4, ETA, MU, **good)) == dd.ERR_INVALID_ARG
+    assert rc_of(lambda: ctx.merge_fragment(t, v, L, [1, 1, 1], 7, -1, ETA, MU, **good)) == dd.ERR_INVALID_ARG
+    assert rc_of(lambda: ctx.merge_fragment(t, v, L, [1, 1, 1], 7, 1, float("nan"), MU, **good)) == dd.ERR_INVALID_ARG
+    assert rc_of(lambda: ctx.merge_fragment(t, v, L, [1, 1, 1], 7, 1, ETA, float("inf"), **good)) == dd.ERR_INVALID_ARG
+    assert rc_of(lambda: ctx.merge_fragment(t, v, [L[0], None, L[2]], [1, 1, 1], 7, 1, ETA, MU, **good)) == dd.ERR_INVALID_ARG
+    assert rc_of(lambda: ctx.merge_fragment(t, v, L, [1, 1, 1], 7, 1, ETA, MU, steps=[1, 0, 1], **good)) == dd.ERR_INVALID_ARG
+    assert rc_of(lambda: ctx.merge_fragment(t, v, L, [1, 1, 1], 7, 1, ETA, MU, flags=1 << 9, **good)) == dd.ERR_INVALID_ARG
+    assert rc_of(lambda: ctx.merge_fragment(t.data_ptr() + 4, v, L, [1, 1, 1], 7, 1, ETA, MU, n=n - 8, learner_dtype=dd.BF16)) == dd.ERR_ALIGNMENT
+    assert rc_of(lambda: ctx.merge_fragment(t, v, [L[0], L[1].data_ptr() + 2, L[2]], [1, 1, 1], 7, 1, ETA, MU, n=n - 8, learner_dtype=dd.BF16)) == dd.ERR_ALIGNMENT
+    assert rc_of(lambda: ctx.merge_fragment(t, t, L, [1, 1, 1], 7, 1, ETA, MU, **good)) == dd.ERR_ALIAS
+    assert rc_of(lambda: ctx.merge_fragment(t, v, [L[0], t, L[2]], [1, 1, 1], 7, 1, ETA, MU, **good)) == dd.ERR_ALIAS
+    assert rc_of(lambda: ctx.merge_fragment(t, v, L * 22, [1] * 66, 7, 1, ETA, MU, **good)) == dd.ERR_TOO_MANY_LEARNERS
+    # an absent learner may alias anything or be null: it is never touched
+    ctx.merge_fragment(t, v, [L[0], t, None], [1, 1, 1], 0b001, 1, ETA, MU, **good)
+    # the same learner buffer listed twice simply counts twice
+    ctx.merge_fragment(t, v, [L[0], L[0], L[1]], [1, 1, 1], 7, 1, ETA, MU, **good)
+    torch.cuda.synchronize()

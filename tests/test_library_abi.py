@@ -1,0 +1,93 @@
+"""The C-ABI library loads on a machine without a GPU, exports every symbol the
+header declares, and its host-only helpers agree with the oracle."""
+import math
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def dd():
+    from paper_2604_21428_b200 import build
+    build.build()
+    from paper_2604_21428_b200 import ddmerge
+    return ddmerge
+
+
+def _declared_functions():
+    names = []
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if not fn.endswith(".h"):
+            continue
+        text = open(os.path.join(ROOT, "include", fn)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names += re.findall(r"\b(dd_[a-z0-9_]+)\s*\(", text)
+    return sorted(set(names))
+
+
+def test_every_declared_symbol_is_exported(dd):
+    declared = _declared_functions()
+    assert "dd_merge_fragment" in declared and "dd_merge_fragments_batched" in declared
+    for name in declared:
+        assert hasattr(dd.lib, name), f"{name} declared in include/ but not exported"
+    assert set(dd.EXPORTS) <= set(declared)
+
+
+def test_record_layout_matches_header(dd):
+    # int32 x2, uint8[64], float[64], double x4, double[64]
+    assert dd.RECORD_BYTES == 8 + 64 + 256 + 32 + 512
+    assert dd.CRecord.w_hat.offset == 72 and dd.CRecord.w_total.offset == 328
+    assert dd.CRecord.delta_m_sq.offset == 360
+
+
+def test_status_strings(dd):
+    assert dd.lib.dd_status_string(0) == b"ok"
+    for rc in range(-6, 0):
+        assert dd.lib.dd_status_string(rc) not in (b"", b"unknown status")
+    assert dd.lib.dd_status_string(-99) == b"unknown status"
+
+
+def test_null_context_is_rejected_without_a_gpu(dd):
+    rc = dd.lib.dd_merge_fragment(None, None, None, None, 1, 0, None, None, 0, 0, 0.7, 0.9, 0, 0,
+                                  None, None, None)
+    assert rc == dd.ERR_INVALID_ARG
+    assert dd.lib.dd_destroy(None) == dd.OK
+
+
+def test_grace_window_matches_oracle_and_closed_form(dd):
+    rng = np.random.default_rng(0)
+    for _ in range(200):
+        tau, step, quorum, sync, gamma = rng.uniform(0, 3, 5)
+        got = dd.grace_window(tau, step, quorum, sync, gamma)
+        assert got == oracle.grace_window(tau, step, quorum, sync, gamma)
+        assert got == max(0.0, gamma * (tau * step - (quorum + sync)))
+
+
+def test_select_quorum_matches_oracle(dd):
+    rng = np.random.default_rng(1)
+    for _ in range(500):
+        M = int(rng.integers(1, 65))
+        arrival = np.round(rng.lognormal(0.0, 0.5, size=M), 1)       # ties are common
+        arrival[rng.random(M) < 0.15] = math.inf
+        K = int(rng.integers(0, M + 1))
+        grace = float(rng.choice([0.0, 0.1, 0.35, 2.0]))
+        st, mask, n_adm = oracle.select_quorum(arrival.tolist(), K, grace)
+        assert dd.select_quorum(arrival.tolist(), K, grace) == (mask, n_adm)
+        assert (st == 0) == (n_adm >= max(K, 1))
+
+
+def test_select_quorum_rejects_bad_input(dd):
+    with pytest.raises(dd.DDMergeError):
+        dd.select_quorum([0.0, float("nan")], 1, 0.0)
+    with pytest.raises(dd.DDMergeError):
+        dd.select_quorum([0.0, 1.0], 3, 0.0)
+    with pytest.raises(dd.DDMergeError):
+        dd.select_quorum([0.0, 1.0], 1, -1.0)
+    with pytest.raises(dd.DDMergeError):
+        dd.select_quorum([0.0] * 65, 1, 0.0)
