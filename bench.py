@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the fused per-fragment merge on B200.
+
+One "step" is one pass of the whole hot path -- participation, weights, outer
+gradients, weighted reduce, outer optimizer step, norm diagnostics -- over one
+synthetic workload (default: one 500M-parameter fragment, 32 bf16 learner
+copies of which 24 are in quorum, fp32 global + momentum).  Prints ONE JSON
+line on rank 0.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME]
+    python bench.py --impl reference      # the CPU oracle on a bounded sample
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "merged_params_per_sec"
+UNIT = "params/s"
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per merged parameter of the merge
+# kernel, from the ncu capture summarised under profiles/ (None until captured).
+NCU_TRAFFIC_BYTES_PER_PARAM = {"scale500m": None}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default="scale500m")
+    ap.add_argument("--scale", type=float, default=1.0, help="shrink every fragment (profiling)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample", type=int, default=1 << 25,
+                    help="elements of the workload the CPU oracle is timed on")
+    ap.add_argument("--out-bf16", action="store_true", help="also write the bf16 broadcast copy")
+    return ap.parse_args()
+
+
+# ---- clocks ------------------------------------------------------------------------
+
+_REASONS = {
+    0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap",
+    0x8: "hw_slowdown", 0x10: "sync_boost", 0x20: "sw_thermal_slowdown",
+    0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting",
+}
+
+
+class ClockSampler:
+    """Samples SM clock and clock-event reasons through NVML (read-only) in a thread."""
+
+    def __init__(self, device_index: int, period_s: float = 0.01):
+        self.period = period_s
+        self.samples, self.reason_bits = [], 0
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            try:
+                uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid).encode())
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                mhz = int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                try:
+                    bits = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                except Exception:
+                    bits = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                self.samples.append(mhz)
+                self.reason_bits |= bits & ~0x1
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        reasons = [name for bit, name in _REASONS.items() if self.reason_bits & bit]
+        return {"sm_mhz": int(statistics.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": reasons, "samples": len(self.samples)}
+
+
+# ---- measured peaks -----------------------------------------------------------------
+
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ---- the reference arm: the CPU oracle ------------------------------------------------
+
+def run_reference(args):
+    """Times the oracle, as it stands, on the host cores: each step is one merge of a
+    bounded sample (2^22 elements) of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+
+    import oracle
+    from paper_2604_21428_b200 import synth
+
+    w = synth.workload(args.workload)
+    sample = min(1 << 22, w.fragment_sizes[0])
+    p = 0
+    part = [m for m in range(w.M) if (w.masks[p] >> m) & 1 and int(w.tokens[p, m]) > 0]
+    theta, v, learners = synth.fragment_cpu(sample, w.M, w.learner_dtype, w.seed, present=part)
+    tokens = [int(x) for x in w.tokens[p]]
+    oracle.build()
+    for _ in range(min(args.warmup, 1)):
+        oracle.merge_fragment(theta, v, learners, tokens, w.masks[p], w.K, synth.OUTER_LR,
+                              synth.OUTER_MU)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.merge_fragment(theta, v, learners, tokens, w.masks[p], w.K, synth.OUTER_LR,
+                              synth.OUTER_MU)
+    dt = time.perf_counter() - t0
+    value = sample * args.steps / dt
+    sample_desc = (f"{sample} elements of fragment 0 of {w.name} per step, "
+                   f"{len(part)} participating {w.learner_dtype} learners, single thread")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": w.name, "sample_elements_per_step": sample, "M": w.M,
+                   "participants": len(part), "learner_dtype": w.learner_dtype},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": sample_desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---- our arm ---------------------------------------------------------------------------
+
+def build_workload(w, device, rank_seed, out_bf16):
+    """Allocates and fills every fragment of workload ``w`` on ``device``."""
+    import torch
+
+    from paper_2604_21428_b200 import synth
+
+    ldt = torch.bfloat16 if w.learner_dtype == "bf16" else torch.float32
+    frags = []
+    for p, n in enumerate(w.fragment_sizes):
+        theta = torch.empty(n, dtype=torch.float32, device=device)
+        mom = torch.empty(n, dtype=torch.float32, device=device)
+        learners = [torch.empty(n, dtype=ldt, device=device) for _ in range(w.M)]
+        synth.fill_fragment_gpu(theta, mom, learners, seed=w.seed * 1000 + p + 100000 * rank_seed)
+        out = torch.empty(n, dtype=torch.bfloat16, device=device) if out_bf16 else None
+        frags.append(dict(global_=theta, momentum=mom, learners=learners, out_bf16=out,
+                          tokens=[int(x) for x in w.tokens[p]], quorum_mask=w.masks[p], K=w.K, n=n))
+    return frags
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_2604_21428_b200 import ddmerge as dd
+    from paper_2604_21428_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    w = synth.workload(args.workload)
+    if args.scale != 1.0:
+        w = synth.scaled(w, args.scale, align=8)
+    frags = build_workload(w, device, rank, args.out_bf16)
+    ctx = dd.Context(local_rank)
+    grid, block, tile = ctx.launch_geometry(dd.BF16 if w.learner_dtype == "bf16" else dd.F32)
+    ldtype = dd.BF16 if w.learner_dtype == "bf16" else dd.F32
+    records = dd.new_records(w.P, device=device)
+    flags = dd.DIAG_STATE
+    eta, mu = synth.OUTER_LR, synth.OUTER_MU
+    stream = torch.cuda.current_stream()
+
+    def step():
+        if w.P == 1:
+            f = frags[0]
+            ctx.merge_fragment(f["global_"], f["momentum"], f["learners"], f["tokens"],
+                               f["quorum_mask"], f["K"], eta, mu, n=f["n"], learner_dtype=ldtype,
+                               flags=flags, out_bf16=f["out_bf16"], record=records, stream=stream)
+        else:
+            ctx.merge_fragments_batched(frags, w.M, ldtype, eta, mu, flags=flags, records=records,
+                                        stream=stream)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    recs = dd.read_records(records)
+    assert all(r.status == 0 for r in recs), [r.status for r in recs]
+
+    sampler = ClockSampler(local_rank)
+    events = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    events[0].record(stream)
+    for k in range(args.steps):
+        step()
+        events[k + 1].record(stream)
+    torch.cuda.synchronize()
+    sampler.stop()
+    if world > 1:
+        dist.barrier()
+    total_ms = events[0].elapsed_time(events[-1])
+    per_launch_ms = [events[k].elapsed_time(events[k + 1]) for k in range(args.steps)]
+    t = torch.tensor([total_ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    max_ms = float(t.item())
+
+    params_per_step = w.total_params
+    value = world * params_per_step * args.steps / (max_ms * 1e-3)
+    alg_bytes = w.algorithmic_bytes(out_bf16=args.out_bf16)
+    avg_launch_ms = sum(per_launch_ms) / len(per_launch_ms)
+    achieved = alg_bytes / (avg_launch_ms * 1e-3) / 1e9
+    peak, peak_kind = hbm_peak()
+    traffic_pp = NCU_TRAFFIC_BYTES_PER_PARAM.get(args.workload)
+    roofline = {
+        "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "frac": achieved / peak, "peak_source": f"of {peak_kind}",
+        "traffic": None if traffic_pp is None else traffic_pp * params_per_step,
+        "algorithmic_bytes_per_launch": alg_bytes,
+        "bytes_per_param": alg_bytes / params_per_step,
+        "kernel_ms": {"avg": avg_launch_ms, "median": statistics.median(per_launch_ms),
+                      "min": min(per_launch_ms), "max": max(per_launch_ms)},
+        "frac_of_nominal_8TBs": achieved / 8000.0,
+    }
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": max_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {
+            "workload": w.name, "fragments": w.P, "params_per_step": params_per_step, "M": w.M,
+            "participants": [w.participants(p) for p in range(w.P)],
+            "learner_dtype": w.learner_dtype, "state_dtype": "f32", "outer_lr": eta,
+            "outer_mu": mu, "flags": "nesterov+diag_state", "out_bf16": bool(args.out_bf16),
+            "grid": grid, "block": block, "tile_elems": tile,
+            "l2": "inputs larger than L2 (no flush)" if alg_bytes > 4 * 126e6 else "L2-resident",
+            "parallelism": f"replica x{world}" if world > 1 else "single",
+        },
+        "clocks": sampler.summary(),
+        "gpu_launches": args.steps,
+        "roofline": roofline,
+    }
+
+    # ---- end to end: host buffers through dd_merge_fragment_host -------------------
+    if not args.no_e2e and w.P == 1:
+        f = frags[0]
+        n = f["n"]
+        part = [m for m in range(w.M) if (f["quorum_mask"] >> m) & 1 and f["tokens"][m] > 0]
+        h_theta = torch.empty(n, dtype=torch.float32, pin_memory=True)
+        h_mom = torch.empty(n, dtype=torch.float32, pin_memory=True)
+        h_theta.copy_(f["global_"])
+        h_mom.copy_(f["momentum"])
+        h_learners = [None] * w.M
+        for m in part:
+            h_learners[m] = torch.empty(n, dtype=f["learners"][m].dtype, pin_memory=True)
+            h_learners[m].copy_(f["learners"][m])
+        esz = 2 if w.learner_dtype == "bf16" else 4
+        h2d = n * (len(part) * esz + 8)
+        d2h = n * 8 + dd.RECORD_BYTES
+        ctx.merge_fragment_host(h_theta, h_mom, h_learners, f["tokens"], f["quorum_mask"], f["K"],
+                                eta, mu, n=n, learner_dtype=ldtype, flags=flags)      # warm-up
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            rec = ctx.merge_fragment_host(h_theta, h_mom, h_learners, f["tokens"],
+                                          f["quorum_mask"], f["K"], eta, mu, n=n,
+                                          learner_dtype=ldtype, flags=flags)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        assert rec.status == 0
+        te = torch.tensor([dt], dtype=torch.float64, device=device)
+        if world > 1:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        line["e2e"] = {"value": world * n * args.e2e_steps / float(te.item()), "unit": UNIT,
+                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                       "steps": args.e2e_steps,
+                       "path": "dd_merge_fragment_host: pinned host buffers, chunked H2D -> "
+                               "kernel -> D2H pipeline, blocking"}
+        del h_learners, h_theta, h_mom
+    else:
+        line["e2e"] = None
+
+    # ---- the oracle on the host cores, bounded sample of the same workload -----------
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        f = frags[0]
+        ns = min(args.cpu_sample, f["n"])
+        part = [m for m in range(w.M) if (f["quorum_mask"] >> m) & 1 and f["tokens"][m] > 0]
+        theta = f["global_"][:ns].cpu().numpy()
+        mom = f["momentum"][:ns].cpu().numpy()
+        learners = [None] * w.M
+        for m in part:
+            t_m = f["learners"][m][:ns].cpu()
+            learners[m] = (t_m.view(torch.int16).numpy().view(np.uint16)
+                           if w.learner_dtype == "bf16" else t_m.numpy())
+        oracle.build()
+        t0 = time.perf_counter()
+        oracle.merge_fragment(theta, mom, learners, f["tokens"], f["quorum_mask"], f["K"], eta, mu)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {
+            "value": ns / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"first {ns} elements of fragment 0 of {w.name}, {len(part)} participating "
+                      f"{w.learner_dtype} learners, one merge, {dt:.1f} s, single thread of "
+                      f"{os.cpu_count()} host cores"}
+    elif rank == 0:
+        line["cpu_baseline"] = None
+
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -151,6 +151,31 @@ int dd_merge_fragments_batched(dd_ctx *ctx, const dd_fragment_desc *descs, int P
                                void *cuda_stream);
 
 /*
+ * The same update for a fragment whose operands live in HOST memory -- the
+ * paper's syncer pulls each learner's fragment from that learner's host RAM and
+ * keeps the global state off the accelerators (Section 4, system overview).
+ * The fragment is cut into chunks of chunk_elems elements (0 = library default,
+ * else a multiple of 8) that are pipelined through device staging buffers owned
+ * by the context: host-to-device copies, the fused kernel and device-to-host
+ * copies of successive chunks overlap.  Only copies of participating learners
+ * are transferred.
+ *
+ *   global, momentum, out_bf16, record, learner_ptrs[m]   all [host]; page-locked
+ *        memory is needed for the copies to run at full PCIe speed and to overlap.
+ *   The call first waits (on the device) for work already queued on cuda_stream,
+ *   and it BLOCKS the calling thread until the results are in host memory.
+ *   record (optional) is the record of the whole fragment: squared norms are
+ *   summed over the chunks in chunk order.
+ * Everything else is as in dd_merge_fragment.
+ */
+int dd_merge_fragment_host(dd_ctx *ctx, float *global, float *momentum,
+                           const void *const *learner_ptrs, int M, dd_dtype learner_dtype,
+                           const uint64_t *tokens, const uint64_t *steps,
+                           uint64_t quorum_mask, int K, float outer_lr, float outer_mu,
+                           uint32_t flags, size_t n, void *out_bf16,
+                           dd_merge_record *record, size_t chunk_elems, void *cuda_stream);
+
+/*
  * Quorum with grace window (Section 3.2, "Adaptive Quorum Window"), host only.
  * arrival_s[m] is when learner m's report arrived (+inf = never).  The syncer
  * may proceed at t_K, the K-th earliest arrival, and then waits grace_s longer:

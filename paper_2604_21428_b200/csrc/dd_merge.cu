@@ -28,60 +28,11 @@ merge_batched_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ 
     merge_body<BF16, PL>(frags, c);
 }
 
-constexpr int kSlots = 4;   // descriptor staging ring (batched calls in flight)
-
-struct Slot {
-    DevFrag *host = nullptr;    // pinned
-    DevFrag *dev = nullptr;
-    size_t cap = 0;             // fragments
-    cudaEvent_t done = nullptr;
-    bool used = false;
-};
-
 }  // namespace ddm
 
-struct dd_ctx {
-    int device = 0;
-    int sm_count = 0;
-    int grid[2][2] = {{0, 0}, {0, 0}};        // [bf16][per-learner diag] persistent grid size
-    double *partials = nullptr;
-    size_t partials_cap = 0;                  // doubles
-    unsigned *tickets = nullptr;
-    size_t tickets_cap = 0;
-    ddm::Slot slots[ddm::kSlots];
-    int next_slot = 0;
-    char cuda_err[256] = {0};
-};
+#include "dd_ctx.h"
 
 namespace ddm {
-
-struct DeviceGuard {
-    int prev = -1;
-    bool ok = true;
-    explicit DeviceGuard(int dev)
-    {
-        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
-        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
-    }
-    ~DeviceGuard()
-    {
-        int cur = -1;
-        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
-    }
-};
-
-static int cuda_fail(dd_ctx *ctx, cudaError_t e, const char *where)
-{
-    if (ctx) snprintf(ctx->cuda_err, sizeof ctx->cuda_err, "%s: %s", where, cudaGetErrorString(e));
-    (void)cudaGetLastError();
-    return DD_ERR_CUDA;
-}
-
-#define DD_CUDA(ctx, call)                                           \
-    do {                                                             \
-        cudaError_t e_ = (call);                                     \
-        if (e_ != cudaSuccess) return cuda_fail((ctx), e_, #call);   \
-    } while (0)
 
 template <bool BF16, bool PL>
 static cudaError_t occupancy(int *blocks)
@@ -247,6 +198,7 @@ extern "C" int dd_destroy(dd_ctx *ctx)
     cudaDeviceSynchronize();
     if (ctx->partials) cudaFree(ctx->partials);
     if (ctx->tickets) cudaFree(ctx->tickets);
+    host_pipe_destroy(ctx);
     for (Slot &s : ctx->slots) {
         if (s.host) cudaFreeHost(s.host);
         if (s.dev) cudaFree(s.dev);

@@ -23,6 +23,7 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libddmerge
 
 EXPORTS = (
     "dd_create", "dd_destroy", "dd_merge_fragment", "dd_merge_fragments_batched",
+    "dd_merge_fragment_host",
     "dd_select_quorum", "dd_grace_window", "dd_status_string", "dd_last_cuda_error",
     "dd_launch_geometry",
 )
@@ -80,6 +81,11 @@ def _load() -> ctypes.CDLL:
     lib.dd_merge_fragments_batched.argtypes = [
         vp, ctypes.POINTER(CFragmentDesc), ctypes.c_int, ctypes.c_int, ctypes.c_int,
         ctypes.c_float, ctypes.c_float, ctypes.c_uint32, vp, vp]
+    lib.dd_merge_fragment_host.restype = ctypes.c_int
+    lib.dd_merge_fragment_host.argtypes = [
+        vp, vp, vp, ctypes.POINTER(vp), ctypes.c_int, ctypes.c_int, u64p, u64p, ctypes.c_uint64,
+        ctypes.c_int, ctypes.c_float, ctypes.c_float, ctypes.c_uint32, ctypes.c_size_t, vp,
+        ctypes.POINTER(CRecord), ctypes.c_size_t, vp]
     lib.dd_select_quorum.restype = ctypes.c_int
     lib.dd_select_quorum.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.c_int,
                                      ctypes.c_double, u64p, ctypes.POINTER(ctypes.c_int)]
@@ -149,17 +155,17 @@ def read_records(buf, count: int | None = None) -> list:
     """Copies the record buffer to the host (synchronises) and parses it."""
     raw = bytes(buf.cpu().numpy().tobytes())
     count = len(raw) // RECORD_BYTES if count is None else count
-    out = []
-    for p in range(count):
-        r = CRecord.from_buffer_copy(raw, p * RECORD_BYTES)
-        s = max(0, min(int(r.n_part), MAX_LEARNERS))
-        out.append(Record(status=int(r.status), n_part=int(r.n_part),
-                          idx=[int(r.idx[j]) for j in range(s)],
-                          w_hat=[float(r.w_hat[j]) for j in range(s)],
-                          w_total=float(r.w_total), delta_sq=float(r.delta_sq),
-                          theta_sq=float(r.theta_sq), mom_sq=float(r.mom_sq),
-                          delta_m_sq=[float(r.delta_m_sq[j]) for j in range(s)]))
-    return out
+    return [_parse_record(CRecord.from_buffer_copy(raw, p * RECORD_BYTES)) for p in range(count)]
+
+
+def _parse_record(r: CRecord) -> Record:
+    s = max(0, min(int(r.n_part), MAX_LEARNERS))
+    return Record(status=int(r.status), n_part=int(r.n_part),
+                  idx=[int(r.idx[j]) for j in range(s)],
+                  w_hat=[float(r.w_hat[j]) for j in range(s)],
+                  w_total=float(r.w_total), delta_sq=float(r.delta_sq),
+                  theta_sq=float(r.theta_sq), mom_sq=float(r.mom_sq),
+                  delta_m_sq=[float(r.delta_m_sq[j]) for j in range(s)])
 
 
 class Context:
@@ -211,6 +217,29 @@ class Context:
             ctypes.c_uint64(quorum_mask & (2**64 - 1)), int(K), ctypes.c_float(outer_lr),
             ctypes.c_float(outer_mu), ctypes.c_uint32(flags), ctypes.c_size_t(n), _ptr(out_bf16),
             _ptr(record), _stream_handle(stream)))
+
+    def merge_fragment_host(self, global_, momentum, learners, tokens, quorum_mask: int, K: int,
+                            outer_lr: float, outer_mu: float, *, n: int | None = None,
+                            learner_dtype: int | None = None, steps=None, flags: int = 0,
+                            out_bf16=None, want_record: bool = True, chunk_elems: int = 0,
+                            stream=None):
+        """``dd_merge_fragment_host``: all tensors are HOST tensors (ideally pinned).
+        Blocks until the results are in host memory; returns the fragment's Record."""
+        M = len(learners)
+        if n is None:
+            n = int(global_.numel())
+        if learner_dtype is None:
+            learner_dtype = _infer_dtype(learners)
+        ptrs = (ctypes.c_void_p * M)(*[_ptr(t) for t in learners])
+        rec = CRecord()
+        self._check(lib.dd_merge_fragment_host(
+            self._h, _ptr(global_), _ptr(momentum), ptrs, M, learner_dtype, _u64_array(tokens),
+            None if steps is None else _u64_array(steps),
+            ctypes.c_uint64(quorum_mask & (2**64 - 1)), int(K), ctypes.c_float(outer_lr),
+            ctypes.c_float(outer_mu), ctypes.c_uint32(flags), ctypes.c_size_t(n), _ptr(out_bf16),
+            ctypes.byref(rec) if want_record else None, ctypes.c_size_t(chunk_elems),
+            _stream_handle(stream)))
+        return _parse_record(rec) if want_record else None
 
     def merge_fragments_batched(self, fragments, M: int, learner_dtype: int, outer_lr: float,
                                 outer_mu: float, *, flags: int = 0, records=None,
