@@ -176,6 +176,43 @@ int dd_merge_fragment_host(dd_ctx *ctx, float *global, float *momentum,
                            dd_merge_record *record, size_t chunk_elems, void *cuda_stream);
 
 /*
+ * The batched merge for callers that cannot allocate device memory.  (The paper
+ * has no counterpart to this entry point; it exists for deployment reasons only.)
+ *
+ * Some hosts of this library may not call cudaMalloc: a syncer living inside a
+ * training process whose framework allocator has already claimed nearly all of
+ * the GPU, a loop that cannot tolerate the device-wide synchronisation that
+ * cudaMalloc / cudaFree imply, or a service with a no-allocation-after-start-up
+ * rule.  This call takes no dd_ctx and calls neither cudaMalloc nor cudaFree nor
+ * any other allocating routine.  Its scratch memory (device copy of the fragment
+ * descriptors, per-CTA partial sums of the norm diagnostics, completion tickets)
+ * is a fixed array of DD_NOALLOC_SCRATCH_BYTES inside the library's device
+ * image; every GPU on which the library runs holds that array until the process
+ * exits.
+ *
+ * Semantics per fragment are those of dd_merge_fragments_batched, on the CURRENT
+ * device, with these limits:
+ *   - P <= DD_NOALLOC_MAX_FRAGMENTS, else DD_ERR_TOO_LARGE (nothing is launched);
+ *   - DD_DIAG_PER_LEARNER is not offered (DD_ERR_INVALID_ARG);
+ *   - the grid is capped at 592 CTAs.
+ * The first call on a device resolves the array's device address (one
+ * cudaGetSymbolAddress) and sizes the grid; make that first call before any
+ * stream capture begins.  All calls on a device share the one array, and it
+ * keeps the previous call's contents: the call itself clears what has to start
+ * at zero, but two calls that overlap on the GPU (different streams, or
+ * different host threads without ordering) race on it and give wrong results.
+ * Calls on one stream are safe back to back.  descs and the arrays it points to
+ * are host memory and are consumed before return; the call may wait for earlier
+ * work on cuda_stream while it hands the descriptors to the driver.
+ */
+#define DD_NOALLOC_MAX_FRAGMENTS 32
+#define DD_NOALLOC_SCRATCH_BYTES (512 * 1024)
+int dd_merge_fragments_batched_noalloc(const dd_fragment_desc *descs, int P, int M,
+                                       dd_dtype learner_dtype, float outer_lr, float outer_mu,
+                                       uint32_t flags, dd_merge_record *records /* [device] P records or NULL */,
+                                       void *cuda_stream);
+
+/*
  * Quorum with grace window (Section 3.2, "Adaptive Quorum Window"), host only.
  * arrival_s[m] is when learner m's report arrived (+inf = never).  The syncer
  * may proceed at t_K, the K-th earliest arrival, and then waits grace_s longer:

@@ -23,7 +23,7 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libddmerge
 
 EXPORTS = (
     "dd_create", "dd_destroy", "dd_merge_fragment", "dd_merge_fragments_batched",
-    "dd_merge_fragment_host",
+    "dd_merge_fragment_host", "dd_merge_fragments_batched_noalloc",
     "dd_select_quorum", "dd_grace_window", "dd_status_string", "dd_last_cuda_error",
     "dd_launch_geometry",
 )
@@ -86,6 +86,10 @@ def _load() -> ctypes.CDLL:
         vp, vp, vp, ctypes.POINTER(vp), ctypes.c_int, ctypes.c_int, u64p, u64p, ctypes.c_uint64,
         ctypes.c_int, ctypes.c_float, ctypes.c_float, ctypes.c_uint32, ctypes.c_size_t, vp,
         ctypes.POINTER(CRecord), ctypes.c_size_t, vp]
+    lib.dd_merge_fragments_batched_noalloc.restype = ctypes.c_int
+    lib.dd_merge_fragments_batched_noalloc.argtypes = [
+        ctypes.POINTER(CFragmentDesc), ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_float,
+        ctypes.c_float, ctypes.c_uint32, vp, vp]
     lib.dd_select_quorum.restype = ctypes.c_int
     lib.dd_select_quorum.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.c_int,
                                      ctypes.c_double, u64p, ctypes.POINTER(ctypes.c_int)]
@@ -248,27 +252,51 @@ class Context:
         global_, momentum, learners, tokens, quorum_mask, K, n and optionally
         steps, out_bf16."""
         P = len(fragments)
-        descs = (CFragmentDesc * max(P, 1))()
-        keep = []
-        for p, f in enumerate(fragments):
-            ptrs = (ctypes.c_void_p * M)(*[_ptr(t) for t in f["learners"]])
-            tok = _u64_array(f["tokens"])
-            stp = None if f.get("steps") is None else _u64_array(f["steps"])
-            keep += [ptrs, tok, stp]
-            d = descs[p]
-            d.global_ = _ptr(f["global_"])
-            d.momentum = _ptr(f["momentum"])
-            d.out_bf16 = _ptr(f.get("out_bf16"))
-            d.learner_ptrs = ptrs
-            d.tokens = tok
-            d.steps = stp if stp is not None else ctypes.POINTER(ctypes.c_uint64)()
-            d.quorum_mask = f["quorum_mask"] & (2**64 - 1)
-            d.K = int(f["K"])
-            d.n = int(f["n"])
+        descs, _keep = _pack_descs(fragments, M)
         self._check(lib.dd_merge_fragments_batched(
             self._h, descs, P, M, learner_dtype, ctypes.c_float(outer_lr),
             ctypes.c_float(outer_mu), ctypes.c_uint32(flags), _ptr(records),
             _stream_handle(stream)))
+
+
+def _pack_descs(fragments, M: int):
+    """Host-side ``dd_fragment_desc`` array for a list of fragment dicts."""
+    P = len(fragments)
+    descs = (CFragmentDesc * max(P, 1))()
+    keep = []
+    for p, f in enumerate(fragments):
+        ptrs = (ctypes.c_void_p * M)(*[_ptr(t) for t in f["learners"]])
+        tok = _u64_array(f["tokens"])
+        stp = None if f.get("steps") is None else _u64_array(f["steps"])
+        keep += [ptrs, tok, stp]
+        d = descs[p]
+        d.global_ = _ptr(f["global_"])
+        d.momentum = _ptr(f["momentum"])
+        d.out_bf16 = _ptr(f.get("out_bf16"))
+        d.learner_ptrs = ptrs
+        d.tokens = tok
+        d.steps = stp if stp is not None else ctypes.POINTER(ctypes.c_uint64)()
+        d.quorum_mask = f["quorum_mask"] & (2**64 - 1)
+        d.K = int(f["K"])
+        d.n = int(f["n"])
+    return descs, keep
+
+
+NOALLOC_MAX_FRAGMENTS = 32
+
+
+def merge_fragments_batched_noalloc(fragments, M: int, learner_dtype: int, outer_lr: float,
+                                    outer_mu: float, *, flags: int = 0, records=None,
+                                    stream=None) -> None:
+    """``dd_merge_fragments_batched_noalloc``: the batched merge on the current
+    device without a context and without any device allocation (at most
+    ``NOALLOC_MAX_FRAGMENTS`` fragments; calls must not overlap on the GPU)."""
+    descs, _keep = _pack_descs(fragments, M)
+    rc = lib.dd_merge_fragments_batched_noalloc(
+        descs, len(fragments), M, learner_dtype, ctypes.c_float(outer_lr),
+        ctypes.c_float(outer_mu), ctypes.c_uint32(flags), _ptr(records), _stream_handle(stream))
+    if rc != OK:
+        raise DDMergeError(rc)
 
 
 def _infer_dtype(learners) -> int:
