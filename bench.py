@@ -29,7 +29,7 @@ UNIT = "params/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per merged parameter of the merge
 # kernel, from the ncu capture summarised under profiles/ (None until captured).
-NCU_TRAFFIC_BYTES_PER_PARAM = {"scale500m": None}
+NCU_TRAFFIC_BYTES_PER_PARAM = {"scale500m": 62.84}
 
 
 def parse_args():
@@ -46,6 +46,9 @@ def parse_args():
     ap.add_argument("--cpu-sample", type=int, default=1 << 25,
                     help="elements of the workload the CPU oracle is timed on")
     ap.add_argument("--out-bf16", action="store_true", help="also write the bf16 broadcast copy")
+    ap.add_argument("--sharding", choices=["replica", "range"], default="replica",
+                    help="N>1: every rank merges its own copy of the workload (weak scaling), or "
+                         "each rank owns a contiguous element range of every fragment (strong)")
     return ap.parse_args()
 
 
@@ -204,6 +207,7 @@ def main():
     import torch.distributed as dist
 
     from paper_2604_21428_b200 import ddmerge as dd
+    from paper_2604_21428_b200 import dist as ddist
     from paper_2604_21428_b200 import synth
 
     rank = int(os.environ.get("RANK", "0"))
@@ -217,6 +221,10 @@ def main():
     w = synth.workload(args.workload)
     if args.scale != 1.0:
         w = synth.scaled(w, args.scale, align=8)
+    job_params = w.total_params * (world if args.sharding == "replica" else 1)
+    if args.sharding == "range" and world > 1:
+        w.fragment_sizes = [hi - lo for lo, hi in
+                            (ddist.shard_range(n, rank, world) for n in w.fragment_sizes)]
     frags = build_workload(w, device, rank, args.out_bf16)
     ctx = dd.Context(local_rank)
     grid, block, tile = ctx.launch_geometry(dd.BF16 if w.learner_dtype == "bf16" else dd.F32)
@@ -258,15 +266,13 @@ def main():
         dist.barrier()
     total_ms = events[0].elapsed_time(events[-1])
     per_launch_ms = [events[k].elapsed_time(events[k + 1]) for k in range(args.steps)]
-    t = torch.tensor([total_ms], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    max_ms = float(t.item())
+    max_ms = ddist.max_over_ranks(total_ms, device=device)
 
     params_per_step = w.total_params
-    value = world * params_per_step * args.steps / (max_ms * 1e-3)
+    value = ddist.whole_job_rate(job_params, args.steps, 1, max_ms)
     alg_bytes = w.algorithmic_bytes(out_bf16=args.out_bf16)
     avg_launch_ms = sum(per_launch_ms) / len(per_launch_ms)
+    slowest = sorted(range(len(per_launch_ms)), key=lambda k: -per_launch_ms[k])[:3]
     achieved = alg_bytes / (avg_launch_ms * 1e-3) / 1e9
     peak, peak_kind = hbm_peak()
     traffic_pp = NCU_TRAFFIC_BYTES_PER_PARAM.get(args.workload)
@@ -277,14 +283,16 @@ def main():
         "algorithmic_bytes_per_launch": alg_bytes,
         "bytes_per_param": alg_bytes / params_per_step,
         "kernel_ms": {"avg": avg_launch_ms, "median": statistics.median(per_launch_ms),
-                      "min": min(per_launch_ms), "max": max(per_launch_ms)},
+                      "min": min(per_launch_ms), "max": max(per_launch_ms),
+                      "slowest_steps": slowest},
         "frac_of_nominal_8TBs": achieved / 8000.0,
     }
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": max_ms / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "scaling": "weak" if args.sharding == "replica" else "strong", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
         "config": {
             "workload": w.name, "fragments": w.P, "params_per_step": params_per_step, "M": w.M,
             "participants": [w.participants(p) for p in range(w.P)],
@@ -292,7 +300,7 @@ def main():
             "outer_mu": mu, "flags": "nesterov+diag_state", "out_bf16": bool(args.out_bf16),
             "grid": grid, "block": block, "tile_elems": tile,
             "l2": "inputs larger than L2 (no flush)" if alg_bytes > 4 * 126e6 else "L2-resident",
-            "parallelism": f"replica x{world}" if world > 1 else "single",
+            "parallelism": f"{args.sharding} x{world}" if world > 1 else "single",
         },
         "clocks": sampler.summary(),
         "gpu_launches": args.steps,
@@ -328,10 +336,9 @@ def main():
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
         assert rec.status == 0
-        te = torch.tensor([dt], dtype=torch.float64, device=device)
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        line["e2e"] = {"value": world * n * args.e2e_steps / float(te.item()), "unit": UNIT,
+        dt_max = ddist.max_over_ranks(dt, device=device)
+        e2e_params = job_params            # every rank streams its own copy / its own range
+        line["e2e"] = {"value": e2e_params * args.e2e_steps / dt_max, "unit": UNIT,
                        "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                        "steps": args.e2e_steps,
                        "path": "dd_merge_fragment_host: pinned host buffers, chunked H2D -> "

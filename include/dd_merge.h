@@ -17,7 +17,9 @@
  *     the library allocates only its own context workspace.
  *   - Theta and v are float32 and are updated IN PLACE.  Learner copies are
  *     read-only, contiguous, all float32 or all bf16 (dd_dtype).
- *   - Device base pointers must be 16-byte aligned.  n is arbitrary.
+ *   - Device base pointers must be 16-byte aligned (32-byte aligned Theta and v
+ *     get 256-bit accesses).  n is arbitrary up to 2^34 elements per fragment
+ *     (DD_ERR_TOO_LARGE beyond).
  *   - Calls enqueue work on the given CUDA stream (a cudaStream_t passed as
  *     void*; NULL = the legacy default stream) and return without waiting.  Host
  *     arrays are consumed before the call returns.

@@ -14,6 +14,7 @@ constexpr int kVec = 8;                  // elements one thread handles per step
 constexpr int kUnroll = 4;               // steps per tile
 constexpr int kTileElems = kThreads * kVec * kUnroll;   // 8192 elements per tile
 constexpr int kNumScalarDiag = 3;        // delta_sq, theta_sq, mom_sq
+constexpr unsigned long long kMaxFragmentElems = 1ull << 34;   // 8-element steps are indexed in 32 bits
 
 // One fragment as the kernel sees it.  Raw counters, mask and pointers travel to
 // the device; participation and weights are derived there.

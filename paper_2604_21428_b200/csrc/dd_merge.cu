@@ -11,8 +11,11 @@
 
 namespace ddm {
 
-// 2 CTAs of 256 threads per SM -> up to 128 registers per thread.
-constexpr int kMinBlocksPerSM = 2;
+// Resident CTAs of 256 threads per SM the kernels are compiled for (2 -> 128 registers per thread).
+#ifndef DD_MIN_BLOCKS
+#define DD_MIN_BLOCKS 2
+#endif
+constexpr int kMinBlocksPerSM = DD_MIN_BLOCKS;
 
 template <bool BF16, bool PL>
 __global__ void __launch_bounds__(kThreads, kMinBlocksPerSM)
@@ -64,6 +67,7 @@ static int fill_fragment(DevFrag &d, float *global, float *momentum, void *out_b
     if (!learner_ptrs || !tokens) return DD_ERR_INVALID_ARG;
     if (K < 0 || K > M) return DD_ERR_INVALID_ARG;
     if (n > 0 && (!global || !momentum)) return DD_ERR_INVALID_ARG;
+    if (n > kMaxFragmentElems) return DD_ERR_TOO_LARGE;
     if (misaligned(global) || misaligned(momentum) || misaligned(out_bf16)) return DD_ERR_ALIGNMENT;
     const size_t lb = (dtype == DD_BF16 ? 2u : 4u) * (size_t)n;
     if (overlaps(global, 4 * n, momentum, 4 * n) || overlaps(global, 4 * n, out_bf16, 2 * n) ||

@@ -9,6 +9,14 @@
 
 #include "dd_internal.h"
 
+// Learner loads a thread issues back to back before it consumes them.
+#ifndef DD_BATCH_BF16
+#define DD_BATCH_BF16 8
+#endif
+#ifndef DD_BATCH_F32
+#define DD_BATCH_F32 4
+#endif
+
 namespace ddm {
 
 struct Smem {
@@ -26,14 +34,17 @@ struct Smem {
     int status;
     int frag;
     int is_last;
-    double red[kWarps][kNumScalarDiag];
-    double dm[kWarps][DD_MAX_LEARNERS];  // per-warp per-participant ||Theta-theta_m||^2 partials
+    int wide;                            // Theta and v are 32-byte aligned: 256-bit accesses
+    double red[kWarps][kNumScalarDiag];  // per-warp ||Delta||^2, ||Theta'||^2, ||v'||^2 of this fragment
+    double dm[kWarps][DD_MAX_LEARNERS];  // per-warp per-participant ||Theta-theta_m||^2
 };
 
 // ---- memory access helpers ---------------------------------------------------
+//
+// Every operand is read once and written once: loads and stores carry the
+// streaming (evict-first) hint so that 30+ GB of learner data does not displace
+// the state lines that are about to be rewritten.
 
-// Read-once streaming loads: evict-first so 30+ GB of learner data does not
-// push the (rewritten) state lines out of L2 before they are stored.
 __device__ __forceinline__ uint4 ld_stream16(const void *p)
 {
     return __ldcs(reinterpret_cast<const uint4 *>(p));
@@ -44,71 +55,47 @@ __device__ __forceinline__ void st_stream16(void *p, uint4 v)
     __stcs(reinterpret_cast<uint4 *>(p), v);
 }
 
-// 8 consecutive floats starting at element 8*vi; `valid` < 8 only for the ragged
-// last step of a fragment (missing elements read as 0).
-__device__ __forceinline__ void load_f32x8(const float *base, unsigned long long vi, int valid,
-                                           float (&x)[8])
+// 8 consecutive floats (32 bytes).  WIDE: one 256-bit access (needs a 32-byte
+// aligned address); otherwise two 128-bit accesses.
+template <bool WIDE>
+__device__ __forceinline__ void load_f32x8(const float *base, unsigned vi, float (&x)[8])
 {
-    if (valid == 8) {
-        const uint4 *p = reinterpret_cast<const uint4 *>(base) + 2 * vi;
-        uint4 a = ld_stream16(p), b = ld_stream16(p + 1);
+    const float *p = base + 8ull * vi;
+    if (WIDE) {
+        asm volatile("ld.global.cs.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=f"(x[0]), "=f"(x[1]), "=f"(x[2]), "=f"(x[3]), "=f"(x[4]), "=f"(x[5]),
+                       "=f"(x[6]), "=f"(x[7])
+                     : "l"(p));
+    } else {
+        const uint4 a = ld_stream16(p), b = ld_stream16(p + 4);
         x[0] = __uint_as_float(a.x); x[1] = __uint_as_float(a.y);
         x[2] = __uint_as_float(a.z); x[3] = __uint_as_float(a.w);
         x[4] = __uint_as_float(b.x); x[5] = __uint_as_float(b.y);
         x[6] = __uint_as_float(b.z); x[7] = __uint_as_float(b.w);
-    } else {
-#pragma unroll
-        for (int k = 0; k < 8; ++k) x[k] = k < valid ? base[8 * vi + k] : 0.0f;
     }
 }
 
-__device__ __forceinline__ void store_f32x8(float *base, unsigned long long vi, int valid,
-                                            const float (&x)[8])
+template <bool WIDE>
+__device__ __forceinline__ void store_f32x8(float *base, unsigned vi, const float (&x)[8])
 {
-    if (valid == 8) {
-        uint4 *p = reinterpret_cast<uint4 *>(base) + 2 * vi;
+    float *p = base + 8ull * vi;
+    if (WIDE) {
+        asm volatile("st.global.cs.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                     :: "l"(p), "f"(x[0]), "f"(x[1]), "f"(x[2]), "f"(x[3]), "f"(x[4]), "f"(x[5]),
+                        "f"(x[6]), "f"(x[7])
+                     : "memory");
+    } else {
         st_stream16(p, make_uint4(__float_as_uint(x[0]), __float_as_uint(x[1]),
                                   __float_as_uint(x[2]), __float_as_uint(x[3])));
-        st_stream16(p + 1, make_uint4(__float_as_uint(x[4]), __float_as_uint(x[5]),
+        st_stream16(p + 4, make_uint4(__float_as_uint(x[4]), __float_as_uint(x[5]),
                                       __float_as_uint(x[6]), __float_as_uint(x[7])));
-    } else {
-#pragma unroll
-        for (int k = 0; k < 8; ++k)
-            if (k < valid) base[8 * vi + k] = x[k];
     }
-}
-
-// 8 consecutive bf16 as four 32-bit words (element 2k in the low half of word k).
-__device__ __forceinline__ uint4 load_bf16x8(const void *base, unsigned long long vi, int valid)
-{
-    if (valid == 8) return ld_stream16(reinterpret_cast<const uint4 *>(base) + vi);
-    const uint16_t *p = reinterpret_cast<const uint16_t *>(base) + 8 * vi;
-    unsigned h[8];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) h[k] = k < valid ? p[k] : 0u;
-    return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16),
-                      h[6] | (h[7] << 16));
 }
 
 __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi)
 {
     __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);     // cvt.rn.bf16x2.f32: .x = lo half
     return *reinterpret_cast<unsigned *>(&b);
-}
-
-__device__ __forceinline__ void store_bf16x8(uint16_t *base, unsigned long long vi, int valid,
-                                             const float (&x)[8])
-{
-    uint4 v = make_uint4(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3]),
-                         pack_bf16x2(x[4], x[5]), pack_bf16x2(x[6], x[7]));
-    if (valid == 8) {
-        st_stream16(reinterpret_cast<uint4 *>(base) + vi, v);
-    } else {
-        const unsigned w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int k = 0; k < 8; ++k)
-            if (k < valid) base[8 * vi + k] = (uint16_t)(w[k >> 1] >> ((k & 1) * 16));
-    }
 }
 
 __device__ __forceinline__ double warp_sum(double x)
@@ -181,8 +168,10 @@ __device__ __forceinline__ void load_header(const DevFrag *f, int p, unsigned lo
         sm.n_part = n_part;
         sm.status = status;
         sm.frag = p;
+        sm.wide = (((unsigned long long)f->theta | (unsigned long long)f->mom) & 31ull) == 0;
     }
     for (int j = lane; j < kWarps * DD_MAX_LEARNERS; j += 32) (&sm.dm[0][0])[j] = 0.0;
+    if (lane < kWarps * kNumScalarDiag) (&sm.red[0][0])[lane] = 0.0;
     __syncwarp();
     // The CTA that owns the fragment's first tile publishes the header.
     if (c.records != nullptr && tile == f->tile_begin) {
@@ -217,24 +206,24 @@ __device__ __forceinline__ int find_frag(const DevFrag *frags, int lo, int P,
 }
 
 // ---- steps 3-5 for 8 consecutive elements --------------------------------------
-// FULL: all 8 elements exist (the only case outside a fragment's ragged last step).
-template <bool BF16, bool PL, bool FULL>
-__device__ __forceinline__ void process_vec(Smem &sm, const Common &c, unsigned long long vi,
-                                            int valid_arg, double &a_delta, double &a_theta,
-                                            double &a_mom)
+//
+// acc = sum_j w_hat_j (theta_j - Theta) = -Delta.  The difference is formed FIRST
+// (exact or nearly so when theta_j is close to Theta), then weighted: factoring
+// Theta out of the sum would lose ~|Theta|/|Delta| ulps.  `active` is false only
+// with per-learner diagnostics, where idle lanes still take part in the shuffles.
+template <bool BF16, bool PL, bool WIDE>
+__device__ __forceinline__ void process_vec(Smem &sm, const Common &c, unsigned vi, bool active,
+                                            float &dsq, float &tsq, float &msq)
 {
-    constexpr int B = BF16 ? 8 : 4;              // learner loads issued back to back
-    const int valid = FULL ? 8 : valid_arg;
+    constexpr int B = BF16 ? DD_BATCH_BF16 : DD_BATCH_F32;
     const int s = sm.n_part;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float T[8], V[8];
     float2 nT[4], acc[4];
-    if (PL && valid == 0) {
+    if (!PL || active) {
+        load_f32x8<WIDE>(sm.theta, vi, T);
+    } else {
 #pragma unroll
         for (int k = 0; k < 8; ++k) { T[k] = 0.0f; V[k] = 0.0f; }
-    } else {
-        load_f32x8(sm.theta, vi, valid, T);
-        load_f32x8(sm.mom, vi, valid, V);
     }
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
@@ -242,97 +231,120 @@ __device__ __forceinline__ void process_vec(Smem &sm, const Common &c, unsigned 
         acc[k] = make_float2(0.0f, 0.0f);
     }
 
-    // acc = sum_j w_hat_j (theta_j - Theta) = -Delta.  The difference is formed
-    // FIRST (it is exact or nearly so when theta_j is close to Theta), then
-    // weighted: factoring Theta out of the sum would lose ~|Theta|/|Delta| ulps.
+#pragma unroll 1
     for (int j0 = 0; j0 < s; j0 += B) {
-        if (BF16) {
-            uint4 r[B];
+        uint4 r[BF16 ? B : 2 * B];
 #pragma unroll
-            for (int b = 0; b < B; ++b)
-                if (j0 + b < s) {
-                    if (PL && valid == 0) r[b] = make_uint4(0u, 0u, 0u, 0u);
-                    else r[b] = load_bf16x8(sm.ptr[j0 + b], vi, valid);
+        for (int b = 0; b < B; ++b) {
+            if (j0 + b < s) {
+                if (PL && !active) {
+                    if (BF16) r[b] = make_uint4(0u, 0u, 0u, 0u);
+                    else r[2 * b] = r[2 * b + 1] = make_uint4(0u, 0u, 0u, 0u);
+                } else if (BF16) {
+                    r[b] = ld_stream16(reinterpret_cast<const uint4 *>(sm.ptr[j0 + b]) + vi);
+                } else {
+                    const uint4 *p = reinterpret_cast<const uint4 *>(sm.ptr[j0 + b]) + 2ull * vi;
+                    r[2 * b] = ld_stream16(p);
+                    r[2 * b + 1] = ld_stream16(p + 1);
                 }
+            }
+        }
+        // The momentum is needed only by the epilogue: fetch it behind the last batch.
+        if (j0 + B >= s && (!PL || active)) load_f32x8<WIDE>(sm.mom, vi, V);
 #pragma unroll
-            for (int b = 0; b < B; ++b)
-                if (j0 + b < s) {
-                    const float w = sm.w[j0 + b];
-                    const float2 w2 = make_float2(w, w);
+        for (int b = 0; b < B; ++b) {
+            if (j0 + b < s) {
+                const float w = sm.w[j0 + b];
+                const float2 w2 = make_float2(w, w);
+                float2 x[4];
+                if (BF16) {
+                    // element 2k sits in the low half of word k, element 2k+1 in the high half
                     const unsigned word[4] = {r[b].x, r[b].y, r[b].z, r[b].w};
-                    float q = 0.0f;
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const float2 th = make_float2(__uint_as_float(word[k] << 16),
-                                                      __uint_as_float(word[k] & 0xffff0000u));
-                        const float2 d = __fadd2_rn(th, nT[k]);
-                        acc[k] = __ffma2_rn(w2, d, acc[k]);
-                        if (PL) q = fmaf(d.x, d.x, fmaf(d.y, d.y, q));
-                    }
-                    if (PL) {
-                        q = warp_sum(q);
-                        if (lane == 0) sm.dm[warp][j0 + b] += (double)q;
-                    }
+                    for (int k = 0; k < 4; ++k)
+                        x[k] = make_float2(__uint_as_float(word[k] << 16),
+                                           __uint_as_float(word[k] & 0xffff0000u));
+                } else {
+                    x[0] = make_float2(__uint_as_float(r[2 * b].x), __uint_as_float(r[2 * b].y));
+                    x[1] = make_float2(__uint_as_float(r[2 * b].z), __uint_as_float(r[2 * b].w));
+                    x[2] = make_float2(__uint_as_float(r[2 * b + 1].x), __uint_as_float(r[2 * b + 1].y));
+                    x[3] = make_float2(__uint_as_float(r[2 * b + 1].z), __uint_as_float(r[2 * b + 1].w));
                 }
-        } else {
-            float th[B][8];
+                float q = 0.0f;
 #pragma unroll
-            for (int b = 0; b < B; ++b)
-                if (j0 + b < s) {
-                    if (PL && valid == 0) {
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) th[b][k] = 0.0f;
-                    } else {
-                        load_f32x8(reinterpret_cast<const float *>(sm.ptr[j0 + b]), vi, valid, th[b]);
-                    }
+                for (int k = 0; k < 4; ++k) {
+                    const float2 d = __fadd2_rn(x[k], nT[k]);
+                    acc[k] = __ffma2_rn(w2, d, acc[k]);
+                    if (PL) q = fmaf(d.x, d.x, fmaf(d.y, d.y, q));
                 }
-#pragma unroll
-            for (int b = 0; b < B; ++b)
-                if (j0 + b < s) {
-                    const float w = sm.w[j0 + b];
-                    const float2 w2 = make_float2(w, w);
-                    float q = 0.0f;
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const float2 d = __fadd2_rn(make_float2(th[b][2 * k], th[b][2 * k + 1]), nT[k]);
-                        acc[k] = __ffma2_rn(w2, d, acc[k]);
-                        if (PL) q = fmaf(d.x, d.x, fmaf(d.y, d.y, q));
-                    }
-                    if (PL) {
-                        q = warp_sum(q);
-                        if (lane == 0) sm.dm[warp][j0 + b] += (double)q;
-                    }
+                if (PL) {
+                    q = warp_sum(q);
+                    if ((threadIdx.x & 31) == 0) sm.dm[threadIdx.x >> 5][j0 + b] += (double)q;
                 }
+            }
         }
     }
-    if (PL && valid == 0) return;
+    if (PL && !active) return;
 
     // Outer step: v' = mu v + Delta; Theta' = Theta - eta (Delta + mu v') (Nesterov)
     // or Theta - eta v' (heavy ball).
     const float eta = c.eta, mu = c.mu;
     const bool heavy = (c.flags & DD_HEAVY_BALL) != 0;
-    float Tn[8], Vn[8];
-    float dsq = 0.0f, tsq = 0.0f, msq = 0.0f;
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-        const float a = (k & 1) ? acc[k >> 1].y : acc[k >> 1].x;
-        const float delta = -a;
+        const float delta = -((k & 1) ? acc[k >> 1].y : acc[k >> 1].x);
         const float vn = fmaf(mu, V[k], delta);
         const float u = heavy ? vn : fmaf(mu, vn, delta);
-        const float tn = fmaf(-eta, u, T[k]);
-        Vn[k] = vn;
-        Tn[k] = tn;
-        if (k < valid) {
-            dsq = fmaf(delta, delta, dsq);
-            tsq = fmaf(tn, tn, tsq);
-            msq = fmaf(vn, vn, msq);
+        const float tn = fmaf(-eta, u, -((k & 1) ? nT[k >> 1].y : nT[k >> 1].x));
+        V[k] = vn;
+        T[k] = tn;
+        dsq = fmaf(delta, delta, dsq);
+        tsq = fmaf(tn, tn, tsq);
+        msq = fmaf(vn, vn, msq);
+    }
+    store_f32x8<WIDE>(sm.mom, vi, V);
+    store_f32x8<WIDE>(sm.theta, vi, T);
+    if (sm.out_bf16 != nullptr)
+        st_stream16(reinterpret_cast<uint4 *>(sm.out_bf16) + vi,
+                    make_uint4(pack_bf16x2(T[0], T[1]), pack_bf16x2(T[2], T[3]),
+                               pack_bf16x2(T[4], T[5]), pack_bf16x2(T[6], T[7])));
+}
+
+// The ragged end of a fragment (n mod 8 elements), one element per lane of warp 0.
+template <bool BF16, bool PL>
+__device__ __forceinline__ void process_tail(Smem &sm, const Common &c, unsigned long long first,
+                                             int count, float &dsq, float &tsq, float &msq)
+{
+    const int lane = threadIdx.x & 31;
+    const bool active = lane < count;
+    const unsigned long long e = first + lane;
+    const int s = sm.n_part;
+    const float T = active ? sm.theta[e] : 0.0f;
+    float acc = 0.0f;
+    for (int j = 0; j < s; ++j) {
+        float th = 0.0f;
+        if (active) {
+            if (BF16) th = __uint_as_float((unsigned)reinterpret_cast<const uint16_t *>(sm.ptr[j])[e] << 16);
+            else th = reinterpret_cast<const float *>(sm.ptr[j])[e];
+        }
+        const float d = th - T;
+        acc = fmaf(sm.w[j], d, acc);
+        if (PL) {
+            const float q = warp_sum(d * d);
+            if (lane == 0) sm.dm[0][j] += (double)q;
         }
     }
-    store_f32x8(sm.mom, vi, valid, Vn);
-    store_f32x8(sm.theta, vi, valid, Tn);
-    if (sm.out_bf16 != nullptr) store_bf16x8(sm.out_bf16, vi, valid, Tn);
-    a_delta += (double)dsq;
-    if (c.flags & DD_DIAG_STATE) { a_theta += (double)tsq; a_mom += (double)msq; }
+    if (!active) return;
+    const float delta = -acc;
+    const float vn = fmaf(c.mu, sm.mom[e], delta);
+    const float u = (c.flags & DD_HEAVY_BALL) ? vn : fmaf(c.mu, vn, delta);
+    const float tn = fmaf(-c.eta, u, T);
+    sm.mom[e] = vn;
+    sm.theta[e] = tn;
+    if (sm.out_bf16 != nullptr) sm.out_bf16[e] = (uint16_t)(pack_bf16x2(tn, 0.0f) & 0xffffu);
+    dsq = fmaf(delta, delta, dsq);
+    tsq = fmaf(tn, tn, tsq);
+    msq = fmaf(vn, vn, msq);
 }
 
 // ---- step 6: per-CTA partials, ticket, fixed-order final reduce ----------------
@@ -342,16 +354,12 @@ __device__ __forceinline__ void process_vec(Smem &sm, const Common &c, unsigned 
 // partials in a fixed order (so the result does not depend on CTA timing) and
 // re-arms the ticket for the next call.
 template <bool PL>
-__device__ __forceinline__ void flush_fragment(Smem &sm, const Common &c, double &a_delta,
-                                               double &a_theta, double &a_mom)
+__device__ __forceinline__ void flush_fragment(Smem &sm, const Common &c)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const unsigned G = gridDim.x;
     const int s = sm.n_part, p = sm.frag;
     const int nq = c.nq;
-    double r0 = warp_sum(a_delta), r1 = warp_sum(a_theta), r2 = warp_sum(a_mom);
-    if (lane == 0) { sm.red[warp][0] = r0; sm.red[warp][1] = r1; sm.red[warp][2] = r2; }
-    a_delta = a_theta = a_mom = 0.0;
     __syncthreads();
     double *part = c.partials + (size_t)p * nq * G;
     if (threadIdx.x < kNumScalarDiag) {
@@ -390,12 +398,46 @@ __device__ __forceinline__ void flush_fragment(Smem &sm, const Common &c, double
         t = warp_sum(t);
         if (lane == 0) {
             if (q == 0) rec->delta_sq = t;
-            else if (q == 1) rec->theta_sq = t;
-            else if (q == 2) rec->mom_sq = t;
+            else if (q == 1) rec->theta_sq = (c.flags & DD_DIAG_STATE) ? t : 0.0;
+            else if (q == 2) rec->mom_sq = (c.flags & DD_DIAG_STATE) ? t : 0.0;
             else rec->delta_m_sq[q - kNumScalarDiag] = t;
         }
     }
     if (threadIdx.x == 0) c.tickets[p] = 0u;
+}
+
+// One tile (kTileElems elements of the current fragment).
+template <bool BF16, bool PL, bool WIDE>
+__device__ __forceinline__ void process_tile(Smem &sm, const Common &c, unsigned long long tile)
+{
+    constexpr unsigned kTileSteps = kTileElems / kVec;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned nfull = (unsigned)(sm.n / kVec);                       // whole 8-element steps
+    const unsigned base = (unsigned)(tile - sm.tile_begin) * kTileSteps;
+    const unsigned end = min(base + kTileSteps, nfull);
+    float dsq = 0.0f, tsq = 0.0f, msq = 0.0f;
+    if (PL) {
+        // per-learner norms are warp-wide sums: the whole warp walks together
+        for (unsigned v0 = base + warp * 32; v0 < end; v0 += kThreads)
+            process_vec<BF16, true, WIDE>(sm, c, v0 + lane, v0 + lane < end, dsq, tsq, msq);
+    } else {
+        for (unsigned vi = base + threadIdx.x; vi < end; vi += kThreads)
+            process_vec<BF16, false, WIDE>(sm, c, vi, true, dsq, tsq, msq);
+    }
+    const int rem = (int)(sm.n % kVec);
+    if (rem != 0 && tile == sm.tile_end - 1 && warp == 0)
+        process_tail<BF16, PL>(sm, c, (unsigned long long)nfull * kVec, rem, dsq, tsq, msq);
+    if (c.records != nullptr) {
+        // fp32 within a tile (at most 32 elements per thread), fp64 from here on
+        dsq = warp_sum(dsq);
+        tsq = warp_sum(tsq);
+        msq = warp_sum(msq);
+        if (lane == 0) {
+            sm.red[warp][0] += (double)dsq;
+            sm.red[warp][1] += (double)tsq;
+            sm.red[warp][2] += (double)msq;
+        }
+    }
 }
 
 // ---- the kernel body ----------------------------------------------------------
@@ -404,14 +446,12 @@ __device__ __forceinline__ void merge_body(const DevFrag *frags, const Common &c
 {
     __shared__ Smem sm;
     const unsigned G = gridDim.x;
-    double a_delta = 0.0, a_theta = 0.0, a_mom = 0.0;
     int cur = -1;
     bool loaded = false;
 
     for (unsigned long long tile = blockIdx.x; tile < c.total_tiles; tile += G) {
         if (!loaded || tile >= sm.tile_end) {                     // CTA-uniform
-            if (loaded && c.records != nullptr && sm.status == DD_STATUS_OK)
-                flush_fragment<PL>(sm, c, a_delta, a_theta, a_mom);
+            if (loaded && c.records != nullptr && sm.status == DD_STATUS_OK) flush_fragment<PL>(sm, c);
             __syncthreads();
             if (threadIdx.x < 32) {
                 cur = find_frag(frags, cur < 0 ? 0 : cur + 1, c.P, tile);
@@ -422,25 +462,10 @@ __device__ __forceinline__ void merge_body(const DevFrag *frags, const Common &c
             loaded = true;
         }
         if (sm.status != DD_STATUS_OK) continue;
-
-        const unsigned long long n = sm.n;
-        const unsigned long long nvec = (n + kVec - 1) / kVec;
-        const int rem = (int)(n % kVec);
-        const unsigned long long base = (tile - sm.tile_begin) * (unsigned long long)(kTileElems / kVec);
-#pragma unroll 1
-        for (int u = 0; u < kUnroll; ++u) {
-            const unsigned long long vi = base + (unsigned long long)u * kThreads + threadIdx.x;
-            if (vi - (threadIdx.x & 31) >= nvec) break;           // warp-uniform
-            const bool active = vi < nvec;
-            const int valid = !active ? 0 : ((rem != 0 && vi == nvec - 1) ? rem : kVec);
-            if (__all_sync(0xffffffffu, valid == kVec))
-                process_vec<BF16, PL, true>(sm, c, vi, kVec, a_delta, a_theta, a_mom);
-            else if (PL || active)
-                process_vec<BF16, PL, false>(sm, c, vi, valid, a_delta, a_theta, a_mom);
-        }
+        if (sm.wide) process_tile<BF16, PL, true>(sm, c, tile);
+        else process_tile<BF16, PL, false>(sm, c, tile);
     }
-    if (loaded && c.records != nullptr && sm.status == DD_STATUS_OK)
-        flush_fragment<PL>(sm, c, a_delta, a_theta, a_mom);
+    if (loaded && c.records != nullptr && sm.status == DD_STATUS_OK) flush_fragment<PL>(sm, c);
 }
 
 }  // namespace ddm

@@ -108,6 +108,7 @@ static int fill(DevFrag &d, const dd_fragment_desc &f, int M, dd_dtype dtype)
 {
     if (!f.learner_ptrs || !f.tokens || f.K < 0 || f.K > M) return DD_ERR_INVALID_ARG;
     if (f.n > 0 && (!f.global || !f.momentum)) return DD_ERR_INVALID_ARG;
+    if (f.n > kMaxFragmentElems) return DD_ERR_TOO_LARGE;
     if (misaligned(f.global) || misaligned(f.momentum) || misaligned(f.out_bf16)) return DD_ERR_ALIGNMENT;
     const size_t n = (size_t)f.n, lb = (dtype == DD_BF16 ? 2u : 4u) * n;
     if (overlaps(f.global, 4 * n, f.momentum, 4 * n) || overlaps(f.global, 4 * n, f.out_bf16, 2 * n) ||

@@ -1,0 +1,131 @@
+"""Parity at full workload sizes, in the launch configuration bench.py times.
+
+The oracle cannot run 5e8 x 24 elements in a test, so the CUDA result is checked
+(a) element by element on sampled windows whose inputs were copied out BEFORE the
+merge and fed to the oracle, and (b) through properties that hold at any size:
+participation and weights (data independent), and the squared norms against
+float64 reductions done with torch on the device.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2604_21428_b200 import synth
+from parity_util import TOL_NORM, TOL_STATE, floor_rel_err
+
+pytestmark = pytest.mark.gpu
+
+ETA, MU = synth.OUTER_LR, synth.OUTER_MU
+WINDOW = 1 << 16
+
+
+def _windows(n, count, rng):
+    """First, last and `count` random windows (8-element aligned starts)."""
+    if n <= 2 * WINDOW:
+        return [(0, n)]
+    starts = {0, n - WINDOW - (n - WINDOW) % 8}
+    while len(starts) < count + 2:
+        starts.add(int(rng.integers(0, (n - WINDOW) // 8)) * 8)
+    return [(s, s + WINDOW) for s in sorted(starts)]
+
+
+def _to_host_learner(t):
+    t = t.cpu()
+    if t.dtype == torch.bfloat16:
+        return t.view(torch.int16).numpy().view(np.uint16).copy()
+    return t.numpy().copy()
+
+
+def _expected_delta_sq(theta, learners, idx, w_hat, chunk=1 << 24):
+    """||sum_j w_j (Theta - theta_j)||^2 in float64 with torch, chunk by chunk."""
+    total = 0.0
+    n = theta.numel()
+    w = [float(x) for x in w_hat]
+    for lo in range(0, n, chunk):
+        hi = min(n, lo + chunk)
+        T = theta[lo:hi].double()
+        d = torch.zeros_like(T)
+        for j, m in enumerate(idx):
+            d += w[j] * (T - learners[m][lo:hi].double())
+        total += float((d * d).sum())
+    return total
+
+
+def _sq(t, chunk=1 << 26):
+    return sum(float((t[lo:lo + chunk].double() ** 2).sum()) for lo in range(0, t.numel(), chunk))
+
+
+def _run(name, n_windows, merges):
+    from paper_2604_21428_b200 import ddmerge as dd
+
+    w = synth.workload(name)
+    need = w.algorithmic_bytes() + 8 * w.total_params
+    free, _ = torch.cuda.mem_get_info()
+    if free < need + (4 << 30):
+        pytest.skip(f"needs {need >> 30} GiB of device memory, {free >> 30} GiB free")
+    dev = torch.device("cuda", 0)
+    ldt = torch.bfloat16 if w.learner_dtype == "bf16" else torch.float32
+    ldtype = dd.BF16 if w.learner_dtype == "bf16" else dd.F32
+    rng = np.random.default_rng(1234)
+    frags = []
+    for p, n in enumerate(w.fragment_sizes):
+        part = [m for m in range(w.M) if (w.masks[p] >> m) & 1 and int(w.tokens[p, m]) > 0]
+        theta = torch.empty(n, dtype=torch.float32, device=dev)
+        mom = torch.empty(n, dtype=torch.float32, device=dev)
+        learners = [torch.empty(n, dtype=ldt, device=dev) if m in part else None for m in range(w.M)]
+        synth.fill_fragment_gpu(theta, mom, learners, seed=w.seed * 1000 + p)
+        frags.append(dict(global_=theta, momentum=mom, learners=learners, part=part,
+                          tokens=[int(x) for x in w.tokens[p]], quorum_mask=w.masks[p], K=w.K, n=n,
+                          windows=_windows(n, n_windows, rng)))
+    ctx = dd.Context(0)
+    records = dd.new_records(w.P, device=dev)
+    flags = dd.DIAG_STATE
+    for k in range(merges):
+        # copy the sampled inputs out before the merge overwrites the state
+        saved = []
+        for f in frags:
+            per = []
+            for lo, hi in f["windows"]:
+                per.append((f["global_"][lo:hi].cpu().numpy().copy(),
+                            f["momentum"][lo:hi].cpu().numpy().copy(),
+                            [None if t is None else _to_host_learner(t[lo:hi]) for t in f["learners"]]))
+            saved.append(per)
+        st, idx0 = oracle.participants(frags[0]["quorum_mask"], frags[0]["tokens"], frags[0]["K"])
+        expect_dsq = None
+        if k == 0:
+            _, w0, _ = oracle.weights(frags[0]["tokens"], None, idx0)
+            expect_dsq = _expected_delta_sq(frags[0]["global_"], frags[0]["learners"], idx0,
+                                            [np.float32(x) for x in w0])
+        if w.P == 1:
+            f = frags[0]
+            ctx.merge_fragment(f["global_"], f["momentum"], f["learners"], f["tokens"],
+                               f["quorum_mask"], f["K"], ETA, MU, n=f["n"], learner_dtype=ldtype,
+                               flags=flags, record=records)
+        else:
+            ctx.merge_fragments_batched(frags, w.M, ldtype, ETA, MU, flags=flags, records=records)
+        torch.cuda.synchronize()
+        recs = dd.read_records(records)
+        for p, f in enumerate(frags):
+            rec = recs[p]
+            for (lo, hi), (t0, v0, ls) in zip(f["windows"], saved[p]):
+                ref = oracle.merge_fragment(t0, v0, ls, f["tokens"], f["quorum_mask"], f["K"], ETA, MU)
+                assert (rec.status, rec.n_part, rec.idx) == (ref.status, ref.n_part, ref.idx)
+                assert rec.w_hat == [float(np.float32(x)) for x in ref.w_hat]
+                e_t = floor_rel_err(f["global_"][lo:hi].cpu().numpy(), t0)
+                e_v = floor_rel_err(f["momentum"][lo:hi].cpu().numpy(), v0)
+                assert e_t <= TOL_STATE and e_v <= TOL_STATE, (k, p, lo, e_t, e_v)
+            assert rec.n_part == len(f["part"])
+            assert abs(rec.theta_sq - _sq(f["global_"])) <= TOL_NORM * rec.theta_sq
+            assert abs(rec.mom_sq - _sq(f["momentum"])) <= TOL_NORM * rec.mom_sq
+        if expect_dsq is not None:
+            assert abs(recs[0].delta_sq - expect_dsq) <= 1e-4 * expect_dsq, (recs[0].delta_sq, expect_dsq)
+    ctx.close()
+
+
+def test_scale500m_full_size_sampled():
+    _run("scale500m", n_windows=10, merges=2)
+
+
+def test_dense150m_full_size_batched_sampled():
+    _run("dense150m", n_windows=4, merges=2)

@@ -29,11 +29,12 @@ def ctx(dd):
     c.close()
 
 
-def _guarded(host: np.ndarray, dtype, device="cuda"):
-    """Device copy of ``host`` with NaN-free canaries around it; returns (full, view)."""
+def _guarded(host: np.ndarray, dtype, device="cuda", shift=0):
+    """Device copy of ``host`` with NaN-free canaries around it; returns (full, view).
+    ``shift`` moves the view by that many elements (to leave 32-byte alignment)."""
     n = host.size
     full = torch.full((n + 2 * GUARD,), 12345.0, dtype=dtype, device=device)
-    view = full[GUARD:GUARD + n]
+    view = full[GUARD + shift:GUARD + shift + n]
     if n:
         view.copy_(torch.from_numpy(host).to(dtype))
     return full, view
@@ -48,13 +49,13 @@ def _resync(dev, host):
         dev.copy_(torch.from_numpy(host))
 
 
-def _check_guard(full, n):
-    assert torch.all(full[:GUARD] == 12345.0) and torch.all(full[GUARD + n:] == 12345.0), \
-        "write outside the output buffer"
+def _check_guard(full, n, shift=0):
+    assert torch.all(full[:GUARD + shift] == 12345.0) and \
+        torch.all(full[GUARD + shift + n:] == 12345.0), "write outside the output buffer"
 
 
 def run_case(dd, ctx, n, M, dtype, tokens, mask, K, *, seed=0, steps=None, flags=0, merges=2,
-             use_out=True, poison_absent=False, null_absent=False, eta=ETA, mu=MU):
+             use_out=True, poison_absent=False, null_absent=False, eta=ETA, mu=MU, shift=0):
     theta, v, learners = synth.fragment_cpu(n, M, dtype, seed)
     part = [m for m in range(M) if (mask >> m) & 1 and tokens[m] > 0]
     if poison_absent:
@@ -65,7 +66,7 @@ def run_case(dd, ctx, n, M, dtype, tokens, mask, K, *, seed=0, steps=None, flags
     if null_absent:
         o_learners = [a if m in part else None for m, a in enumerate(learners)]
     d_learners = [to_torch_learner(a, "cuda") for a in o_learners]
-    t_full, t_dev = _guarded(theta, torch.float32)
+    t_full, t_dev = _guarded(theta, torch.float32, shift=shift)
     v_full, v_dev = _guarded(v, torch.float32)
     out_full = out_dev = None
     if use_out:
@@ -92,7 +93,7 @@ def run_case(dd, ctx, n, M, dtype, tokens, mask, K, *, seed=0, steps=None, flags
             # identical except where the fp32 state differs by an ulp across a rounding boundary
             same = np.mean(out_dev.cpu().view(torch.int16).numpy().view(np.uint16) == o_out) if n else 1.0
             assert same > 0.999
-        _check_guard(t_full, n)
+        _check_guard(t_full, n, shift)
         _check_guard(v_full, n)
         if use_out:
             _check_guard(out_full, n)
@@ -114,6 +115,15 @@ def test_tiny_config(dd, ctx):
 def test_ragged_sizes(dd, ctx, n, dtype):
     run_case(dd, ctx, n, 5, dtype, [100, 200, 0, 400, 500], 0b11101, 2, seed=n % 97,
              flags=dd.DIAG_STATE | dd.DIAG_PER_LEARNER)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_state_only_16_byte_aligned(dd, ctx, dtype):
+    # Theta 16- but not 32-byte aligned: the 2 x 128-bit access path instead of 256-bit
+    run_case(dd, ctx, 40_003, 5, dtype, [100, 200, 0, 400, 500], 0b11101, 2, seed=31,
+             flags=dd.DIAG_STATE | dd.DIAG_PER_LEARNER, shift=4)
+    run_case(dd, ctx, 40_003, 5, dtype, [100, 200, 0, 400, 500], 0b11101, 2, seed=31, flags=0,
+             shift=4)
 
 
 @pytest.mark.parametrize("flags", [0, 1, 2, 4, 7])

@@ -1,0 +1,90 @@
+"""world_size-2 (and 3) gloo tests of the multi-rank path: range sharding of a
+fragment, combination of per-rank records, and max-over-ranks timing.  The
+per-rank merge is done by the oracle here (no GPU in this suite); the plumbing
+under test is the same code bench.py and a sharded deployment use."""
+import os
+import socket
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+import oracle
+from paper_2604_21428_b200 import dist as ddist
+from paper_2604_21428_b200 import synth
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def test_shard_range_partitions_exactly():
+    for n in (0, 1, 7, 8, 9, 1000, 8191, 8192, 500_000_000):
+        for world in (1, 2, 3, 8):
+            prev = 0
+            for r in range(world):
+                lo, hi = ddist.shard_range(n, r, world)
+                assert lo == prev and lo <= hi <= n
+                assert lo % 8 == 0 or lo == n
+                prev = hi
+            assert prev == n
+    sizes = [ddist.shard_range(1000, r, 3)[1] - ddist.shard_range(1000, r, 3)[0] for r in range(3)]
+    assert max(sizes) - min(sizes) <= 8
+    with pytest.raises(ValueError):
+        ddist.shard_range(10, 2, 2)
+
+
+def _worker(rank, world, port, n, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        M, tokens, mask, K = 5, [100, 0, 300, 400, 500], 0b11101, 3
+        theta, v, learners = synth.fragment_cpu(n, M, "bf16", seed=77)       # same on every rank
+        lo, hi = ddist.shard_range(n, rank, world)
+        t_s, v_s = theta[lo:hi].copy(), v[lo:hi].copy()
+        l_s = [a[lo:hi].copy() for a in learners]
+        rec = oracle.merge_fragment(t_s, v_s, l_s, tokens, mask, K, 0.7, 0.9)
+        rec = ddist.allreduce_record(rec)
+        slowest = ddist.max_over_ranks(10.0 + rank)
+        # gather the shards on rank 0 and compare with the unsharded merge
+        parts = [None] * world
+        dist.all_gather_object(parts, (lo, hi, t_s, v_s))
+        if rank == 0:
+            t_full, v_full = np.empty_like(theta), np.empty_like(v)
+            for a, b, ts, vs in parts:
+                t_full[a:b], v_full[a:b] = ts, vs
+            ref = oracle.merge_fragment(theta, v, learners, tokens, mask, K, 0.7, 0.9)
+            ok = (np.array_equal(t_full, theta) and np.array_equal(v_full, v)
+                  and rec.idx == ref.idx and rec.w_hat == ref.w_hat and rec.status == ref.status
+                  and abs(rec.delta_sq - ref.delta_sq) <= 1e-12 * ref.delta_sq
+                  and abs(rec.theta_sq - ref.theta_sq) <= 1e-12 * ref.theta_sq
+                  and abs(rec.mom_sq - ref.mom_sq) <= 1e-12 * ref.mom_sq
+                  and all(abs(a - b) <= 1e-12 * b for a, b in zip(rec.delta_m_sq, ref.delta_m_sq))
+                  and slowest == 10.0 + world - 1)
+            out.put(bool(ok))
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world,n", [(2, 10_007), (3, 4_096), (2, 5)])
+def test_range_sharded_merge_equals_unsharded(world, n):
+    ctx = mp.get_context("spawn")
+    out = ctx.SimpleQueue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, world, port, n, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    for p in procs:
+        p.join(120)
+        assert p.exitcode == 0
+    assert out.get() is True
+
+
+def test_whole_job_rate():
+    assert ddist.whole_job_rate(500, 4, 2, 1000.0) == 4000.0
+    assert ddist.max_over_ranks(3.5) == 3.5          # no process group: identity
