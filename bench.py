@@ -46,6 +46,8 @@ def parse_args():
     ap.add_argument("--cpu-sample", type=int, default=1 << 25,
                     help="elements of the workload the CPU oracle is timed on")
     ap.add_argument("--out-bf16", action="store_true", help="also write the bf16 broadcast copy")
+    ap.add_argument("--resident", choices=["all", "participants"], default="all",
+                    help="allocate every learner copy, or only those that take part")
     ap.add_argument("--sharding", choices=["replica", "range"], default="replica",
                     help="N>1: every rank merges its own copy of the workload (weak scaling), or "
                          "each rank owns a contiguous element range of every fragment (strong)")
@@ -177,7 +179,7 @@ def run_reference(args):
 
 # ---- our arm ---------------------------------------------------------------------------
 
-def build_workload(w, device, rank_seed, out_bf16):
+def build_workload(w, device, rank_seed, out_bf16, resident="all"):
     """Allocates and fills every fragment of workload ``w`` on ``device``."""
     import torch
 
@@ -188,7 +190,10 @@ def build_workload(w, device, rank_seed, out_bf16):
     for p, n in enumerate(w.fragment_sizes):
         theta = torch.empty(n, dtype=torch.float32, device=device)
         mom = torch.empty(n, dtype=torch.float32, device=device)
-        learners = [torch.empty(n, dtype=ldt, device=device) for _ in range(w.M)]
+        keep = [m for m in range(w.M)
+                if resident == "all" or ((w.masks[p] >> m) & 1 and int(w.tokens[p, m]) > 0)]
+        learners = [torch.empty(n, dtype=ldt, device=device) if m in keep else None
+                    for m in range(w.M)]
         synth.fill_fragment_gpu(theta, mom, learners, seed=w.seed * 1000 + p + 100000 * rank_seed)
         out = torch.empty(n, dtype=torch.bfloat16, device=device) if out_bf16 else None
         frags.append(dict(global_=theta, momentum=mom, learners=learners, out_bf16=out,
@@ -225,7 +230,7 @@ def main():
     if args.sharding == "range" and world > 1:
         w.fragment_sizes = [hi - lo for lo, hi in
                             (ddist.shard_range(n, rank, world) for n in w.fragment_sizes)]
-    frags = build_workload(w, device, rank, args.out_bf16)
+    frags = build_workload(w, device, rank, args.out_bf16, args.resident)
     ctx = dd.Context(local_rank)
     grid, block, tile = ctx.launch_geometry(dd.BF16 if w.learner_dtype == "bf16" else dd.F32)
     ldtype = dd.BF16 if w.learner_dtype == "bf16" else dd.F32
