@@ -46,6 +46,8 @@ def parse_args():
     ap.add_argument("--cpu-sample", type=int, default=1 << 25,
                     help="elements of the workload the CPU oracle is timed on")
     ap.add_argument("--out-bf16", action="store_true", help="also write the bf16 broadcast copy")
+    ap.add_argument("--merge", choices=["avg", "rda"], default="avg",
+                    help="weighted direct averaging (the headline path) or radial-directional")
     ap.add_argument("--resident", choices=["all", "participants"], default="all",
                     help="allocate every learner copy, or only those that take part")
     ap.add_argument("--sharding", choices=["replica", "range"], default="replica",
@@ -240,7 +242,10 @@ def main():
     stream = torch.cuda.current_stream()
 
     def step():
-        if w.P == 1:
+        if args.merge == "rda":
+            ctx.merge_fragments_batched_rda(frags, w.M, ldtype, eta, mu, flags=flags,
+                                            records=records, stream=stream)
+        elif w.P == 1:
             f = frags[0]
             ctx.merge_fragment(f["global_"], f["momentum"], f["learners"], f["tokens"],
                                f["quorum_mask"], f["K"], eta, mu, n=f["n"], learner_dtype=ldtype,
@@ -276,6 +281,14 @@ def main():
     params_per_step = w.total_params
     value = ddist.whole_job_rate(job_params, args.steps, 1, max_ms)
     alg_bytes = w.algorithmic_bytes(out_bf16=args.out_bf16)
+    launches_per_step = 1
+    if args.merge == "rda":
+        # learner copies and Theta are read twice (norms, direction), the direction is
+        # written and read back once: 2 (s b + 4) + 24 bytes per parameter
+        esz = 2 if w.learner_dtype == "bf16" else 4
+        alg_bytes = sum(n * (2 * (w.participants(p) * esz + 4) + 24)
+                        for p, n in enumerate(w.fragment_sizes))
+        launches_per_step = 3
     avg_launch_ms = sum(per_launch_ms) / len(per_launch_ms)
     slowest = sorted(range(len(per_launch_ms)), key=lambda k: -per_launch_ms[k])[:3]
     achieved = alg_bytes / (avg_launch_ms * 1e-3) / 1e9
@@ -303,17 +316,18 @@ def main():
             "participants": [w.participants(p) for p in range(w.P)],
             "learner_dtype": w.learner_dtype, "state_dtype": "f32", "outer_lr": eta,
             "outer_mu": mu, "flags": "nesterov+diag_state", "out_bf16": bool(args.out_bf16),
+            "merge": args.merge,
             "grid": grid, "block": block, "tile_elems": tile,
             "l2": "inputs larger than L2 (no flush)" if alg_bytes > 4 * 126e6 else "L2-resident",
             "parallelism": f"{args.sharding} x{world}" if world > 1 else "single",
         },
         "clocks": sampler.summary(),
-        "gpu_launches": args.steps,
+        "gpu_launches": args.steps * launches_per_step,
         "roofline": roofline,
     }
 
     # ---- end to end: host buffers through dd_merge_fragment_host -------------------
-    if not args.no_e2e and w.P == 1:
+    if not args.no_e2e and w.P == 1 and args.merge == "avg":
         f = frags[0]
         n = f["n"]
         part = [m for m in range(w.M) if (f["quorum_mask"] >> m) & 1 and f["tokens"][m] > 0]

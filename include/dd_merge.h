@@ -45,6 +45,9 @@ typedef struct dd_ctx dd_ctx;
 
 typedef enum { DD_F32 = 0, DD_BF16 = 1 } dd_dtype;
 
+/* How the per-learner outer gradients of a fragment are merged (Appendix "Merging methods"). */
+typedef enum { DD_MERGE_AVG = 0, DD_MERGE_RDA = 1 } dd_merge_kind;
+
 typedef enum {
     DD_OK = 0,
     DD_ERR_INVALID_ARG = -1,        /* null where not allowed, M / K / P out of range, non-finite lr or mu */
@@ -151,6 +154,50 @@ int dd_merge_fragments_batched(dd_ctx *ctx, const dd_fragment_desc *descs, int P
                                dd_dtype learner_dtype, float outer_lr, float outer_mu,
                                uint32_t flags, dd_merge_record *records /* [device] P records or NULL */,
                                void *cuda_stream);
+
+/*
+ * Radial-directional averaging (RDA, Appendix "Merging methods"): the merged outer
+ * gradient keeps the weighted mean NORM of the per-learner outer gradients
+ * D_m = Theta - theta_m and takes the direction of their weighted mean direction,
+ *
+ *   Delta = ( sum_m w^_m ||D_m|| ) * phi( sum_m w^_m phi(D_m) ),   phi(x) = x / ||x||,
+ *
+ * so that ||Delta|| does not shrink like 1/sqrt(M) when the D_m are nearly
+ * orthogonal; the outer step is the same as for dd_merge_fragment.  (The printed
+ * weighted formula shows the mean vector in the first factor; it is read as the
+ * weighted mean of the norms, "completely analogously" to the unweighted one.)
+ * A participant with D_m = 0 adds its (zero) norm to the radial mean and nothing
+ * to the direction; if the mean direction vanishes, Delta = 0.
+ *
+ * Three launches on cuda_stream: norms, mean direction (kept in `scratch`), outer
+ * step.  Learner copies are read twice; bytes per parameter = 2 (s b_theta + 4) + 24.
+ *
+ *   scratch   [device] n floats (16-byte aligned), or NULL: the context allocates
+ *             and keeps one (growing it synchronises the device)
+ *   record    as for dd_merge_fragment; delta_m_sq is always filled, delta_sq is
+ *             ||Delta||^2 of the RDA result.  DD_DIAG_PER_LEARNER is implied.
+ * Everything else is as in dd_merge_fragment.
+ */
+int dd_merge_fragment_rda(dd_ctx *ctx, float *global, float *momentum,
+                          const void *const *learner_ptrs, int M, dd_dtype learner_dtype,
+                          const uint64_t *tokens, const uint64_t *steps,
+                          uint64_t quorum_mask, int K, float outer_lr, float outer_mu,
+                          uint32_t flags, size_t n, void *out_bf16,
+                          dd_merge_record *record, float *scratch, void *cuda_stream);
+
+/*
+ * Many fragments, each merged by the kind given in merge_kinds[p] (host array of
+ * dd_merge_kind values as bytes; NULL = all RDA).  The paper's main runs average
+ * the embedding directly and use RDA everywhere else (Section 5 set-up): this call
+ * does both in the same three launches.  scratch holds, back to back, n_p rounded
+ * up to 8 floats for every RDA fragment (scratch_elems = its capacity in floats;
+ * NULL/0 = context-owned).
+ */
+int dd_merge_fragments_batched_rda(dd_ctx *ctx, const dd_fragment_desc *descs, int P, int M,
+                                   dd_dtype learner_dtype, float outer_lr, float outer_mu,
+                                   uint32_t flags, const uint8_t *merge_kinds,
+                                   dd_merge_record *records, float *scratch,
+                                   size_t scratch_elems, void *cuda_stream);
 
 /*
  * The same update for a fragment whose operands live in HOST memory -- the

@@ -33,6 +33,10 @@ struct dd_ctx {
     size_t tickets_cap = 0;
     ddm::Slot slots[ddm::kSlots];
     int next_slot = 0;
+    float *rda_scratch = nullptr;             // mean direction of radial-directional merges
+    size_t rda_scratch_cap = 0;               // floats
+    dd_merge_record *rda_records = nullptr;   // hand-over records when the caller passes none
+    size_t rda_records_cap = 0;
     ddm::HostPipe *pipe = nullptr;
     char cuda_err[256] = {0};
 };

@@ -28,6 +28,9 @@ struct alignas(16) DevFrag {
     unsigned long long mask;
     int K;
     int has_steps;
+    float *scratch;                      // radial-directional merge: n floats for the mean direction
+    int kind;                            // DD_MERGE_AVG or DD_MERGE_RDA
+    int pad_;
     const void *ptrs[DD_MAX_LEARNERS];
     unsigned long long tokens[DD_MAX_LEARNERS];
     unsigned long long steps[DD_MAX_LEARNERS];

@@ -21,14 +21,22 @@ template <bool BF16, bool PL>
 __global__ void __launch_bounds__(kThreads, kMinBlocksPerSM)
 merge_single_kernel(const __grid_constant__ DevFrag frag, const __grid_constant__ Common c)
 {
-    merge_body<BF16, PL>(&frag, c);
+    merge_body<BF16, PL, kModeMerge>(&frag, c);
 }
 
 template <bool BF16, bool PL>
 __global__ void __launch_bounds__(kThreads, kMinBlocksPerSM)
 merge_batched_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ Common c)
 {
-    merge_body<BF16, PL>(frags, c);
+    merge_body<BF16, PL, kModeMerge>(frags, c);
+}
+
+// One pass of a radial-directional merge over a batch of fragments.
+template <bool BF16, int MODE>
+__global__ void __launch_bounds__(kThreads, kMinBlocksPerSM)
+rda_pass_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ Common c)
+{
+    merge_body<BF16, MODE == kModeNorms, MODE>(frags, c);
 }
 
 }  // namespace ddm
@@ -142,6 +150,27 @@ static int ensure_workspace(dd_ctx *ctx, size_t P, size_t nq, size_t grid)
     return DD_OK;
 }
 
+// Takes the next descriptor staging slot (pinned host + device array of at least P
+// fragments); waits only if a call from kSlots calls ago still owns it.
+static int acquire_slot(dd_ctx *ctx, int P)
+{
+    Slot &slot = ctx->slots[ctx->next_slot];
+    if (slot.used) DD_CUDA(ctx, cudaEventSynchronize(slot.done));
+    if (!slot.done) DD_CUDA(ctx, cudaEventCreateWithFlags(&slot.done, cudaEventDisableTiming));
+    if ((size_t)P > slot.cap) {
+        if (slot.host) cudaFreeHost(slot.host);
+        if (slot.dev) cudaFree(slot.dev);
+        slot.host = nullptr;
+        slot.dev = nullptr;
+        slot.cap = 0;
+        const size_t cap = P < 32 ? 32 : (size_t)P;
+        DD_CUDA(ctx, cudaMallocHost(&slot.host, cap * sizeof(DevFrag)));
+        DD_CUDA(ctx, cudaMalloc(&slot.dev, cap * sizeof(DevFrag)));
+        slot.cap = cap;
+    }
+    return DD_OK;
+}
+
 template <bool BF16, bool PL>
 static cudaError_t launch(bool single, const DevFrag *one, const DevFrag *dev_frags,
                           const Common &c, unsigned grid, cudaStream_t stream)
@@ -202,6 +231,8 @@ extern "C" int dd_destroy(dd_ctx *ctx)
     cudaDeviceSynchronize();
     if (ctx->partials) cudaFree(ctx->partials);
     if (ctx->tickets) cudaFree(ctx->tickets);
+    if (ctx->rda_scratch) cudaFree(ctx->rda_scratch);
+    if (ctx->rda_records) cudaFree(ctx->rda_records);
     host_pipe_destroy(ctx);
     for (Slot &s : ctx->slots) {
         if (s.host) cudaFreeHost(s.host);
@@ -270,21 +301,9 @@ extern "C" int dd_merge_fragments_batched(dd_ctx *ctx, const dd_fragment_desc *d
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
 
-    // Take the next staging slot; wait only if a call from kSlots calls ago still owns it.
+    rc = acquire_slot(ctx, P);
+    if (rc != DD_OK) return rc;
     Slot &slot = ctx->slots[ctx->next_slot];
-    if (slot.used) DD_CUDA(ctx, cudaEventSynchronize(slot.done));
-    if (!slot.done) DD_CUDA(ctx, cudaEventCreateWithFlags(&slot.done, cudaEventDisableTiming));
-    if ((size_t)P > slot.cap) {
-        if (slot.host) cudaFreeHost(slot.host);
-        if (slot.dev) cudaFree(slot.dev);
-        slot.host = nullptr;
-        slot.dev = nullptr;
-        slot.cap = 0;
-        const size_t cap = P < 32 ? 32 : (size_t)P;
-        DD_CUDA(ctx, cudaMallocHost(&slot.host, cap * sizeof(DevFrag)));
-        DD_CUDA(ctx, cudaMalloc(&slot.dev, cap * sizeof(DevFrag)));
-        slot.cap = cap;
-    }
 
     unsigned long long tile = 0;
     for (int p = 0; p < P; ++p) {
@@ -324,6 +343,145 @@ extern "C" int dd_merge_fragments_batched(dd_ctx *ctx, const dd_fragment_desc *d
     slot.used = true;
     ctx->next_slot = (ctx->next_slot + 1) % kSlots;
     return DD_OK;
+}
+
+namespace ddm {
+
+template <bool BF16>
+static cudaError_t launch_rda_passes(const DevFrag *dev_frags, const Common &c, unsigned grid,
+                                     cudaStream_t stream)
+{
+    rda_pass_kernel<BF16, kModeNorms><<<grid, kThreads, 0, stream>>>(dev_frags, c);
+    rda_pass_kernel<BF16, kModeDir><<<grid, kThreads, 0, stream>>>(dev_frags, c);
+    rda_pass_kernel<BF16, kModeApply><<<grid, kThreads, 0, stream>>>(dev_frags, c);
+    return cudaGetLastError();
+}
+
+static size_t round_up8(size_t n) { return (n + 7) / 8 * 8; }
+
+}  // namespace ddm
+
+extern "C" int dd_merge_fragments_batched_rda(dd_ctx *ctx, const dd_fragment_desc *descs, int P,
+                                              int M, dd_dtype learner_dtype, float outer_lr,
+                                              float outer_mu, uint32_t flags,
+                                              const uint8_t *merge_kinds, dd_merge_record *records,
+                                              float *scratch, size_t scratch_elems,
+                                              void *cuda_stream)
+{
+    int rc = check_common(ctx, M, learner_dtype, outer_lr, outer_mu, flags);
+    if (rc != DD_OK) return rc;
+    if (flags & DD_DIAG_PER_LEARNER) flags &= ~(uint32_t)DD_DIAG_PER_LEARNER;   // always on for RDA fragments
+    if (P < 0 || (P > 0 && !descs)) return DD_ERR_INVALID_ARG;
+    if (P > (1 << 20)) return DD_ERR_TOO_LARGE;
+    if (P == 0) return DD_OK;
+    if (misaligned(scratch)) return DD_ERR_ALIGNMENT;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
+
+    // Scratch for the mean direction: n floats per radial-directional fragment.
+    size_t need = 0;
+    for (int p = 0; p < P; ++p)
+        if (!merge_kinds || merge_kinds[p] == DD_MERGE_RDA) need += round_up8((size_t)descs[p].n);
+        else if (merge_kinds[p] != DD_MERGE_AVG) return DD_ERR_INVALID_ARG;
+    if (scratch) {
+        if (scratch_elems < need) return DD_ERR_INVALID_ARG;
+    } else if (need > ctx->rda_scratch_cap) {
+        DD_CUDA(ctx, cudaDeviceSynchronize());
+        if (ctx->rda_scratch) cudaFree(ctx->rda_scratch);
+        ctx->rda_scratch = nullptr;
+        ctx->rda_scratch_cap = 0;
+        DD_CUDA(ctx, cudaMalloc(&ctx->rda_scratch, need * sizeof(float)));
+        ctx->rda_scratch_cap = need;
+    }
+    // The passes hand norms to one another through the records: use the context's
+    // own when the caller wants none.
+    if (!records) {
+        if ((size_t)P > ctx->rda_records_cap) {
+            DD_CUDA(ctx, cudaDeviceSynchronize());
+            if (ctx->rda_records) cudaFree(ctx->rda_records);
+            ctx->rda_records = nullptr;
+            ctx->rda_records_cap = 0;
+            DD_CUDA(ctx, cudaMalloc(&ctx->rda_records, (size_t)P * sizeof(dd_merge_record)));
+            ctx->rda_records_cap = (size_t)P;
+        }
+        records = ctx->rda_records;
+    }
+
+    rc = acquire_slot(ctx, P);
+    if (rc != DD_OK) return rc;
+    Slot &slot = ctx->slots[ctx->next_slot];
+    float *next_scratch = scratch ? scratch : ctx->rda_scratch;
+    unsigned long long tile = 0;
+    for (int p = 0; p < P; ++p) {
+        const dd_fragment_desc &d = descs[p];
+        DevFrag &f = slot.host[p];
+        rc = fill_fragment(f, d.global, d.momentum, d.out_bf16, d.learner_ptrs, d.tokens, d.steps,
+                           d.quorum_mask, d.K, d.n, M, learner_dtype);
+        if (rc != DD_OK) return rc;
+        f.kind = (!merge_kinds || merge_kinds[p] == DD_MERGE_RDA) ? DD_MERGE_RDA : DD_MERGE_AVG;
+        if (f.kind == DD_MERGE_RDA) {
+            f.scratch = next_scratch;
+            next_scratch += round_up8((size_t)d.n);
+            const size_t n = (size_t)d.n;
+            if (overlaps(f.scratch, 4 * n, d.global, 4 * n) || overlaps(f.scratch, 4 * n, d.momentum, 4 * n) ||
+                overlaps(f.scratch, 4 * n, d.out_bf16, 2 * n))
+                return DD_ERR_ALIAS;
+        }
+        f.tile_begin = tile;
+        tile += tiles_of(d.n);
+        f.tile_end = tile;
+    }
+
+    const bool bf16 = learner_dtype == DD_BF16;
+    unsigned long long g = (unsigned long long)ctx->grid[bf16][1];
+    if (g > tile) g = tile;
+    Common c;
+    c.eta = outer_lr;
+    c.mu = outer_mu;
+    c.flags = flags;
+    c.M = M;
+    c.P = P;
+    c.total_tiles = tile;
+    c.records = records;
+    c.nq = kNumScalarDiag + M;
+    rc = ensure_workspace(ctx, (size_t)P, (size_t)c.nq, (size_t)ctx->grid[bf16][1]);
+    if (rc != DD_OK) return rc;
+    c.partials = ctx->partials;
+    c.tickets = ctx->tickets;
+
+    DD_CUDA(ctx, cudaMemcpyAsync(slot.dev, slot.host, (size_t)P * sizeof(DevFrag),
+                                 cudaMemcpyHostToDevice, stream));
+    cudaError_t e = bf16 ? launch_rda_passes<true>(slot.dev, c, (unsigned)g, stream)
+                         : launch_rda_passes<false>(slot.dev, c, (unsigned)g, stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "rda_pass_kernel launch");
+    DD_CUDA(ctx, cudaEventRecord(slot.done, stream));
+    slot.used = true;
+    ctx->next_slot = (ctx->next_slot + 1) % kSlots;
+    return DD_OK;
+}
+
+extern "C" int dd_merge_fragment_rda(dd_ctx *ctx, float *global, float *momentum,
+                                     const void *const *learner_ptrs, int M, dd_dtype learner_dtype,
+                                     const uint64_t *tokens, const uint64_t *steps,
+                                     uint64_t quorum_mask, int K, float outer_lr, float outer_mu,
+                                     uint32_t flags, size_t n, void *out_bf16,
+                                     dd_merge_record *record, float *scratch, void *cuda_stream)
+{
+    dd_fragment_desc d;
+    d.global = global;
+    d.momentum = momentum;
+    d.out_bf16 = out_bf16;
+    d.learner_ptrs = learner_ptrs;
+    d.tokens = tokens;
+    d.steps = steps;
+    d.quorum_mask = quorum_mask;
+    d.K = K;
+    d.n = n;
+    return dd_merge_fragments_batched_rda(ctx, &d, 1, M, learner_dtype, outer_lr, outer_mu, flags,
+                                          nullptr, record, scratch, scratch ? round_up8(n) : 0,
+                                          cuda_stream);
 }
 
 extern "C" const char *dd_last_cuda_error(const dd_ctx *ctx)

@@ -19,6 +19,13 @@
 
 namespace ddm {
 
+// What a launch does with a fragment.  The weighted direct average needs one
+// launch (kModeMerge).  Radial-directional averaging ("Merging methods" appendix)
+// needs three: per-participant norms, the mean direction u = sum_j (w_j/||D_j||) D_j
+// written to a scratch array together with ||u||^2, and the outer step with
+// Delta = (sum_j w_j ||D_j||) u / ||u||.
+enum : int { kModeMerge = 0, kModeNorms = 1, kModeDir = 2, kModeApply = 3 };
+
 struct Smem {
     const void *ptr[DD_MAX_LEARNERS];    // participant j's buffer (compacted)
     double wraw[DD_MAX_LEARNERS];        // raw weights, participant order
@@ -34,7 +41,10 @@ struct Smem {
     int status;
     int frag;
     int is_last;
-    int wide;                            // Theta and v are 32-byte aligned: 256-bit accesses
+    int wide;                            // Theta, v (and scratch) are 32-byte aligned: 256-bit accesses
+    int kind;                            // DD_MERGE_AVG / DD_MERGE_RDA of this fragment
+    float *scratch;                      // RDA: the mean direction u
+    float cscale;                        // RDA apply: Delta = cscale * u
     double red[kWarps][kNumScalarDiag];  // per-warp ||Delta||^2, ||Theta'||^2, ||v'||^2 of this fragment
     double dm[kWarps][DD_MAX_LEARNERS];  // per-warp per-participant ||Theta-theta_m||^2
 };
@@ -118,6 +128,7 @@ __device__ __forceinline__ float warp_sum(float x)
 // each member its rank), quorum test |S| >= max(K,1), w = tokens (or
 // tokens^2/steps), w_hat = w / sum_S w.  Integer work is exact; the token sum is
 // an order-free uint64 butterfly, the tokens^2/steps sum is taken in rank order.
+template <int MODE>
 __device__ __forceinline__ void load_header(const DevFrag *f, int p, unsigned long long tile,
                                             const Common &c, Smem &sm)
 {
@@ -168,13 +179,39 @@ __device__ __forceinline__ void load_header(const DevFrag *f, int p, unsigned lo
         sm.n_part = n_part;
         sm.status = status;
         sm.frag = p;
-        sm.wide = (((unsigned long long)f->theta | (unsigned long long)f->mom) & 31ull) == 0;
+        sm.wide = (((unsigned long long)f->theta | (unsigned long long)f->mom |
+                    (unsigned long long)f->scratch) & 31ull) == 0;
+        sm.kind = f->kind;
+        sm.scratch = f->scratch;
+        sm.cscale = 0.0f;
     }
     for (int j = lane; j < kWarps * DD_MAX_LEARNERS; j += 32) (&sm.dm[0][0])[j] = 0.0;
     if (lane < kWarps * kNumScalarDiag) (&sm.red[0][0])[lane] = 0.0;
     __syncwarp();
-    // The CTA that owns the fragment's first tile publishes the header.
-    if (c.records != nullptr && tile == f->tile_begin) {
+    if ((MODE == kModeDir || MODE == kModeApply) && f->kind == DD_MERGE_RDA &&
+        status == DD_STATUS_OK) {
+        // The norms pass left ||Theta - theta_j||^2 in this fragment's record.
+        const dd_merge_record *rec = c.records + p;
+        const double n0 = j0 < n_part && p0 ? sqrt(__ldcg(&rec->delta_m_sq[j0])) : 0.0;
+        const double n1 = p1 ? sqrt(__ldcg(&rec->delta_m_sq[j1])) : 0.0;
+        if (MODE == kModeDir) {
+            // direction weights a_j = w_hat_j / ||D_j||; a zero outer gradient has no direction
+            if (p0) sm.w[j0] = n0 > 0.0 ? (float)((double)sm.w[j0] / n0) : 0.0f;
+            if (p1) sm.w[j1] = n1 > 0.0 ? (float)((double)sm.w[j1] / n1) : 0.0f;
+        } else {
+            // radial part sum_j w_hat_j ||D_j|| over the mean direction's length
+            double radial = (p0 ? (double)sm.w[j0] * n0 : 0.0) + (p1 ? (double)sm.w[j1] * n1 : 0.0);
+            radial = warp_sum(radial);
+            const double usq = __ldcg(&rec->delta_sq);
+            if (lane == 0) sm.cscale = usq > 0.0 ? (float)(radial / sqrt(usq)) : 0.0f;
+        }
+        __syncwarp();
+    }
+    // The CTA that owns the fragment's first tile publishes the header (once per
+    // call: the later passes of a radial-directional merge leave it alone).
+    const bool publish = MODE == kModeMerge ? f->kind == DD_MERGE_AVG
+                                            : (MODE == kModeNorms && f->kind == DD_MERGE_RDA);
+    if (publish && c.records != nullptr && tile == f->tile_begin) {
         dd_merge_record *rec = c.records + p;
         for (int j = lane; j < DD_MAX_LEARNERS; j += 32) {
             const bool on = j < n_part && status == DD_STATUS_OK;
@@ -211,7 +248,7 @@ __device__ __forceinline__ int find_frag(const DevFrag *frags, int lo, int P,
 // (exact or nearly so when theta_j is close to Theta), then weighted: factoring
 // Theta out of the sum would lose ~|Theta|/|Delta| ulps.  `active` is false only
 // with per-learner diagnostics, where idle lanes still take part in the shuffles.
-template <bool BF16, bool PL, bool WIDE>
+template <bool BF16, bool PL, bool WIDE, int MODE>
 __device__ __forceinline__ void process_vec(Smem &sm, const Common &c, unsigned vi, bool active,
                                             float &dsq, float &tsq, float &msq)
 {
@@ -231,60 +268,83 @@ __device__ __forceinline__ void process_vec(Smem &sm, const Common &c, unsigned 
         acc[k] = make_float2(0.0f, 0.0f);
     }
 
+    if (MODE != kModeApply) {
 #pragma unroll 1
-    for (int j0 = 0; j0 < s; j0 += B) {
-        uint4 r[BF16 ? B : 2 * B];
+        for (int j0 = 0; j0 < s; j0 += B) {
+            uint4 r[BF16 ? B : 2 * B];
 #pragma unroll
-        for (int b = 0; b < B; ++b) {
-            if (j0 + b < s) {
-                if (PL && !active) {
-                    if (BF16) r[b] = make_uint4(0u, 0u, 0u, 0u);
-                    else r[2 * b] = r[2 * b + 1] = make_uint4(0u, 0u, 0u, 0u);
-                } else if (BF16) {
-                    r[b] = ld_stream16(reinterpret_cast<const uint4 *>(sm.ptr[j0 + b]) + vi);
-                } else {
-                    const uint4 *p = reinterpret_cast<const uint4 *>(sm.ptr[j0 + b]) + 2ull * vi;
-                    r[2 * b] = ld_stream16(p);
-                    r[2 * b + 1] = ld_stream16(p + 1);
+            for (int b = 0; b < B; ++b) {
+                if (j0 + b < s) {
+                    if (PL && !active) {
+                        if (BF16) r[b] = make_uint4(0u, 0u, 0u, 0u);
+                        else r[2 * b] = r[2 * b + 1] = make_uint4(0u, 0u, 0u, 0u);
+                    } else if (BF16) {
+                        r[b] = ld_stream16(reinterpret_cast<const uint4 *>(sm.ptr[j0 + b]) + vi);
+                    } else {
+                        const uint4 *p = reinterpret_cast<const uint4 *>(sm.ptr[j0 + b]) + 2ull * vi;
+                        r[2 * b] = ld_stream16(p);
+                        r[2 * b + 1] = ld_stream16(p + 1);
+                    }
                 }
             }
-        }
-        // The momentum is needed only by the epilogue: fetch it behind the last batch.
-        if (j0 + B >= s && (!PL || active)) load_f32x8<WIDE>(sm.mom, vi, V);
+            // The momentum is needed only by the epilogue: fetch it behind the last batch.
+            if (MODE == kModeMerge && j0 + B >= s && (!PL || active)) load_f32x8<WIDE>(sm.mom, vi, V);
 #pragma unroll
-        for (int b = 0; b < B; ++b) {
-            if (j0 + b < s) {
-                const float w = sm.w[j0 + b];
-                const float2 w2 = make_float2(w, w);
-                float2 x[4];
-                if (BF16) {
-                    // element 2k sits in the low half of word k, element 2k+1 in the high half
-                    const unsigned word[4] = {r[b].x, r[b].y, r[b].z, r[b].w};
+            for (int b = 0; b < B; ++b) {
+                if (j0 + b < s) {
+                    const float w = sm.w[j0 + b];
+                    const float2 w2 = make_float2(w, w);
+                    float2 x[4];
+                    if (BF16) {
+                        // element 2k sits in the low half of word k, element 2k+1 in the high half
+                        const unsigned word[4] = {r[b].x, r[b].y, r[b].z, r[b].w};
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        x[k] = make_float2(__uint_as_float(word[k] << 16),
-                                           __uint_as_float(word[k] & 0xffff0000u));
-                } else {
-                    x[0] = make_float2(__uint_as_float(r[2 * b].x), __uint_as_float(r[2 * b].y));
-                    x[1] = make_float2(__uint_as_float(r[2 * b].z), __uint_as_float(r[2 * b].w));
-                    x[2] = make_float2(__uint_as_float(r[2 * b + 1].x), __uint_as_float(r[2 * b + 1].y));
-                    x[3] = make_float2(__uint_as_float(r[2 * b + 1].z), __uint_as_float(r[2 * b + 1].w));
-                }
-                float q = 0.0f;
+                        for (int k = 0; k < 4; ++k)
+                            x[k] = make_float2(__uint_as_float(word[k] << 16),
+                                               __uint_as_float(word[k] & 0xffff0000u));
+                    } else {
+                        x[0] = make_float2(__uint_as_float(r[2 * b].x), __uint_as_float(r[2 * b].y));
+                        x[1] = make_float2(__uint_as_float(r[2 * b].z), __uint_as_float(r[2 * b].w));
+                        x[2] = make_float2(__uint_as_float(r[2 * b + 1].x), __uint_as_float(r[2 * b + 1].y));
+                        x[3] = make_float2(__uint_as_float(r[2 * b + 1].z), __uint_as_float(r[2 * b + 1].w));
+                    }
+                    float q = 0.0f;
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const float2 d = __fadd2_rn(x[k], nT[k]);
-                    acc[k] = __ffma2_rn(w2, d, acc[k]);
-                    if (PL) q = fmaf(d.x, d.x, fmaf(d.y, d.y, q));
-                }
-                if (PL) {
-                    q = warp_sum(q);
-                    if ((threadIdx.x & 31) == 0) sm.dm[threadIdx.x >> 5][j0 + b] += (double)q;
+                    for (int k = 0; k < 4; ++k) {
+                        const float2 d = __fadd2_rn(x[k], nT[k]);
+                        if (MODE != kModeNorms) acc[k] = __ffma2_rn(w2, d, acc[k]);
+                        if (PL) q = fmaf(d.x, d.x, fmaf(d.y, d.y, q));
+                    }
+                    if (PL) {
+                        q = warp_sum(q);
+                        if ((threadIdx.x & 31) == 0) sm.dm[threadIdx.x >> 5][j0 + b] += (double)q;
+                    }
                 }
             }
         }
     }
     if (PL && !active) return;
+    if (MODE == kModeNorms) return;
+
+    if (MODE == kModeDir) {
+        // the mean direction u = sum_j a_j (Theta - theta_j), kept for the apply pass
+        float U[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            U[k] = -((k & 1) ? acc[k >> 1].y : acc[k >> 1].x);
+            dsq = fmaf(U[k], U[k], dsq);
+        }
+        store_f32x8<WIDE>(sm.scratch, vi, U);
+        return;
+    }
+    if (MODE == kModeApply) {
+        float U[8];
+        load_f32x8<WIDE>(sm.scratch, vi, U);
+        load_f32x8<WIDE>(sm.mom, vi, V);
+        const float cs = sm.cscale;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) acc[k] = make_float2(-cs * U[2 * k], -cs * U[2 * k + 1]);
+    }
 
     // Outer step: v' = mu v + Delta; Theta' = Theta - eta (Delta + mu v') (Nesterov)
     // or Theta - eta v' (heavy ball).
@@ -311,7 +371,7 @@ __device__ __forceinline__ void process_vec(Smem &sm, const Common &c, unsigned 
 }
 
 // The ragged end of a fragment (n mod 8 elements), one element per lane of warp 0.
-template <bool BF16, bool PL>
+template <bool BF16, bool PL, int MODE>
 __device__ __forceinline__ void process_tail(Smem &sm, const Common &c, unsigned long long first,
                                              int count, float &dsq, float &tsq, float &msq)
 {
@@ -321,21 +381,28 @@ __device__ __forceinline__ void process_tail(Smem &sm, const Common &c, unsigned
     const int s = sm.n_part;
     const float T = active ? sm.theta[e] : 0.0f;
     float acc = 0.0f;
-    for (int j = 0; j < s; ++j) {
-        float th = 0.0f;
-        if (active) {
-            if (BF16) th = __uint_as_float((unsigned)reinterpret_cast<const uint16_t *>(sm.ptr[j])[e] << 16);
-            else th = reinterpret_cast<const float *>(sm.ptr[j])[e];
-        }
-        const float d = th - T;
-        acc = fmaf(sm.w[j], d, acc);
-        if (PL) {
-            const float q = warp_sum(d * d);
-            if (lane == 0) sm.dm[0][j] += (double)q;
+    if (MODE != kModeApply) {
+        for (int j = 0; j < s; ++j) {
+            float th = 0.0f;
+            if (active) {
+                if (BF16) th = __uint_as_float((unsigned)reinterpret_cast<const uint16_t *>(sm.ptr[j])[e] << 16);
+                else th = reinterpret_cast<const float *>(sm.ptr[j])[e];
+            }
+            const float d = th - T;
+            acc = fmaf(sm.w[j], d, acc);
+            if (PL) {
+                const float q = warp_sum(d * d);
+                if (lane == 0) sm.dm[0][j] += (double)q;
+            }
         }
     }
-    if (!active) return;
-    const float delta = -acc;
+    if (!active || MODE == kModeNorms) return;
+    if (MODE == kModeDir) {
+        sm.scratch[e] = -acc;
+        dsq = fmaf(acc, acc, dsq);
+        return;
+    }
+    const float delta = MODE == kModeApply ? sm.cscale * sm.scratch[e] : -acc;
     const float vn = fmaf(c.mu, sm.mom[e], delta);
     const float u = (c.flags & DD_HEAVY_BALL) ? vn : fmaf(c.mu, vn, delta);
     const float tn = fmaf(-c.eta, u, T);
@@ -407,7 +474,7 @@ __device__ __forceinline__ void flush_fragment(Smem &sm, const Common &c)
 }
 
 // One tile (kTileElems elements of the current fragment).
-template <bool BF16, bool PL, bool WIDE>
+template <bool BF16, bool PL, bool WIDE, int MODE>
 __device__ __forceinline__ void process_tile(Smem &sm, const Common &c, unsigned long long tile)
 {
     constexpr unsigned kTileSteps = kTileElems / kVec;
@@ -419,15 +486,15 @@ __device__ __forceinline__ void process_tile(Smem &sm, const Common &c, unsigned
     if (PL) {
         // per-learner norms are warp-wide sums: the whole warp walks together
         for (unsigned v0 = base + warp * 32; v0 < end; v0 += kThreads)
-            process_vec<BF16, true, WIDE>(sm, c, v0 + lane, v0 + lane < end, dsq, tsq, msq);
+            process_vec<BF16, true, WIDE, MODE>(sm, c, v0 + lane, v0 + lane < end, dsq, tsq, msq);
     } else {
         for (unsigned vi = base + threadIdx.x; vi < end; vi += kThreads)
-            process_vec<BF16, false, WIDE>(sm, c, vi, true, dsq, tsq, msq);
+            process_vec<BF16, false, WIDE, MODE>(sm, c, vi, true, dsq, tsq, msq);
     }
     const int rem = (int)(sm.n % kVec);
     if (rem != 0 && tile == sm.tile_end - 1 && warp == 0)
-        process_tail<BF16, PL>(sm, c, (unsigned long long)nfull * kVec, rem, dsq, tsq, msq);
-    if (c.records != nullptr) {
+        process_tail<BF16, PL, MODE>(sm, c, (unsigned long long)nfull * kVec, rem, dsq, tsq, msq);
+    if (c.records != nullptr && MODE != kModeNorms) {
         // fp32 within a tile (at most 32 elements per thread), fp64 from here on
         dsq = warp_sum(dsq);
         tsq = warp_sum(tsq);
@@ -441,31 +508,52 @@ __device__ __forceinline__ void process_tile(Smem &sm, const Common &c, unsigned
 }
 
 // ---- the kernel body ----------------------------------------------------------
-template <bool BF16, bool PL>
+//
+// MODE is what this launch does with fragments merged radial-directionally; a
+// fragment of kind DD_MERGE_AVG is skipped by the norms and direction passes and
+// gets the ordinary fused merge in the apply pass, so one batch can mix both.
+template <bool BF16, bool PL, int MODE>
 __device__ __forceinline__ void merge_body(const DevFrag *frags, const Common &c)
 {
     __shared__ Smem sm;
     const unsigned G = gridDim.x;
     int cur = -1;
     bool loaded = false;
+    auto worked_on = [&]() {
+        return sm.status == DD_STATUS_OK && (MODE == kModeMerge || MODE == kModeApply || sm.kind == DD_MERGE_RDA);
+    };
 
     for (unsigned long long tile = blockIdx.x; tile < c.total_tiles; tile += G) {
         if (!loaded || tile >= sm.tile_end) {                     // CTA-uniform
-            if (loaded && c.records != nullptr && sm.status == DD_STATUS_OK) flush_fragment<PL>(sm, c);
+            if (loaded && c.records != nullptr && worked_on()) {
+                if (MODE == kModeApply && sm.kind == DD_MERGE_AVG) flush_fragment<false>(sm, c);
+                else flush_fragment<PL>(sm, c);
+            }
             __syncthreads();
             if (threadIdx.x < 32) {
                 cur = find_frag(frags, cur < 0 ? 0 : cur + 1, c.P, tile);
-                load_header(frags + cur, cur, tile, c, sm);
+                if (MODE == kModeApply && frags[cur].kind == DD_MERGE_AVG)
+                    load_header<kModeMerge>(frags + cur, cur, tile, c, sm);
+                else
+                    load_header<MODE>(frags + cur, cur, tile, c, sm);
             }
             __syncthreads();
             cur = sm.frag;
             loaded = true;
         }
-        if (sm.status != DD_STATUS_OK) continue;
-        if (sm.wide) process_tile<BF16, PL, true>(sm, c, tile);
-        else process_tile<BF16, PL, false>(sm, c, tile);
+        if (!worked_on()) continue;
+        if (MODE == kModeApply && sm.kind == DD_MERGE_AVG) {
+            if (sm.wide) process_tile<BF16, false, true, kModeMerge>(sm, c, tile);
+            else process_tile<BF16, false, false, kModeMerge>(sm, c, tile);
+        } else {
+            if (sm.wide) process_tile<BF16, PL, true, MODE>(sm, c, tile);
+            else process_tile<BF16, PL, false, MODE>(sm, c, tile);
+        }
     }
-    if (loaded && c.records != nullptr && sm.status == DD_STATUS_OK) flush_fragment<PL>(sm, c);
+    if (loaded && c.records != nullptr && worked_on()) {
+        if (MODE == kModeApply && sm.kind == DD_MERGE_AVG) flush_fragment<false>(sm, c);
+        else flush_fragment<PL>(sm, c);
+    }
 }
 
 }  // namespace ddm

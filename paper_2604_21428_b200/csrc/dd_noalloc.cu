@@ -40,13 +40,13 @@ static __device__ __align__(256) unsigned char g_scratch[DD_NOALLOC_SCRATCH_BYTE
 __global__ void __launch_bounds__(kThreads, 2)
 merge_batched_noalloc_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ Common c)
 {
-    merge_body<true, false>(frags, c);
+    merge_body<true, false, kModeMerge>(frags, c);
 }
 
 __global__ void __launch_bounds__(kThreads, 2)
 merge_batched_noalloc_kernel_f32(const DevFrag *__restrict__ frags, const __grid_constant__ Common c)
 {
-    merge_body<false, false>(frags, c);
+    merge_body<false, false, kModeMerge>(frags, c);
 }
 
 struct DeviceState {

@@ -18,12 +18,14 @@ ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_ALIAS, ERR_TOO_MANY_LEARNERS, ERR_CUDA, ERR_
     -1, -2, -3, -4, -5, -6
 STATUS_OK, STATUS_QUORUM_NOT_MET, STATUS_ZERO_WEIGHT, STATUS_WAIT_LIMIT = 0, 1, 2, 3
 HEAVY_BALL, DIAG_PER_LEARNER, DIAG_STATE = 1, 2, 4
+MERGE_AVG, MERGE_RDA = 0, 1
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libddmerge.so")
 
 EXPORTS = (
     "dd_create", "dd_destroy", "dd_merge_fragment", "dd_merge_fragments_batched",
     "dd_merge_fragment_host", "dd_merge_fragments_batched_noalloc",
+    "dd_merge_fragment_rda", "dd_merge_fragments_batched_rda",
     "dd_select_quorum", "dd_grace_window", "dd_status_string", "dd_last_cuda_error",
     "dd_launch_geometry",
 )
@@ -81,6 +83,15 @@ def _load() -> ctypes.CDLL:
     lib.dd_merge_fragments_batched.argtypes = [
         vp, ctypes.POINTER(CFragmentDesc), ctypes.c_int, ctypes.c_int, ctypes.c_int,
         ctypes.c_float, ctypes.c_float, ctypes.c_uint32, vp, vp]
+    lib.dd_merge_fragment_rda.restype = ctypes.c_int
+    lib.dd_merge_fragment_rda.argtypes = [
+        vp, vp, vp, ctypes.POINTER(vp), ctypes.c_int, ctypes.c_int, u64p, u64p, ctypes.c_uint64,
+        ctypes.c_int, ctypes.c_float, ctypes.c_float, ctypes.c_uint32, ctypes.c_size_t, vp, vp, vp, vp]
+    lib.dd_merge_fragments_batched_rda.restype = ctypes.c_int
+    lib.dd_merge_fragments_batched_rda.argtypes = [
+        vp, ctypes.POINTER(CFragmentDesc), ctypes.c_int, ctypes.c_int, ctypes.c_int,
+        ctypes.c_float, ctypes.c_float, ctypes.c_uint32, ctypes.POINTER(ctypes.c_uint8), vp, vp,
+        ctypes.c_size_t, vp]
     lib.dd_merge_fragment_host.restype = ctypes.c_int
     lib.dd_merge_fragment_host.argtypes = [
         vp, vp, vp, ctypes.POINTER(vp), ctypes.c_int, ctypes.c_int, u64p, u64p, ctypes.c_uint64,
@@ -221,6 +232,38 @@ class Context:
             ctypes.c_uint64(quorum_mask & (2**64 - 1)), int(K), ctypes.c_float(outer_lr),
             ctypes.c_float(outer_mu), ctypes.c_uint32(flags), ctypes.c_size_t(n), _ptr(out_bf16),
             _ptr(record), _stream_handle(stream)))
+
+    def merge_fragment_rda(self, global_, momentum, learners, tokens, quorum_mask: int, K: int,
+                           outer_lr: float, outer_mu: float, *, n: int | None = None,
+                           learner_dtype: int | None = None, steps=None, flags: int = 0,
+                           out_bf16=None, record=None, scratch=None, stream=None) -> None:
+        """``dd_merge_fragment_rda``: radial-directional merge of one fragment."""
+        M = len(learners)
+        if n is None:
+            n = int(global_.numel())
+        if learner_dtype is None:
+            learner_dtype = _infer_dtype(learners)
+        ptrs = (ctypes.c_void_p * M)(*[_ptr(t) for t in learners])
+        self._check(lib.dd_merge_fragment_rda(
+            self._h, _ptr(global_), _ptr(momentum), ptrs, M, learner_dtype, _u64_array(tokens),
+            None if steps is None else _u64_array(steps),
+            ctypes.c_uint64(quorum_mask & (2**64 - 1)), int(K), ctypes.c_float(outer_lr),
+            ctypes.c_float(outer_mu), ctypes.c_uint32(flags), ctypes.c_size_t(n), _ptr(out_bf16),
+            _ptr(record), _ptr(scratch), _stream_handle(stream)))
+
+    def merge_fragments_batched_rda(self, fragments, M: int, learner_dtype: int, outer_lr: float,
+                                    outer_mu: float, *, merge_kinds=None, flags: int = 0,
+                                    records=None, scratch=None, stream=None) -> None:
+        """``dd_merge_fragments_batched_rda``: ``merge_kinds`` is a list of MERGE_AVG /
+        MERGE_RDA per fragment (None = all RDA); ``scratch`` an optional float32 tensor."""
+        P = len(fragments)
+        descs, _keep = _pack_descs(fragments, M)
+        kinds = None if merge_kinds is None else (ctypes.c_uint8 * P)(*[int(k) for k in merge_kinds])
+        self._check(lib.dd_merge_fragments_batched_rda(
+            self._h, descs, P, M, learner_dtype, ctypes.c_float(outer_lr), ctypes.c_float(outer_mu),
+            ctypes.c_uint32(flags), kinds, _ptr(records), _ptr(scratch),
+            ctypes.c_size_t(0 if scratch is None else int(scratch.numel())),
+            _stream_handle(stream)))
 
     def merge_fragment_host(self, global_, momentum, learners, tokens, quorum_mask: int, K: int,
                             outer_lr: float, outer_mu: float, *, n: int | None = None,
