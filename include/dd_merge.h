@@ -279,6 +279,32 @@ int dd_select_quorum(const double *arrival_s, int M, int K, double grace_s,
 double dd_grace_window(double tau, double xi_step, double xi_quorum, double xi_sync,
                        double gamma);
 
+/*
+ * Fragmentation planner (Appendix "Fragmentation strategies"), host only: assigns
+ * each of the model's Q tensors to one of P fragments.
+ *
+ *   DD_FRAG_LAYER     fragment 0 holds every non-transformer tensor; transformer
+ *                     layer l (0-based) goes to fragment 1 + (l mod (P-1)) -- strided
+ *                     selection; needs 2 <= P and P-1 <= number of layers.
+ *   DD_FRAG_TENSOR    fragment 0 holds every non-transformer tensor; the i-th (0-based,
+ *                     in the given order) transformer tensor goes to 1 + (i mod (P-1)).
+ *   DD_FRAG_BALANCED  greedy number partitioning over ALL tensors: in descending order
+ *                     of size (ties: given order) each tensor joins the fragment whose
+ *                     total is smallest (ties: lowest index).  The largest fragment is
+ *                     at most 4/3 of the best possible.
+ *
+ *   size_bits    [host] Q tensor sizes in bits
+ *   layer        [host] Q entries: 0-based transformer layer of the tensor, or -1 for a
+ *                non-transformer tensor (embedding, final norm, head); may be NULL for
+ *                DD_FRAG_BALANCED
+ *   fragment_of  [host] out, Q fragment indices in [0, P)
+ *   fragment_bits[host] out, optional, P totals
+ * Returns DD_OK or DD_ERR_INVALID_ARG (P < 1, Q < 0, a strategy's requirement unmet).
+ */
+typedef enum { DD_FRAG_LAYER = 0, DD_FRAG_TENSOR = 1, DD_FRAG_BALANCED = 2 } dd_frag_strategy;
+int dd_plan_fragments(const uint64_t *size_bits, const int32_t *layer, int Q, int P,
+                      dd_frag_strategy strategy, int32_t *fragment_of, uint64_t *fragment_bits);
+
 /* Text for a dd_error / the most recent CUDA error string seen by ctx. */
 const char *dd_status_string(int rc);
 const char *dd_last_cuda_error(const dd_ctx *ctx);

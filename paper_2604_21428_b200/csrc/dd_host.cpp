@@ -44,6 +44,50 @@ extern "C" int dd_select_quorum(const double *arrival_s, int M, int K, double gr
     return DD_OK;
 }
 
+extern "C" int dd_plan_fragments(const uint64_t *size_bits, const int32_t *layer, int Q, int P,
+                                 dd_frag_strategy strategy, int32_t *fragment_of,
+                                 uint64_t *fragment_bits)
+{
+    if (Q < 0 || P < 1 || (Q > 0 && (!size_bits || !fragment_of))) return DD_ERR_INVALID_ARG;
+    std::vector<uint64_t> total((size_t)P, 0);
+    if (strategy == DD_FRAG_BALANCED) {
+        // Greedy number partitioning: largest tensor first, always into the lightest fragment.
+        std::vector<int> order((size_t)Q);
+        for (int q = 0; q < Q; ++q) order[(size_t)q] = q;
+        std::stable_sort(order.begin(), order.end(),
+                         [&](int a, int b) { return size_bits[a] > size_bits[b]; });
+        for (int q : order) {
+            int best = 0;
+            for (int p = 1; p < P; ++p)
+                if (total[(size_t)p] < total[(size_t)best]) best = p;
+            fragment_of[q] = best;
+            total[(size_t)best] += size_bits[q];
+        }
+    } else if (strategy == DD_FRAG_LAYER || strategy == DD_FRAG_TENSOR) {
+        if (!layer && Q > 0) return DD_ERR_INVALID_ARG;
+        int n_layers = 0;
+        for (int q = 0; q < Q; ++q) {
+            if (layer[q] < -1) return DD_ERR_INVALID_ARG;
+            n_layers = std::max(n_layers, layer[q] + 1);
+        }
+        const int buckets = P - 1;                   // fragment 0 is the non-transformer one
+        int next = 0;                                // running index of transformer tensors
+        for (int q = 0; q < Q; ++q) {
+            if (layer[q] < 0) { fragment_of[q] = 0; total[0] += size_bits[q]; continue; }
+            if (buckets < 1) return DD_ERR_INVALID_ARG;
+            if (strategy == DD_FRAG_LAYER && buckets > n_layers) return DD_ERR_INVALID_ARG;
+            const int key = strategy == DD_FRAG_LAYER ? layer[q] : next++;
+            fragment_of[q] = 1 + key % buckets;
+            total[(size_t)fragment_of[q]] += size_bits[q];
+        }
+    } else {
+        return DD_ERR_INVALID_ARG;
+    }
+    if (fragment_bits)
+        for (int p = 0; p < P; ++p) fragment_bits[p] = total[(size_t)p];
+    return DD_OK;
+}
+
 extern "C" const char *dd_status_string(int rc)
 {
     switch (rc) {

@@ -19,6 +19,7 @@ ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_ALIAS, ERR_TOO_MANY_LEARNERS, ERR_CUDA, ERR_
 STATUS_OK, STATUS_QUORUM_NOT_MET, STATUS_ZERO_WEIGHT, STATUS_WAIT_LIMIT = 0, 1, 2, 3
 HEAVY_BALL, DIAG_PER_LEARNER, DIAG_STATE = 1, 2, 4
 MERGE_AVG, MERGE_RDA = 0, 1
+FRAG_LAYER, FRAG_TENSOR, FRAG_BALANCED = 0, 1, 2
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libddmerge.so")
 
@@ -26,7 +27,7 @@ EXPORTS = (
     "dd_create", "dd_destroy", "dd_merge_fragment", "dd_merge_fragments_batched",
     "dd_merge_fragment_host", "dd_merge_fragments_batched_noalloc",
     "dd_merge_fragment_rda", "dd_merge_fragments_batched_rda",
-    "dd_select_quorum", "dd_grace_window", "dd_status_string", "dd_last_cuda_error",
+    "dd_plan_fragments", "dd_select_quorum", "dd_grace_window", "dd_status_string", "dd_last_cuda_error",
     "dd_launch_geometry",
 )
 
@@ -104,6 +105,10 @@ def _load() -> ctypes.CDLL:
     lib.dd_select_quorum.restype = ctypes.c_int
     lib.dd_select_quorum.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.c_int,
                                      ctypes.c_double, u64p, ctypes.POINTER(ctypes.c_int)]
+    lib.dd_plan_fragments.restype = ctypes.c_int
+    lib.dd_plan_fragments.argtypes = [u64p, ctypes.POINTER(ctypes.c_int32), ctypes.c_int,
+                                      ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int32),
+                                      u64p]
     lib.dd_grace_window.restype = ctypes.c_double
     lib.dd_grace_window.argtypes = [ctypes.c_double] * 5
     lib.dd_status_string.restype = ctypes.c_char_p
@@ -366,3 +371,18 @@ def grace_window(tau: float, xi_step: float, xi_quorum: float, xi_sync: float,
                  gamma: float) -> float:
     """``dd_grace_window``."""
     return float(lib.dd_grace_window(tau, xi_step, xi_quorum, xi_sync, gamma))
+
+
+def plan_fragments(size_bits, layer, P: int, strategy: int):
+    """``dd_plan_fragments``: returns (fragment index per tensor, total bits per fragment).
+    ``layer`` holds the 0-based transformer layer of each tensor or -1 (may be None for
+    FRAG_BALANCED)."""
+    Q = len(size_bits)
+    sizes = _u64_array(size_bits)
+    lay = None if layer is None else (ctypes.c_int32 * Q)(*[int(x) for x in layer])
+    out = (ctypes.c_int32 * max(Q, 1))()
+    totals = (ctypes.c_uint64 * max(P, 1))()
+    rc = lib.dd_plan_fragments(sizes, lay, Q, int(P), int(strategy), out, totals)
+    if rc != OK:
+        raise DDMergeError(rc)
+    return [int(out[q]) for q in range(Q)], [int(totals[p]) for p in range(P)]
