@@ -262,6 +262,22 @@ int dd_merge_fragments_batched_noalloc(const dd_fragment_desc *descs, int P, int
                                        void *cuda_stream);
 
 /*
+ * The learner side of a syncer update (Algorithm 1 step 3; Appendix "Mixing learner
+ * and syncer params"): for every learner m whose bit is set in apply_mask,
+ *     theta_m <- alpha * theta_m + (1 - alpha) * Theta'
+ * in the learner dtype (round to nearest even for bf16).  alpha = 0 -- what the
+ * paper settles on -- overwrites the copy with the global fragment.  Learners whose
+ * bit is clear are not touched (their pointers may be NULL).  Resetting the
+ * per-fragment counters is the caller's bookkeeping.
+ *
+ *   global        [device] float32[n], read only
+ *   learner_ptrs  [host]   M device pointers to learner_dtype[n], updated in place
+ */
+int dd_broadcast_fragment(dd_ctx *ctx, const float *global, void *const *learner_ptrs, int M,
+                          dd_dtype learner_dtype, uint64_t apply_mask, float alpha, size_t n,
+                          void *cuda_stream);
+
+/*
  * Quorum with grace window (Section 3.2, "Adaptive Quorum Window"), host only.
  * arrival_s[m] is when learner m's report arrived (+inf = never).  The syncer
  * may proceed at t_K, the K-th earliest arrival, and then waits grace_s longer:
@@ -278,6 +294,23 @@ int dd_select_quorum(const double *arrival_s, int M, int K, double grace_s,
  */
 double dd_grace_window(double tau, double xi_step, double xi_quorum, double xi_sync,
                        double gamma);
+
+/*
+ * Adaptive grace window (Section 3.2): the durations of a learner step, of reaching
+ * the quorum and of a synchronisation are tracked by exponential moving averages,
+ *     x <- beta * x + (1 - beta) * observation     (the first observation initialises x)
+ * and the window is dd_grace_window(tau, xi_step, xi_quorum, xi_sync, gamma).  The
+ * paper names the averages but not their coefficient: beta is the caller's.
+ * Plain data, host only; 0 <= beta < 1, 0 <= gamma < 1.
+ */
+typedef struct {
+    double tau, gamma, beta;
+    double xi_step, xi_quorum, xi_sync;
+    int32_t n_obs;
+} dd_grace_controller;
+int dd_grace_controller_init(dd_grace_controller *gc, double tau, double gamma, double beta);
+int dd_grace_controller_observe(dd_grace_controller *gc, double step_s, double quorum_s, double sync_s);
+double dd_grace_controller_window(const dd_grace_controller *gc);   /* 0 before the first observation */
 
 /*
  * Fragmentation planner (Appendix "Fragmentation strategies"), host only: assigns

@@ -89,6 +89,9 @@ def _load():
             ctypes.c_int, u64p, u64p, ctypes.c_uint64, ctypes.c_int, ctypes.c_float,
             ctypes.c_float, ctypes.c_int, ctypes.c_int, ctypes.c_size_t, ctypes.c_void_p,
             ctypes.POINTER(_Record)]
+        lib.ddo_apply_to_learner.restype = None
+        lib.ddo_apply_to_learner.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p,
+                                             ctypes.c_float, ctypes.c_size_t]
         lib.ddo_grace_window.restype = ctypes.c_double
         lib.ddo_grace_window.argtypes = [ctypes.c_double] * 5
         lib.ddo_select_quorum.restype = ctypes.c_int
@@ -204,3 +207,24 @@ def select_quorum(arrival, K: int, grace: float):
     if st == INVALID:
         raise ValueError("oracle: invalid quorum arguments")
     return st, int(mask.value), int(n_adm.value)
+
+
+def apply_to_learner(learner: np.ndarray, theta: np.ndarray, alpha: float) -> None:
+    """theta_m <- alpha theta_m + (1 - alpha) Theta, IN PLACE on ``learner`` (float32 or
+    uint16 holding bf16 bits)."""
+    lib = _load()
+    assert theta.dtype == np.float32 and learner.size == theta.size
+    assert learner.flags.c_contiguous and theta.flags.c_contiguous
+    lib.ddo_apply_to_learner(learner.ctypes.data, int(learner.dtype == np.uint16), theta.ctypes.data,
+                             ctypes.c_float(alpha), theta.size)
+
+
+def grace_controller_window(tau, gamma, beta, observations) -> float:
+    """Moving averages x <- beta x + (1 - beta) obs (first observation initialises),
+    then the largest admissible grace window; written out with plain floats."""
+    xs = None
+    for obs in observations:
+        xs = list(obs) if xs is None else [beta * x + (1.0 - beta) * o for x, o in zip(xs, obs)]
+    if xs is None:
+        return 0.0
+    return grace_window(tau, xs[0], xs[1], xs[2], gamma)

@@ -251,6 +251,21 @@ int ddo_merge_fragment(float *Theta, float *v, const void *const *learners, int 
     return 0;
 }
 
+/* ---- learner side of an update (Algorithm 1 step 3; appendix "Mixing learner and syncer params") */
+
+/* theta_m <- alpha theta_m + (1 - alpha) Theta, rounded to the learner dtype. */
+void ddo_apply_to_learner(void *learner, int learner_is_bf16, const float *Theta, float alpha,
+                          size_t n)
+{
+    const double a = (double)alpha;
+    size_t i;
+    for (i = 0; i < n; ++i) {
+        double x = a * learner_at(learner, learner_is_bf16, i) + (1.0 - a) * (double)Theta[i];
+        if (learner_is_bf16) ((uint16_t *)learner)[i] = ddo_bf16_rne((float)x);
+        else ((float *)learner)[i] = (float)x;
+    }
+}
+
 /* ---- quorum / grace window ("Adaptive Quorum Window", Section 3.2) --------- */
 
 /*

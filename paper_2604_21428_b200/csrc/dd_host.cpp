@@ -2,6 +2,7 @@
 // "Adaptive Quorum Window") and status strings.  No CUDA here.
 #include <algorithm>
 #include <cmath>
+#include <cstdint>
 #include <vector>
 
 #include "dd_merge.h"
@@ -13,6 +14,42 @@ extern "C" double dd_grace_window(double tau, double xi_step, double xi_quorum, 
     // without slack the syncer proceeds as soon as the quorum is met.
     const double slack = tau * xi_step - (xi_quorum + xi_sync);
     return std::max(0.0, gamma * slack);
+}
+
+extern "C" int dd_grace_controller_init(dd_grace_controller *gc, double tau, double gamma, double beta)
+{
+    if (!gc || !(tau > 0.0) || !(gamma >= 0.0 && gamma < 1.0) || !(beta >= 0.0 && beta < 1.0))
+        return DD_ERR_INVALID_ARG;
+    gc->tau = tau;
+    gc->gamma = gamma;
+    gc->beta = beta;
+    gc->xi_step = gc->xi_quorum = gc->xi_sync = 0.0;
+    gc->n_obs = 0;
+    return DD_OK;
+}
+
+extern "C" int dd_grace_controller_observe(dd_grace_controller *gc, double step_s, double quorum_s,
+                                           double sync_s)
+{
+    if (!gc || !(step_s >= 0.0) || !(quorum_s >= 0.0) || !(sync_s >= 0.0)) return DD_ERR_INVALID_ARG;
+    if (gc->n_obs == 0) {
+        gc->xi_step = step_s;
+        gc->xi_quorum = quorum_s;
+        gc->xi_sync = sync_s;
+    } else {
+        const double b = gc->beta;
+        gc->xi_step = b * gc->xi_step + (1.0 - b) * step_s;
+        gc->xi_quorum = b * gc->xi_quorum + (1.0 - b) * quorum_s;
+        gc->xi_sync = b * gc->xi_sync + (1.0 - b) * sync_s;
+    }
+    if (gc->n_obs < INT32_MAX) gc->n_obs += 1;
+    return DD_OK;
+}
+
+extern "C" double dd_grace_controller_window(const dd_grace_controller *gc)
+{
+    if (!gc || gc->n_obs == 0) return 0.0;
+    return dd_grace_window(gc->tau, gc->xi_step, gc->xi_quorum, gc->xi_sync, gc->gamma);
 }
 
 extern "C" int dd_select_quorum(const double *arrival_s, int M, int K, double grace_s,

@@ -27,7 +27,8 @@ EXPORTS = (
     "dd_create", "dd_destroy", "dd_merge_fragment", "dd_merge_fragments_batched",
     "dd_merge_fragment_host", "dd_merge_fragments_batched_noalloc",
     "dd_merge_fragment_rda", "dd_merge_fragments_batched_rda",
-    "dd_plan_fragments", "dd_select_quorum", "dd_grace_window", "dd_status_string", "dd_last_cuda_error",
+    "dd_broadcast_fragment", "dd_grace_controller_init", "dd_grace_controller_observe",
+    "dd_grace_controller_window", "dd_plan_fragments", "dd_select_quorum", "dd_grace_window", "dd_status_string", "dd_last_cuda_error",
     "dd_launch_geometry",
 )
 
@@ -60,6 +61,13 @@ class CFragmentDesc(ctypes.Structure):
         ("K", ctypes.c_int32),
         ("n", ctypes.c_uint64),
     ]
+
+
+class CGraceController(ctypes.Structure):
+    """Mirror of ``dd_grace_controller``."""
+    _fields_ = [("tau", ctypes.c_double), ("gamma", ctypes.c_double), ("beta", ctypes.c_double),
+                ("xi_step", ctypes.c_double), ("xi_quorum", ctypes.c_double),
+                ("xi_sync", ctypes.c_double), ("n_obs", ctypes.c_int32)]
 
 
 RECORD_BYTES = ctypes.sizeof(CRecord)
@@ -105,6 +113,16 @@ def _load() -> ctypes.CDLL:
     lib.dd_select_quorum.restype = ctypes.c_int
     lib.dd_select_quorum.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.c_int,
                                      ctypes.c_double, u64p, ctypes.POINTER(ctypes.c_int)]
+    lib.dd_broadcast_fragment.restype = ctypes.c_int
+    lib.dd_broadcast_fragment.argtypes = [vp, vp, ctypes.POINTER(vp), ctypes.c_int, ctypes.c_int,
+                                          ctypes.c_uint64, ctypes.c_float, ctypes.c_size_t, vp]
+    gcp = ctypes.POINTER(CGraceController)
+    lib.dd_grace_controller_init.restype = ctypes.c_int
+    lib.dd_grace_controller_init.argtypes = [gcp, ctypes.c_double, ctypes.c_double, ctypes.c_double]
+    lib.dd_grace_controller_observe.restype = ctypes.c_int
+    lib.dd_grace_controller_observe.argtypes = [gcp, ctypes.c_double, ctypes.c_double, ctypes.c_double]
+    lib.dd_grace_controller_window.restype = ctypes.c_double
+    lib.dd_grace_controller_window.argtypes = [gcp]
     lib.dd_plan_fragments.restype = ctypes.c_int
     lib.dd_plan_fragments.argtypes = [u64p, ctypes.POINTER(ctypes.c_int32), ctypes.c_int,
                                       ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int32),
@@ -270,6 +288,22 @@ class Context:
             ctypes.c_size_t(0 if scratch is None else int(scratch.numel())),
             _stream_handle(stream)))
 
+    def broadcast_fragment(self, global_, learners, apply_mask: int, alpha: float = 0.0, *,
+                           n: int | None = None, learner_dtype: int | None = None,
+                           stream=None) -> None:
+        """``dd_broadcast_fragment``: theta_m <- alpha theta_m + (1 - alpha) Theta' for the
+        learners selected by ``apply_mask``."""
+        M = len(learners)
+        if n is None:
+            n = int(global_.numel())
+        if learner_dtype is None:
+            learner_dtype = _infer_dtype(learners)
+        ptrs = (ctypes.c_void_p * M)(*[_ptr(t) for t in learners])
+        self._check(lib.dd_broadcast_fragment(
+            self._h, _ptr(global_), ptrs, M, learner_dtype,
+            ctypes.c_uint64(apply_mask & (2**64 - 1)), ctypes.c_float(alpha), ctypes.c_size_t(n),
+            _stream_handle(stream)))
+
     def merge_fragment_host(self, global_, momentum, learners, tokens, quorum_mask: int, K: int,
                             outer_lr: float, outer_mu: float, *, n: int | None = None,
                             learner_dtype: int | None = None, steps=None, flags: int = 0,
@@ -386,3 +420,26 @@ def plan_fragments(size_bits, layer, P: int, strategy: int):
     if rc != OK:
         raise DDMergeError(rc)
     return [int(out[q]) for q in range(Q)], [int(totals[p]) for p in range(P)]
+
+
+class GraceController:
+    """``dd_grace_controller``: moving averages of step / quorum / sync durations and the
+    grace window they allow."""
+
+    def __init__(self, tau: float, gamma: float, beta: float):
+        self._c = CGraceController()
+        rc = lib.dd_grace_controller_init(ctypes.byref(self._c), tau, gamma, beta)
+        if rc != OK:
+            raise DDMergeError(rc)
+
+    def observe(self, step_s: float, quorum_s: float, sync_s: float) -> None:
+        rc = lib.dd_grace_controller_observe(ctypes.byref(self._c), step_s, quorum_s, sync_s)
+        if rc != OK:
+            raise DDMergeError(rc)
+
+    def window(self) -> float:
+        return float(lib.dd_grace_controller_window(ctypes.byref(self._c)))
+
+    @property
+    def averages(self):
+        return self._c.xi_step, self._c.xi_quorum, self._c.xi_sync

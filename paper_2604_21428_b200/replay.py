@@ -1,0 +1,88 @@
+"""Syncer loop (Algorithm 2) driven by a recorded or synthetic event tape.
+
+A tape fixes, for every syncer step, when each learner's report arrived and the
+per-(learner, fragment) token / step counters it carried -- exactly what the
+paper's deterministic replay records ("participant subsets and token
+weightings").  ``Syncer.step`` turns one tape entry into library calls: quorum
+selection with the grace window, ONE batched merge launch over the fragments that
+are due, and the broadcast of the updated fragments to the learners that are
+alive.  All arithmetic happens in libddmerge; this module only sequences calls.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+from . import ddmerge as dd
+
+
+@dataclass
+class TapeEntry:
+    arrival_s: list                 # M arrival times of the reports (inf = no report)
+    tokens: list                    # P x M counters since the learner last received fragment p
+    steps: list | None = None       # P x M, optional
+
+
+@dataclass
+class StepResult:
+    due: list = field(default_factory=list)
+    mask: int = 0
+    n_admitted: int = 0
+    records: list = field(default_factory=list)
+
+
+class Syncer:
+    """Holds the global fragments and the outer momentum on one GPU."""
+
+    def __init__(self, ctx: "dd.Context", global_fragments, momentum_fragments, *, H: int,
+                 offsets, K: int, outer_lr: float, outer_mu: float, learner_dtype: int,
+                 merge_kinds=None, alpha: float = 0.0, flags: int = 0):
+        self.ctx = ctx
+        self.theta = list(global_fragments)
+        self.mom = list(momentum_fragments)
+        self.P = len(self.theta)
+        self.H, self.offsets, self.K = int(H), list(offsets), int(K)
+        self.lr, self.mu = float(outer_lr), float(outer_mu)
+        self.dtype = learner_dtype
+        self.kinds = list(merge_kinds) if merge_kinds is not None else [dd.MERGE_AVG] * self.P
+        self.alpha = float(alpha)
+        self.flags = int(flags)
+        self._records = dd.new_records(self.P, device=self.theta[0].device)
+
+    def due(self, t: int):
+        """Fragments synchronised at step t: those with t mod H equal to their offset."""
+        return [p for p in range(self.P) if t % self.H == self.offsets[p]]
+
+    def step(self, t: int, entry: TapeEntry, learner_fragments, grace_s: float = 0.0,
+             stream=None) -> StepResult:
+        """``learner_fragments[m][p]`` is learner m's device copy of fragment p (or None)."""
+        res = StepResult(due=self.due(t))
+        if not res.due:
+            return res
+        M = len(entry.arrival_s)
+        res.mask, res.n_admitted = dd.select_quorum(entry.arrival_s, self.K, grace_s)
+        frags = []
+        for p in res.due:
+            frags.append(dict(global_=self.theta[p], momentum=self.mom[p],
+                              learners=[learner_fragments[m][p] for m in range(M)],
+                              tokens=entry.tokens[p],
+                              steps=None if entry.steps is None else entry.steps[p],
+                              quorum_mask=res.mask, K=self.K, n=int(self.theta[p].numel())))
+        recs = self._records[: len(frags) * dd.RECORD_BYTES]
+        kinds = [self.kinds[p] for p in res.due]
+        if any(k == dd.MERGE_RDA for k in kinds):
+            self.ctx.merge_fragments_batched_rda(frags, M, self.dtype, self.lr, self.mu,
+                                                 merge_kinds=kinds, flags=self.flags, records=recs,
+                                                 stream=stream)
+        else:
+            self.ctx.merge_fragments_batched(frags, M, self.dtype, self.lr, self.mu,
+                                             flags=self.flags, records=recs, stream=stream)
+        res.records = dd.read_records(recs, len(frags))
+        # every learner that is alive receives the new fragment (and resets its counters)
+        alive = sum(1 << m for m in range(M) if entry.arrival_s[m] != float("inf"))
+        for p, rec in zip(res.due, res.records):
+            if rec.status == dd.STATUS_OK and alive:
+                self.ctx.broadcast_fragment(self.theta[p],
+                                            [learner_fragments[m][p] for m in range(M)], alive,
+                                            self.alpha, n=int(self.theta[p].numel()),
+                                            learner_dtype=self.dtype, stream=stream)
+        return res

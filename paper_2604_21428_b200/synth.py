@@ -215,3 +215,45 @@ def fill_fragment_gpu(theta, momentum, learners, seed: int, chunk: int = 1 << 26
             noise = torch.randn(hi - lo, generator=g, device=theta.device, dtype=torch.float32)
             noise.mul_(LEARNER_NOISE_STD).add_(base)
             t[lo:hi].copy_(noise)
+
+
+# ---- event tapes ------------------------------------------------------------------
+
+def synthetic_tape(M: int, P: int, H: int, offsets, steps_total: int, seed: int, *,
+                   batch_tokens: int = 4096, fail_prob: float = 0.08, recover_prob: float = 0.4,
+                   straggle_prob: float = 0.15):
+    """A seeded stand-in for a recorded event tape: per syncer step, the arrival time
+    of every learner's report (inf while the learner is down) and the per-(fragment,
+    learner) token / step counters accumulated since that learner last received the
+    fragment.  A learner that is up takes one inner step per syncer step (none when it
+    straggles); counters of a fragment are reset for every learner that is up when the
+    fragment is due (it then receives the new global fragment).
+    Returns a list of dicts {arrival_s, tokens, steps} (plain lists).
+    """
+    rng = np.random.default_rng(seed)
+    up = [True] * M
+    tokens = np.zeros((P, M), dtype=np.int64)
+    steps = np.zeros((P, M), dtype=np.int64)
+    tape = []
+    for t in range(steps_total):
+        arrival = []
+        for m in range(M):
+            if up[m] and rng.random() < fail_prob:
+                up[m] = False
+            elif not up[m] and rng.random() < recover_prob:
+                up[m] = True
+            if up[m]:
+                took = 0 if rng.random() < straggle_prob else 1
+                tokens[:, m] += took * batch_tokens * int(rng.integers(1, 3))
+                steps[:, m] += took
+                arrival.append(float(np.round(rng.lognormal(0.0, 0.5), 3)))
+            else:
+                arrival.append(float("inf"))
+        tape.append(dict(arrival_s=arrival, tokens=tokens.tolist(), steps=steps.tolist()))
+        for p in range(P):
+            if t % H == offsets[p]:
+                for m in range(M):
+                    if up[m]:
+                        tokens[p, m] = 0
+                        steps[p, m] = 0
+    return tape

@@ -386,3 +386,34 @@ def test_host_buffers_entry_point(dd, ctx, n, chunk):
                                   learner_dtype=dd.BF16)
     assert got.status == dd.STATUS_QUORUM_NOT_MET and got.n_part == 5
     assert torch.equal(before, h_theta)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("alpha", [0.0, 0.5, 0.25])
+def test_broadcast_to_learners(dd, ctx, dtype, alpha):
+    # learner side of an update: theta_m <- alpha theta_m + (1 - alpha) Theta'
+    n, M = 50_003, 5
+    theta, _, learners = synth.fragment_cpu(n, M, dtype, 91)
+    mask = 0b10110
+    t_dev = torch.from_numpy(theta).cuda()
+    full = [_guarded(a.view(np.int16) if dtype == "bf16" else a,
+                     torch.int16 if dtype == "bf16" else torch.float32) for a in learners]
+    views = [v.view(torch.bfloat16) if dtype == "bf16" else v for _, v in full]
+    ptrs = [views[m] if m != 0 else None for m in range(M)]          # learner 0: not selected, null
+    ctx.broadcast_fragment(t_dev, ptrs, mask, alpha, n=n, learner_dtype=dd.BF16 if dtype == "bf16" else dd.F32)
+    torch.cuda.synchronize()
+    for m in range(M):
+        got = views[m].cpu()
+        got = got.view(torch.int16).numpy().view(np.uint16) if dtype == "bf16" else got.numpy()
+        ref = learners[m].copy()
+        if (mask >> m) & 1:
+            oracle.apply_to_learner(ref, theta, alpha)
+            if alpha == 0.0:
+                np.testing.assert_array_equal(got, ref)
+            elif dtype == "bf16":
+                assert floor_rel_err(oracle.bf16_to_f32(got), oracle.bf16_to_f32(ref)) <= TOL_BF16
+                assert np.mean(got == ref) > 0.999
+            else:
+                assert floor_rel_err(got, ref) <= 1e-6
+        else:
+            np.testing.assert_array_equal(got, ref)                # untouched

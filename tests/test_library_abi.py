@@ -91,3 +91,20 @@ def test_select_quorum_rejects_bad_input(dd):
         dd.select_quorum([0.0, 1.0], 1, -1.0)
     with pytest.raises(dd.DDMergeError):
         dd.select_quorum([0.0] * 65, 1, 0.0)
+
+
+def test_grace_controller_matches_oracle(dd):
+    rng = np.random.default_rng(5)
+    for _ in range(50):
+        tau, gamma, beta = float(rng.uniform(1, 3)), float(rng.uniform(0, 0.99)), float(rng.uniform(0, 0.99))
+        gc = dd.GraceController(tau, gamma, beta)
+        assert gc.window() == 0.0
+        obs = [tuple(float(x) for x in rng.uniform(0, 2, 3)) for _ in range(int(rng.integers(1, 12)))]
+        for o in obs:
+            gc.observe(*o)
+        assert math.isclose(gc.window(), oracle.grace_controller_window(tau, gamma, beta, obs),
+                            rel_tol=1e-12, abs_tol=1e-15)
+    with pytest.raises(dd.DDMergeError):
+        dd.GraceController(2.0, 1.0, 0.5)           # gamma must stay below 1
+    with pytest.raises(dd.DDMergeError):
+        dd.GraceController(2.0, 0.5, 0.5).observe(-1.0, 0.0, 0.0)

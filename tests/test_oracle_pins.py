@@ -430,3 +430,34 @@ def test_rda_matches_definition():
     oracle.merge_fragment(theta, v, learners, tokens, _full_mask(M), M, 1.0, 0.0,
                           merge=oracle.MERGE_RDA)
     np.testing.assert_allclose(v, expect.astype(np.float32), rtol=1e-5, atol=1e-10)
+
+
+# ---- learner side: theta <- alpha theta + (1 - alpha) Theta ---------------------------
+
+def test_apply_to_learner_special_cases():
+    theta, _, learners = _frag(n=3000, M=2, dtype="bf16", seed=51)
+    before = learners[0].copy()
+    # alpha = 0 (the paper's choice): a plain overwrite with the rounded global fragment
+    oracle.apply_to_learner(learners[0], theta, 0.0)
+    ref = torch.from_numpy(theta).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    np.testing.assert_array_equal(learners[0], ref)
+    # alpha = 1: the learner keeps its copy
+    oracle.apply_to_learner(learners[1], theta, 1.0)
+    _, _, again = _frag(n=3000, M=2, dtype="bf16", seed=51)
+    np.testing.assert_array_equal(learners[1], again[1])
+    # alpha = 1/2 in float32: the midpoint
+    t32, _, l32 = _frag(n=3000, M=1, dtype="f32", seed=52)
+    mid = (0.5 * l32[0].astype(np.float64) + 0.5 * t32.astype(np.float64)).astype(np.float32)
+    oracle.apply_to_learner(l32[0], t32, 0.5)
+    np.testing.assert_array_equal(l32[0], mid)
+    assert not np.array_equal(before, learners[0])
+
+
+def test_grace_controller_moving_average_closed_form():
+    # constant observations: averages stay put; a step change decays geometrically
+    w = oracle.grace_controller_window(2.0, 0.5, 0.9, [(1.0, 0.2, 0.3)] * 7)
+    assert math.isclose(w, 0.5 * (2.0 * 1.0 - 0.5), rel_tol=1e-12)
+    obs = [(1.0, 0.0, 0.0)] + [(2.0, 0.0, 0.0)] * 5
+    xi = 2.0 - 0.9 ** 5                         # 1 -> 2 with beta = 0.9 after 5 updates
+    assert math.isclose(oracle.grace_controller_window(1.0, 0.5, 0.9, obs), 0.5 * xi, rel_tol=1e-12)
+    assert oracle.grace_controller_window(2.0, 0.5, 0.9, []) == 0.0
