@@ -7,11 +7,14 @@
 
 #include <cuda_runtime.h>
 
-#include "dd_merge_kernel.cuh"
+#include "dd_merge_tma.cuh"
 
 namespace ddm {
 
 // Resident CTAs of 256 threads per SM the kernels are compiled for (2 -> 128 registers per thread).
+#ifndef DD_USE_TMA
+#define DD_USE_TMA 1
+#endif
 #ifndef DD_MIN_BLOCKS
 #define DD_MIN_BLOCKS 2
 #endif
@@ -31,6 +34,22 @@ merge_batched_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ 
     merge_body<BF16, PL, kModeMerge>(frags, c);
 }
 
+// The staged (bulk-copy) form of the direct-averaging merge: what the library
+// launches whenever per-learner norms are not requested.
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads, 2)
+merge_single_tma_kernel(const __grid_constant__ DevFrag frag, const __grid_constant__ Common c)
+{
+    merge_body_tma<BF16>(&frag, c);
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads, 2)
+merge_batched_tma_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ Common c)
+{
+    merge_body_tma<BF16>(frags, c);
+}
+
 // One pass of a radial-directional merge over a batch of fragments.
 template <bool BF16, int MODE>
 __global__ void __launch_bounds__(kThreads, kMinBlocksPerSM)
@@ -44,6 +63,26 @@ rda_pass_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ Commo
 #include "dd_ctx.h"
 
 namespace ddm {
+
+template <bool BF16>
+static cudaError_t occupancy_tma(int *blocks)
+{
+    cudaError_t e = cudaFuncSetAttribute(merge_single_tma_kernel<BF16>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTmaRingBytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(merge_batched_tma_kernel<BF16>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTmaRingBytes);
+    if (e == cudaSuccess)
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, merge_batched_tma_kernel<BF16>,
+                                                          kThreads, kTmaRingBytes);
+    int b2 = 0;
+    if (e == cudaSuccess)
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2, merge_single_tma_kernel<BF16>,
+                                                          kThreads, kTmaRingBytes);
+    if (e == cudaSuccess && b2 < *blocks) *blocks = b2;
+    if (e == cudaSuccess && *blocks > 2) *blocks = 2;      // 16 warps x 2 pieces in flight is the sweet spot
+    return e;
+}
 
 template <bool BF16, bool PL>
 static cudaError_t occupancy(int *blocks)
@@ -175,6 +214,13 @@ template <bool BF16, bool PL>
 static cudaError_t launch(bool single, const DevFrag *one, const DevFrag *dev_frags,
                           const Common &c, unsigned grid, cudaStream_t stream)
 {
+    if (!PL && DD_USE_TMA) {
+        if (single)
+            merge_single_tma_kernel<BF16><<<grid, kThreads, kTmaRingBytes, stream>>>(*one, c);
+        else
+            merge_batched_tma_kernel<BF16><<<grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
+        return cudaGetLastError();
+    }
     if (single)
         merge_single_kernel<BF16, PL><<<grid, kThreads, 0, stream>>>(*one, c);
     else
@@ -209,9 +255,9 @@ extern "C" int dd_create(dd_ctx **out, int device)
     cudaError_t e = guard.ok ? cudaSuccess : cudaErrorInvalidDevice;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
     int occ[2][2] = {{0, 0}, {0, 0}};
-    if (e == cudaSuccess) e = occupancy<false, false>(&occ[0][0]);
+    if (e == cudaSuccess) e = DD_USE_TMA ? occupancy_tma<false>(&occ[0][0]) : occupancy<false, false>(&occ[0][0]);
     if (e == cudaSuccess) e = occupancy<false, true>(&occ[0][1]);
-    if (e == cudaSuccess) e = occupancy<true, false>(&occ[1][0]);
+    if (e == cudaSuccess) e = DD_USE_TMA ? occupancy_tma<true>(&occ[1][0]) : occupancy<true, false>(&occ[1][0]);
     if (e == cudaSuccess) e = occupancy<true, true>(&occ[1][1]);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();

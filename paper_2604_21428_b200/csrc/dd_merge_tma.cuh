@@ -1,0 +1,343 @@
+// The fused merge with its operands staged through shared memory by bulk
+// asynchronous copies (cp.async.bulk: the TMA engine, no tensor map, no
+// multicast).  Same arithmetic as process_vec; what changes is who moves the
+// bytes.  A warp owns a private ring of kTmaStages slots of 2 KB.  Its lane 0
+// asks the copy engine for the next 2 KB piece -- 1024 bf16 elements of one
+// learner copy, or 512 floats of Theta / v -- up to kTmaStages-1 pieces ahead of
+// the piece the warp is consuming, each piece signalling its own mbarrier.  The
+// loads therefore cost neither registers nor load/store-unit slots, and 2 KB
+// requests keep HBM streaming with only 16 warps per SM.
+//
+// Synchronisation is warp-local: lanes wait on the slot's mbarrier (try_wait in
+// a loop with an iteration limit; on giving up the warp records
+// DD_STATUS_WAIT_LIMIT, waits -- again bounded -- for its copies in flight and
+// leaves), and a slot is handed back to lane 0 by __syncwarp().  No CTA-wide
+// barrier, no flag shared between CTAs.
+#pragma once
+
+#include "dd_merge_kernel.cuh"
+
+#ifndef DD_TMA_STAGES
+#define DD_TMA_STAGES 3
+#endif
+
+namespace ddm {
+
+constexpr int kTmaStages = DD_TMA_STAGES;
+constexpr int kTmaChunk = 2048;                           // bytes per slot / per bulk copy
+constexpr int kSuperRow = 1024;                           // elements a warp merges per round (4 steps per lane)
+constexpr size_t kTmaRingBytes = (size_t)kWarps * kTmaStages * kTmaChunk;
+constexpr int kWaitLimit = 1 << 22;                       // try_wait attempts before giving up
+static_assert(kTileElems == kWarps * kSuperRow, "one super-row per warp per tile");
+
+__device__ __forceinline__ unsigned smem_addr(const void *p)
+{
+    return (unsigned)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(unsigned long long *bar, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_addr(bar)), "r"(count) : "memory");
+}
+
+// The issuing thread's arrival plus the number of bytes the copies will deliver.
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long *bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                 :: "r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long *bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+                 " selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+
+// Bounded wait for one phase of a slot's barrier.
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned long long *bar, unsigned parity)
+{
+    for (int spins = 0; spins < kWaitLimit; ++spins)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+
+// global -> this CTA's shared memory, 16-byte aligned on both sides, bytes % 16 == 0.
+__device__ __forceinline__ void bulk_copy_g2s(void *dst, const void *src, unsigned bytes,
+                                              unsigned long long *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+
+// Ring position of a warp; survives from one fragment to the next (the ring is
+// always drained in between, so producer and consumer meet at the same slot).
+struct TmaRing {
+    int islot = 0;           // next slot to fill
+    int cslot = 0;           // next slot to consume
+    unsigned cphase = 0;     // parity of the phase the consumer waits for
+    bool failed = false;     // a bounded wait gave up
+};
+
+// All tiles of the current fragment that belong to this CTA (tile, tile+G, ...):
+// warp w merges super-row w of each of them.  Pieces per super-row, in order:
+//   Theta[0:512) Theta[512:1024) | learner pieces (1 per bf16 copy, 2 per fp32 copy) | v[0:512) v[512:1024)
+template <bool BF16, bool WIDE>
+__device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
+                                                     unsigned long long tile, unsigned char *ring_base,
+                                                     unsigned long long *bars, TmaRing &rs)
+{
+    constexpr int LB = BF16 ? 1 : 2;                      // 2 KB pieces per learner per super-row
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned G = gridDim.x;
+    unsigned char *const ring = ring_base + (size_t)warp * kTmaStages * kTmaChunk;
+    unsigned long long *const bar = bars + warp * kTmaStages;
+    const unsigned nfull = (unsigned)(sm.n / kVec);
+    const unsigned long long tile_end = sm.tile_end, tile_begin = sm.tile_begin;
+    const int s = sm.n_part;
+    const int npieces = 4 + s * LB;
+    const float *const theta = sm.theta;
+    const float *const mom = sm.mom;
+
+    // first step (of 8 elements) of the super-row warp `warp` has in tile t
+    auto first_step = [&](unsigned long long t) {
+        return ((unsigned)(t - tile_begin) * kWarps + (unsigned)warp) * (unsigned)(kSuperRow / kVec);
+    };
+
+    // ---- producer (lane 0): one piece per call ---------------------------------------
+    unsigned long long itile = tile;
+    int ipiece = 0;
+    int outstanding = 0;
+    auto issue = [&]() {
+        if (rs.failed || itile >= tile_end) return;
+        const unsigned v0 = first_step(itile);
+        if (v0 >= nfull) { itile = tile_end; return; }
+        if (lane == 0) {
+            const unsigned cnt = min(128u, nfull - v0);            // steps in this super-row
+            const void *src;
+            unsigned bytes;
+            if (ipiece < 2 || ipiece >= 2 + s * LB) {              // Theta or v: halves of 64 steps x 32 B
+                const int half = ipiece < 2 ? ipiece : ipiece - (2 + s * LB);
+                const unsigned nv = cnt > 64u * half ? min(64u, cnt - 64u * half) : 0u;
+                src = (ipiece < 2 ? theta : mom) + 8ull * (v0 + 64u * half);
+                bytes = nv * 32u;
+            } else if (BF16) {
+                src = reinterpret_cast<const char *>(sm.ptr[ipiece - 2]) + 16ull * v0;
+                bytes = cnt * 16u;
+            } else {
+                const int j = (ipiece - 2) >> 1, half = (ipiece - 2) & 1;
+                const unsigned nv = cnt > 64u * half ? min(64u, cnt - 64u * half) : 0u;
+                src = reinterpret_cast<const char *>(sm.ptr[j]) + 32ull * (v0 + 64u * half);
+                bytes = nv * 32u;
+            }
+            mbar_arrive_expect_tx(bar + rs.islot, bytes);
+            if (bytes != 0) bulk_copy_g2s(ring + rs.islot * kTmaChunk, src, bytes, bar + rs.islot);
+        }
+        if (++ipiece == npieces) { ipiece = 0; itile += G; }
+        if (++rs.islot == kTmaStages) rs.islot = 0;
+        ++outstanding;
+    };
+    // ---- consumer: the next piece is in rs.cslot once its barrier flips -----------------
+    auto acquire = [&]() -> const unsigned char * {
+        __syncwarp();                                              // the slot consumed last is free again
+        if (!rs.failed) {
+            issue();
+            const bool ok = mbar_wait_bounded(bar + rs.cslot, rs.cphase);
+            if (!__all_sync(0xffffffffu, ok)) rs.failed = true;    // the whole warp gives up together
+        }
+        return ring + rs.cslot * kTmaChunk;
+    };
+    auto release = [&]() {
+        if (rs.failed) return;
+        if (++rs.cslot == kTmaStages) { rs.cslot = 0; rs.cphase ^= 1u; }
+        --outstanding;
+    };
+
+#pragma unroll 1
+    for (int p = 0; p < kTmaStages - 1; ++p) issue();
+
+    const float eta = c.eta, mu = c.mu;
+    const bool heavy = (c.flags & DD_HEAVY_BALL) != 0;
+#pragma unroll 1
+    for (unsigned long long ctile = tile; ctile < tile_end && !rs.failed; ctile += G) {
+        const unsigned v0 = first_step(ctile);
+        if (v0 >= nfull) break;
+        const unsigned cnt = min(128u, nfull - v0);
+        float2 nT[4][4], acc[4][4];
+        // Theta: two pieces of 64 steps; lane owns steps r*32 + lane, r = 0..3
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const unsigned char *slot = acquire();
+#pragma unroll
+            for (int rr = 0; rr < 2; ++rr) {
+                const int r = 2 * half + rr;
+                const uint4 *p = reinterpret_cast<const uint4 *>(slot + (rr * 32 + lane) * 32);
+                const uint4 a = p[0], b = p[1];
+                nT[r][0] = make_float2(-__uint_as_float(a.x), -__uint_as_float(a.y));
+                nT[r][1] = make_float2(-__uint_as_float(a.z), -__uint_as_float(a.w));
+                nT[r][2] = make_float2(-__uint_as_float(b.x), -__uint_as_float(b.y));
+                nT[r][3] = make_float2(-__uint_as_float(b.z), -__uint_as_float(b.w));
+#pragma unroll
+                for (int k = 0; k < 4; ++k) acc[r][k] = make_float2(0.0f, 0.0f);
+            }
+            release();
+        }
+        // acc = sum_j w_hat_j (theta_j - Theta) = -Delta; the difference first, then the weight
+#pragma unroll 1
+        for (int j = 0; j < s; ++j) {
+            const float w = sm.w[j];
+            const float2 w2 = make_float2(w, w);
+            if (BF16) {
+                const unsigned char *slot = acquire();
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const uint4 x = *reinterpret_cast<const uint4 *>(slot + r * 512 + lane * 16);
+                    const unsigned word[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float2 th = make_float2(__uint_as_float(word[k] << 16),
+                                                      __uint_as_float(word[k] & 0xffff0000u));
+                        acc[r][k] = __ffma2_rn(w2, __fadd2_rn(th, nT[r][k]), acc[r][k]);
+                    }
+                }
+                release();
+            } else {
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const unsigned char *slot = acquire();
+#pragma unroll
+                    for (int rr = 0; rr < 2; ++rr) {
+                        const int r = 2 * half + rr;
+                        const uint4 *p = reinterpret_cast<const uint4 *>(slot + (rr * 32 + lane) * 32);
+                        const uint4 a = p[0], b = p[1];
+                        const float2 th[4] = {make_float2(__uint_as_float(a.x), __uint_as_float(a.y)),
+                                              make_float2(__uint_as_float(a.z), __uint_as_float(a.w)),
+                                              make_float2(__uint_as_float(b.x), __uint_as_float(b.y)),
+                                              make_float2(__uint_as_float(b.z), __uint_as_float(b.w))};
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            acc[r][k] = __ffma2_rn(w2, __fadd2_rn(th[k], nT[r][k]), acc[r][k]);
+                    }
+                    release();
+                }
+            }
+        }
+        // v and the outer step: v' = mu v + Delta; Theta' = Theta - eta (Delta + mu v')
+        float dsq = 0.0f, tsq = 0.0f, msq = 0.0f;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const unsigned char *slot = acquire();
+#pragma unroll
+            for (int rr = 0; rr < 2; ++rr) {
+                const int r = 2 * half + rr;
+                const unsigned step = (unsigned)(r * 32 + lane);
+                const uint4 *p = reinterpret_cast<const uint4 *>(slot + (rr * 32 + lane) * 32);
+                const uint4 a = p[0], b = p[1];
+                float V[8] = {__uint_as_float(a.x), __uint_as_float(a.y), __uint_as_float(a.z),
+                              __uint_as_float(a.w), __uint_as_float(b.x), __uint_as_float(b.y),
+                              __uint_as_float(b.z), __uint_as_float(b.w)};
+                float T[8];
+                if (step < cnt && !rs.failed) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const float delta = -((k & 1) ? acc[r][k >> 1].y : acc[r][k >> 1].x);
+                        const float vn = fmaf(mu, V[k], delta);
+                        const float u = heavy ? vn : fmaf(mu, vn, delta);
+                        const float tn = fmaf(-eta, u, -((k & 1) ? nT[r][k >> 1].y : nT[r][k >> 1].x));
+                        V[k] = vn;
+                        T[k] = tn;
+                        dsq = fmaf(delta, delta, dsq);
+                        tsq = fmaf(tn, tn, tsq);
+                        msq = fmaf(vn, vn, msq);
+                    }
+                    const unsigned vi = v0 + step;
+                    store_f32x8<WIDE>(sm.mom, vi, V);
+                    store_f32x8<WIDE>(sm.theta, vi, T);
+                    if (sm.out_bf16 != nullptr)
+                        st_stream16(reinterpret_cast<uint4 *>(sm.out_bf16) + vi,
+                                    make_uint4(pack_bf16x2(T[0], T[1]), pack_bf16x2(T[2], T[3]),
+                                               pack_bf16x2(T[4], T[5]), pack_bf16x2(T[6], T[7])));
+                }
+            }
+            release();
+        }
+        if (c.records != nullptr) {
+            dsq = warp_sum(dsq);
+            tsq = warp_sum(tsq);
+            msq = warp_sum(msq);
+            if (lane == 0) {
+                sm.red[warp][0] += (double)dsq;
+                sm.red[warp][1] += (double)tsq;
+                sm.red[warp][2] += (double)msq;
+            }
+        }
+    }
+
+    if (rs.failed) {
+        // Give the copies still in flight a bounded chance to land before this
+        // warp's slots can be reused or the CTA exits, and say what happened.
+        for (int k = 0; k < outstanding; ++k) {
+            (void)mbar_wait_bounded(bar + rs.cslot, rs.cphase);
+            if (++rs.cslot == kTmaStages) { rs.cslot = 0; rs.cphase ^= 1u; }
+        }
+        rs.islot = rs.cslot;
+        if (lane == 0 && c.records != nullptr) atomicMax(&c.records[sm.frag].status, (int)DD_STATUS_WAIT_LIMIT);
+    }
+}
+
+// Kernel body of the staged merge (direct averaging, no per-learner norms).
+template <bool BF16>
+__device__ __forceinline__ void merge_body_tma(const DevFrag *frags, const Common &c)
+{
+    __shared__ Smem sm;
+    __shared__ unsigned long long bars[kWarps * kTmaStages];
+    extern __shared__ __align__(128) unsigned char ring_base[];
+    const unsigned G = gridDim.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0)
+        for (int d = 0; d < kTmaStages; ++d) mbar_init(bars + warp * kTmaStages + d, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+
+    TmaRing rs;
+    int cur = -1;
+    unsigned long long tile = blockIdx.x;
+    while (tile < c.total_tiles) {
+        __syncthreads();
+        if (threadIdx.x < 32) {
+            cur = find_frag(frags, cur < 0 ? 0 : cur + 1, c.P, tile);
+            load_header<kModeMerge>(frags + cur, cur, tile, c, sm);
+        }
+        __syncthreads();
+        cur = sm.frag;
+        const unsigned long long tile_end = sm.tile_end;
+        const unsigned long long mine = (tile_end - tile + G - 1) / G;      // this CTA's tiles in the fragment
+        if (sm.status == DD_STATUS_OK) {
+            if (!rs.failed) {
+                if (sm.wide) process_fragment_tma<BF16, true>(sm, c, tile, ring_base, bars, rs);
+                else process_fragment_tma<BF16, false>(sm, c, tile, ring_base, bars, rs);
+            }
+            const int rem = (int)(sm.n % kVec);
+            if (rem != 0 && warp == 0 && tile + (mine - 1) * G == tile_end - 1) {
+                float dsq = 0.0f, tsq = 0.0f, msq = 0.0f;
+                process_tail<BF16, false, kModeMerge>(sm, c, (sm.n / kVec) * kVec, rem, dsq, tsq, msq);
+                if (c.records != nullptr) {
+                    dsq = warp_sum(dsq);
+                    tsq = warp_sum(tsq);
+                    msq = warp_sum(msq);
+                    if (lane == 0) {
+                        sm.red[0][0] += (double)dsq;
+                        sm.red[0][1] += (double)tsq;
+                        sm.red[0][2] += (double)msq;
+                    }
+                }
+            }
+            if (c.records != nullptr) flush_fragment<false>(sm, c);
+        }
+        tile += mine * G;
+    }
+}
+
+}  // namespace ddm
