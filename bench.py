@@ -29,7 +29,7 @@ UNIT = "params/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per merged parameter of the merge
 # kernel, from the ncu capture summarised under profiles/ (None until captured).
-NCU_TRAFFIC_BYTES_PER_PARAM = {"scale500m": 62.84}
+NCU_TRAFFIC_BYTES_PER_PARAM = {"scale500m": 63.04}
 
 
 def parse_args():

@@ -27,7 +27,8 @@ constexpr int kTmaStages = DD_TMA_STAGES;
 constexpr int kTmaChunk = 2048;                           // bytes per slot / per bulk copy
 constexpr int kSuperRow = 1024;                           // elements a warp merges per round (4 steps per lane)
 constexpr size_t kTmaRingBytes = (size_t)kWarps * kTmaStages * kTmaChunk;
-constexpr int kWaitLimit = 1 << 22;                       // try_wait attempts before giving up
+constexpr int kWaitLimit = 1 << 18;                       // try_wait attempts before giving up
+constexpr unsigned kWaitHintNs = 4000;                    // each attempt may sleep this long (~1 s in all)
 static_assert(kTileElems == kWarps * kSuperRow, "one super-row per warp per tile");
 
 __device__ __forceinline__ unsigned smem_addr(const void *p)
@@ -50,9 +51,10 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long *bar, u
 __device__ __forceinline__ bool mbar_try_wait(unsigned long long *bar, unsigned parity)
 {
     unsigned ok;
-    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+    // The attempt suspends the thread until the phase completes or the hint expires.
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
                  " selp.u32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity), "r"(kWaitHintNs) : "memory");
     return ok != 0;
 }
 
