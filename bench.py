@@ -43,7 +43,9 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-sample", type=int, default=1 << 25,
+    ap.add_argument("--no-ceilings", action="store_true",
+                    help="skip the same-run copy / read bandwidth ceilings (torch kernels)")
+    ap.add_argument("--cpu-sample", type=int, default=1 << 27,
                     help="elements of the workload the CPU oracle is timed on")
     ap.add_argument("--out-bf16", action="store_true", help="also write the bf16 broadcast copy")
     ap.add_argument("--merge", choices=["avg", "rda"], default="avg",
@@ -131,6 +133,33 @@ def hbm_peak():
             return float(json.load(f)["hbm_gbs"]), "measured"
     except Exception:
         return FALLBACK_HBM_GBS, "fallback"
+
+
+def measure_ceilings(device, reps=10):
+    """What this machine gives plain streaming kernels in the same run (torch library
+    kernels, not the product): a device-to-device copy and a read-only reduction."""
+    import torch
+
+    n = 1 << 29                                        # 2 GiB of float32 per array
+    a = torch.ones(n, dtype=torch.float32, device=device)
+    b = torch.empty_like(a)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    out = {}
+    for name, fn, nbytes in (("copy_ceiling_gbs", lambda: b.copy_(a), 8 * n),
+                             ("read_ceiling_gbs", lambda: a.sum(), 4 * n)):
+        for _ in range(3):
+            fn()
+        best = None
+        for _ in range(reps):
+            ev0.record()
+            fn()
+            ev1.record()
+            ev1.synchronize()
+            ms = ev0.elapsed_time(ev1)
+            best = ms if best is None or ms < best else best
+        out[name] = nbytes / (best * 1e-3) / 1e9
+    del a, b
+    return out
 
 
 # ---- the reference arm: the CPU oracle ------------------------------------------------
@@ -305,6 +334,8 @@ def main():
                       "slowest_steps": slowest},
         "frac_of_nominal_8TBs": achieved / 8000.0,
     }
+    if not args.no_ceilings:
+        roofline["same_run_ceilings"] = measure_ceilings(device)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -70,7 +70,13 @@ enum {
 enum {
     DD_HEAVY_BALL = 1u << 0,        /* Theta' = Theta - lr v' instead of the Nesterov form */
     DD_DIAG_PER_LEARNER = 1u << 1,  /* also ||Theta - theta_m||^2 for every participant */
-    DD_DIAG_STATE = 1u << 2         /* also ||Theta'||^2 and ||v'||^2 */
+    DD_DIAG_STATE = 1u << 2,        /* also ||Theta'||^2 and ||v'||^2 */
+    /* Test hook for the error path, not for production: every warp's first bulk copy
+     * is made to wait for bytes that never come, so its bounded wait expires (about a
+     * second), the fragment's record reports DD_STATUS_WAIT_LIMIT and the kernel
+     * returns normally with the context still usable.  Needs a record; the
+     * fragment's state is unspecified afterwards. */
+    DD_DEBUG_EXPIRE_WAIT = 1u << 30
 };
 
 /*

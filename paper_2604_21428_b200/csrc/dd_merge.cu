@@ -159,7 +159,8 @@ static int check_common(const dd_ctx *ctx, int M, dd_dtype dtype, float lr, floa
     if (M < 1) return DD_ERR_INVALID_ARG;
     if (dtype != DD_F32 && dtype != DD_BF16) return DD_ERR_INVALID_ARG;
     if (!std::isfinite(lr) || !std::isfinite(mu)) return DD_ERR_INVALID_ARG;
-    if (flags & ~(uint32_t)(DD_HEAVY_BALL | DD_DIAG_PER_LEARNER | DD_DIAG_STATE)) return DD_ERR_INVALID_ARG;
+    if (flags & ~(uint32_t)(DD_HEAVY_BALL | DD_DIAG_PER_LEARNER | DD_DIAG_STATE | DD_DEBUG_EXPIRE_WAIT))
+        return DD_ERR_INVALID_ARG;
     return DD_OK;
 }
 

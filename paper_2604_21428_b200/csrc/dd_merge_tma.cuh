@@ -134,7 +134,9 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
                 src = reinterpret_cast<const char *>(sm.ptr[j]) + 32ull * (v0 + 64u * half);
                 bytes = nv * 32u;
             }
-            mbar_arrive_expect_tx(bar + rs.islot, bytes);
+            // (test hook) announce 16 bytes that no copy will deliver: the wait must expire
+            const unsigned phantom = (c.flags & DD_DEBUG_EXPIRE_WAIT) && itile == tile && ipiece == 0 ? 16u : 0u;
+            mbar_arrive_expect_tx(bar + rs.islot, bytes + phantom);
             if (bytes != 0) bulk_copy_g2s(ring + rs.islot * kTmaChunk, src, bytes, bar + rs.islot);
         }
         if (++ipiece == npieces) { ipiece = 0; itile += G; }

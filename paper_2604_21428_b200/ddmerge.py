@@ -18,6 +18,7 @@ ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_ALIAS, ERR_TOO_MANY_LEARNERS, ERR_CUDA, ERR_
     -1, -2, -3, -4, -5, -6
 STATUS_OK, STATUS_QUORUM_NOT_MET, STATUS_ZERO_WEIGHT, STATUS_WAIT_LIMIT = 0, 1, 2, 3
 HEAVY_BALL, DIAG_PER_LEARNER, DIAG_STATE = 1, 2, 4
+DEBUG_EXPIRE_WAIT = 1 << 30
 MERGE_AVG, MERGE_RDA = 0, 1
 FRAG_LAYER, FRAG_TENSOR, FRAG_BALANCED = 0, 1, 2
 

@@ -417,3 +417,29 @@ def test_broadcast_to_learners(dd, ctx, dtype, alpha):
                 assert floor_rel_err(got, ref) <= 1e-6
         else:
             np.testing.assert_array_equal(got, ref)                # untouched
+
+
+def test_bounded_wait_expires_and_context_survives(dd, ctx):
+    # Error path of the staged kernel: with the test hook every warp's first copy waits
+    # for bytes that never come; the bounded wait gives up after about a second, the
+    # record says so, nothing hangs, and the same context merges correctly afterwards.
+    n, M = 20_000, 3
+    theta, v, learners = synth.fragment_cpu(n, M, "bf16", 61)
+    t_dev, v_dev = torch.from_numpy(theta).cuda(), torch.from_numpy(v).cuda()
+    L = [to_torch_learner(a, "cuda") for a in learners]
+    rec_buf = dd.new_records(1)
+    ctx.merge_fragment(t_dev, v_dev, L, [1, 2, 3], 0b111, 1, ETA, MU, flags=dd.DEBUG_EXPIRE_WAIT,
+                       record=rec_buf)
+    torch.cuda.synchronize()
+    rec = dd.read_records(rec_buf)[0]
+    assert rec.status == dd.STATUS_WAIT_LIMIT and rec.idx == [0, 1, 2]
+    # the context and the device are still healthy: a normal merge matches the oracle
+    t_dev.copy_(torch.from_numpy(theta))
+    v_dev.copy_(torch.from_numpy(v))
+    ref = oracle.merge_fragment(theta, v, learners, [1, 2, 3], 0b111, 1, ETA, MU)
+    ctx.merge_fragment(t_dev, v_dev, L, [1, 2, 3], 0b111, 1, ETA, MU, flags=dd.DIAG_STATE,
+                       record=rec_buf)
+    torch.cuda.synchronize()
+    assert_record_matches(dd.read_records(rec_buf)[0], ref, per_learner=False)
+    assert floor_rel_err(t_dev.cpu().numpy(), theta) <= TOL_STATE
+    assert floor_rel_err(v_dev.cpu().numpy(), v) <= TOL_STATE
