@@ -11,51 +11,31 @@
 
 namespace ddm {
 
-// Resident CTAs of 256 threads per SM the kernels are compiled for (2 -> 128 registers per thread).
-#ifndef DD_USE_TMA
-#define DD_USE_TMA 1
-#endif
-#ifndef DD_MIN_BLOCKS
-#define DD_MIN_BLOCKS 2
-#endif
-constexpr int kMinBlocksPerSM = DD_MIN_BLOCKS;
+// Every kernel runs 2 CTAs of 256 threads per SM (up to 128 registers per thread),
+// each CTA with kTmaRingBytes of dynamic shared memory for its warps' rings.
 
+// Direct averaging, one fragment passed by value in the kernel parameters.
 template <bool BF16, bool PL>
-__global__ void __launch_bounds__(kThreads, kMinBlocksPerSM)
-merge_single_kernel(const __grid_constant__ DevFrag frag, const __grid_constant__ Common c)
-{
-    merge_body<BF16, PL, kModeMerge>(&frag, c);
-}
-
-template <bool BF16, bool PL>
-__global__ void __launch_bounds__(kThreads, kMinBlocksPerSM)
-merge_batched_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ Common c)
-{
-    merge_body<BF16, PL, kModeMerge>(frags, c);
-}
-
-// The staged (bulk-copy) form of the direct-averaging merge: what the library
-// launches whenever per-learner norms are not requested.
-template <bool BF16>
 __global__ void __launch_bounds__(kThreads, 2)
 merge_single_tma_kernel(const __grid_constant__ DevFrag frag, const __grid_constant__ Common c)
 {
-    merge_body_tma<BF16>(&frag, c);
+    merge_body_tma<BF16, kModeMerge, PL>(&frag, c);
 }
 
-template <bool BF16>
+// Direct averaging, many fragments from a descriptor table in global memory.
+template <bool BF16, bool PL>
 __global__ void __launch_bounds__(kThreads, 2)
 merge_batched_tma_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ Common c)
 {
-    merge_body_tma<BF16>(frags, c);
+    merge_body_tma<BF16, kModeMerge, PL>(frags, c);
 }
 
 // One pass of a radial-directional merge over a batch of fragments.
 template <bool BF16, int MODE>
-__global__ void __launch_bounds__(kThreads, kMinBlocksPerSM)
+__global__ void __launch_bounds__(kThreads, 2)
 rda_pass_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ Common c)
 {
-    merge_body<BF16, MODE == kModeNorms, MODE>(frags, c);
+    merge_body_tma<BF16, MODE, MODE == kModeNorms>(frags, c);
 }
 
 }  // namespace ddm
@@ -64,35 +44,30 @@ rda_pass_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ Commo
 
 namespace ddm {
 
-template <bool BF16>
-static cudaError_t occupancy_tma(int *blocks)
+// Opts a kernel in to its dynamic shared memory and reports how many CTAs fit on an SM.
+template <typename K>
+static cudaError_t prepare_kernel(K kernel, int *blocks)
 {
-    cudaError_t e = cudaFuncSetAttribute(merge_single_tma_kernel<BF16>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTmaRingBytes);
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)kTmaRingBytes);
+    int b = 0;
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(merge_batched_tma_kernel<BF16>,
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTmaRingBytes);
-    if (e == cudaSuccess)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, merge_batched_tma_kernel<BF16>,
-                                                          kThreads, kTmaRingBytes);
-    int b2 = 0;
-    if (e == cudaSuccess)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2, merge_single_tma_kernel<BF16>,
-                                                          kThreads, kTmaRingBytes);
-    if (e == cudaSuccess && b2 < *blocks) *blocks = b2;
-    if (e == cudaSuccess && *blocks > 2) *blocks = 2;      // 16 warps x 2 pieces in flight is the sweet spot
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kernel, kThreads, kTmaRingBytes);
+    if (e == cudaSuccess && b < *blocks) *blocks = b;
     return e;
 }
 
 template <bool BF16, bool PL>
 static cudaError_t occupancy(int *blocks)
 {
-    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-        blocks, merge_batched_kernel<BF16, PL>, kThreads, 0);
-    if (e != cudaSuccess) return e;
-    int b2 = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2, merge_single_kernel<BF16, PL>, kThreads, 0);
-    if (e == cudaSuccess && b2 < *blocks) *blocks = b2;
+    *blocks = 2;      // 16 warps x 2 pieces in flight per SM is the measured sweet spot
+    cudaError_t e = prepare_kernel(merge_single_tma_kernel<BF16, PL>, blocks);
+    if (e == cudaSuccess) e = prepare_kernel(merge_batched_tma_kernel<BF16, PL>, blocks);
+    if (PL) {         // the RDA passes share the grid of the per-learner-norm variants
+        if (e == cudaSuccess) e = prepare_kernel(rda_pass_kernel<BF16, kModeNorms>, blocks);
+        if (e == cudaSuccess) e = prepare_kernel(rda_pass_kernel<BF16, kModeDir>, blocks);
+        if (e == cudaSuccess) e = prepare_kernel(rda_pass_kernel<BF16, kModeApply>, blocks);
+    }
     return e;
 }
 
@@ -215,17 +190,10 @@ template <bool BF16, bool PL>
 static cudaError_t launch(bool single, const DevFrag *one, const DevFrag *dev_frags,
                           const Common &c, unsigned grid, cudaStream_t stream)
 {
-    if (!PL && DD_USE_TMA) {
-        if (single)
-            merge_single_tma_kernel<BF16><<<grid, kThreads, kTmaRingBytes, stream>>>(*one, c);
-        else
-            merge_batched_tma_kernel<BF16><<<grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
-        return cudaGetLastError();
-    }
     if (single)
-        merge_single_kernel<BF16, PL><<<grid, kThreads, 0, stream>>>(*one, c);
+        merge_single_tma_kernel<BF16, PL><<<grid, kThreads, kTmaRingBytes, stream>>>(*one, c);
     else
-        merge_batched_kernel<BF16, PL><<<grid, kThreads, 0, stream>>>(dev_frags, c);
+        merge_batched_tma_kernel<BF16, PL><<<grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
     return cudaGetLastError();
 }
 
@@ -256,9 +224,9 @@ extern "C" int dd_create(dd_ctx **out, int device)
     cudaError_t e = guard.ok ? cudaSuccess : cudaErrorInvalidDevice;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
     int occ[2][2] = {{0, 0}, {0, 0}};
-    if (e == cudaSuccess) e = DD_USE_TMA ? occupancy_tma<false>(&occ[0][0]) : occupancy<false, false>(&occ[0][0]);
+    if (e == cudaSuccess) e = occupancy<false, false>(&occ[0][0]);
     if (e == cudaSuccess) e = occupancy<false, true>(&occ[0][1]);
-    if (e == cudaSuccess) e = DD_USE_TMA ? occupancy_tma<true>(&occ[1][0]) : occupancy<true, false>(&occ[1][0]);
+    if (e == cudaSuccess) e = occupancy<true, false>(&occ[1][0]);
     if (e == cudaSuccess) e = occupancy<true, true>(&occ[1][1]);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
@@ -398,9 +366,9 @@ template <bool BF16>
 static cudaError_t launch_rda_passes(const DevFrag *dev_frags, const Common &c, unsigned grid,
                                      cudaStream_t stream)
 {
-    rda_pass_kernel<BF16, kModeNorms><<<grid, kThreads, 0, stream>>>(dev_frags, c);
-    rda_pass_kernel<BF16, kModeDir><<<grid, kThreads, 0, stream>>>(dev_frags, c);
-    rda_pass_kernel<BF16, kModeApply><<<grid, kThreads, 0, stream>>>(dev_frags, c);
+    rda_pass_kernel<BF16, kModeNorms><<<grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
+    rda_pass_kernel<BF16, kModeDir><<<grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
+    rda_pass_kernel<BF16, kModeApply><<<grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
     return cudaGetLastError();
 }
 

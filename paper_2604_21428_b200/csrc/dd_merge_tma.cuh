@@ -86,7 +86,11 @@ struct TmaRing {
 // All tiles of the current fragment that belong to this CTA (tile, tile+G, ...):
 // warp w merges super-row w of each of them.  Pieces per super-row, in order:
 //   Theta[0:512) Theta[512:1024) | learner pieces (1 per bf16 copy, 2 per fp32 copy) | v[0:512) v[512:1024)
-template <bool BF16, bool WIDE>
+// The passes of a radial-directional merge use the same pipeline: the norms and
+// direction passes have no v pieces; the apply pass reads the two halves of the
+// stored direction u in place of the learner pieces.  PL adds the per-participant
+// squared norms of the outer gradients (always on in the norms pass).
+template <bool BF16, bool WIDE, int MODE, bool PL>
 __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
                                                      unsigned long long tile, unsigned char *ring_base,
                                                      unsigned long long *bars, TmaRing &rs)
@@ -99,7 +103,10 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
     const unsigned nfull = (unsigned)(sm.n / kVec);
     const unsigned long long tile_end = sm.tile_end, tile_begin = sm.tile_begin;
     const int s = sm.n_part;
-    const int npieces = 4 + s * LB;
+    constexpr bool kHasV = MODE == kModeMerge || MODE == kModeApply;
+    constexpr bool kNorms = PL || MODE == kModeNorms;
+    const int nmid = MODE == kModeApply ? 2 : s * LB;      // pieces between Theta and v
+    const int npieces = 2 + nmid + (kHasV ? 2 : 0);
     const float *const theta = sm.theta;
     const float *const mom = sm.mom;
 
@@ -120,10 +127,12 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
             const unsigned cnt = min(128u, nfull - v0);            // steps in this super-row
             const void *src;
             unsigned bytes;
-            if (ipiece < 2 || ipiece >= 2 + s * LB) {              // Theta or v: halves of 64 steps x 32 B
-                const int half = ipiece < 2 ? ipiece : ipiece - (2 + s * LB);
+            if (ipiece < 2 || ipiece >= 2 + nmid || MODE == kModeApply) {
+                // float32 operand (Theta, stored direction, v): halves of 64 steps x 32 B
+                const float *base = ipiece < 2 ? theta : (ipiece < 2 + nmid ? sm.scratch : mom);
+                const int half = ipiece < 2 ? ipiece : (ipiece < 2 + nmid ? ipiece - 2 : ipiece - 2 - nmid);
                 const unsigned nv = cnt > 64u * half ? min(64u, cnt - 64u * half) : 0u;
-                src = (ipiece < 2 ? theta : mom) + 8ull * (v0 + 64u * half);
+                src = base + 8ull * (v0 + 64u * half);
                 bytes = nv * 32u;
             } else if (BF16) {
                 src = reinterpret_cast<const char *>(sm.ptr[ipiece - 2]) + 16ull * v0;
@@ -188,84 +197,137 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
             }
             release();
         }
-        // acc = sum_j w_hat_j (theta_j - Theta) = -Delta; the difference first, then the weight
-#pragma unroll 1
-        for (int j = 0; j < s; ++j) {
-            const float w = sm.w[j];
-            const float2 w2 = make_float2(w, w);
-            if (BF16) {
+        if (MODE == kModeApply) {
+            // Delta = cscale * u: the stored mean direction, two halves
+            const float cs = sm.cscale;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
                 const unsigned char *slot = acquire();
 #pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const uint4 x = *reinterpret_cast<const uint4 *>(slot + r * 512 + lane * 16);
-                    const unsigned word[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const float2 th = make_float2(__uint_as_float(word[k] << 16),
-                                                      __uint_as_float(word[k] & 0xffff0000u));
-                        acc[r][k] = __ffma2_rn(w2, __fadd2_rn(th, nT[r][k]), acc[r][k]);
-                    }
+                for (int rr = 0; rr < 2; ++rr) {
+                    const int r = 2 * half + rr;
+                    const uint4 *p = reinterpret_cast<const uint4 *>(slot + (rr * 32 + lane) * 32);
+                    const uint4 a = p[0], b = p[1];
+                    acc[r][0] = make_float2(-cs * __uint_as_float(a.x), -cs * __uint_as_float(a.y));
+                    acc[r][1] = make_float2(-cs * __uint_as_float(a.z), -cs * __uint_as_float(a.w));
+                    acc[r][2] = make_float2(-cs * __uint_as_float(b.x), -cs * __uint_as_float(b.y));
+                    acc[r][3] = make_float2(-cs * __uint_as_float(b.z), -cs * __uint_as_float(b.w));
                 }
                 release();
-            } else {
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {
+            }
+        } else {
+            // acc = sum_j w_j (theta_j - Theta) = -Delta; the difference first, then the weight
+#pragma unroll 1
+            for (int j = 0; j < s; ++j) {
+                const float w = sm.w[j];
+                const float2 w2 = make_float2(w, w);
+                float q = 0.0f;
+                if (BF16) {
                     const unsigned char *slot = acquire();
 #pragma unroll
-                    for (int rr = 0; rr < 2; ++rr) {
-                        const int r = 2 * half + rr;
-                        const uint4 *p = reinterpret_cast<const uint4 *>(slot + (rr * 32 + lane) * 32);
-                        const uint4 a = p[0], b = p[1];
-                        const float2 th[4] = {make_float2(__uint_as_float(a.x), __uint_as_float(a.y)),
-                                              make_float2(__uint_as_float(a.z), __uint_as_float(a.w)),
-                                              make_float2(__uint_as_float(b.x), __uint_as_float(b.y)),
-                                              make_float2(__uint_as_float(b.z), __uint_as_float(b.w))};
+                    for (int r = 0; r < 4; ++r) {
+                        const uint4 x = *reinterpret_cast<const uint4 *>(slot + r * 512 + lane * 16);
+                        const unsigned word[4] = {x.x, x.y, x.z, x.w};
+                        float qr = 0.0f;
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            acc[r][k] = __ffma2_rn(w2, __fadd2_rn(th[k], nT[r][k]), acc[r][k]);
+                        for (int k = 0; k < 4; ++k) {
+                            const float2 th = make_float2(__uint_as_float(word[k] << 16),
+                                                          __uint_as_float(word[k] & 0xffff0000u));
+                            const float2 d = __fadd2_rn(th, nT[r][k]);
+                            if (MODE != kModeNorms) acc[r][k] = __ffma2_rn(w2, d, acc[r][k]);
+                            if (kNorms) qr = fmaf(d.x, d.x, fmaf(d.y, d.y, qr));
+                        }
+                        if (kNorms && (unsigned)(r * 32 + lane) < cnt) q += qr;
                     }
                     release();
+                } else {
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        const unsigned char *slot = acquire();
+#pragma unroll
+                        for (int rr = 0; rr < 2; ++rr) {
+                            const int r = 2 * half + rr;
+                            const uint4 *p = reinterpret_cast<const uint4 *>(slot + (rr * 32 + lane) * 32);
+                            const uint4 a = p[0], b = p[1];
+                            const float2 th[4] = {make_float2(__uint_as_float(a.x), __uint_as_float(a.y)),
+                                                  make_float2(__uint_as_float(a.z), __uint_as_float(a.w)),
+                                                  make_float2(__uint_as_float(b.x), __uint_as_float(b.y)),
+                                                  make_float2(__uint_as_float(b.z), __uint_as_float(b.w))};
+                            float qr = 0.0f;
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const float2 d = __fadd2_rn(th[k], nT[r][k]);
+                                if (MODE != kModeNorms) acc[r][k] = __ffma2_rn(w2, d, acc[r][k]);
+                                if (kNorms) qr = fmaf(d.x, d.x, fmaf(d.y, d.y, qr));
+                            }
+                            if (kNorms && (unsigned)(r * 32 + lane) < cnt) q += qr;
+                        }
+                        release();
+                    }
+                }
+                if (kNorms && !rs.failed) {
+                    q = warp_sum(q);
+                    if (lane == 0) sm.dm[warp][j] += (double)q;
                 }
             }
         }
-        // v and the outer step: v' = mu v + Delta; Theta' = Theta - eta (Delta + mu v')
+        if (MODE == kModeNorms) continue;
+
         float dsq = 0.0f, tsq = 0.0f, msq = 0.0f;
+        if (MODE == kModeDir) {
+            // the mean direction u = sum_j a_j (Theta - theta_j), kept for the apply pass
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            const unsigned char *slot = acquire();
-#pragma unroll
-            for (int rr = 0; rr < 2; ++rr) {
-                const int r = 2 * half + rr;
+            for (int r = 0; r < 4; ++r) {
                 const unsigned step = (unsigned)(r * 32 + lane);
-                const uint4 *p = reinterpret_cast<const uint4 *>(slot + (rr * 32 + lane) * 32);
-                const uint4 a = p[0], b = p[1];
-                float V[8] = {__uint_as_float(a.x), __uint_as_float(a.y), __uint_as_float(a.z),
-                              __uint_as_float(a.w), __uint_as_float(b.x), __uint_as_float(b.y),
-                              __uint_as_float(b.z), __uint_as_float(b.w)};
-                float T[8];
                 if (step < cnt && !rs.failed) {
+                    float U[8];
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
-                        const float delta = -((k & 1) ? acc[r][k >> 1].y : acc[r][k >> 1].x);
-                        const float vn = fmaf(mu, V[k], delta);
-                        const float u = heavy ? vn : fmaf(mu, vn, delta);
-                        const float tn = fmaf(-eta, u, -((k & 1) ? nT[r][k >> 1].y : nT[r][k >> 1].x));
-                        V[k] = vn;
-                        T[k] = tn;
-                        dsq = fmaf(delta, delta, dsq);
-                        tsq = fmaf(tn, tn, tsq);
-                        msq = fmaf(vn, vn, msq);
+                        U[k] = -((k & 1) ? acc[r][k >> 1].y : acc[r][k >> 1].x);
+                        dsq = fmaf(U[k], U[k], dsq);
                     }
-                    const unsigned vi = v0 + step;
-                    store_f32x8<WIDE>(sm.mom, vi, V);
-                    store_f32x8<WIDE>(sm.theta, vi, T);
-                    if (sm.out_bf16 != nullptr)
-                        st_stream16(reinterpret_cast<uint4 *>(sm.out_bf16) + vi,
-                                    make_uint4(pack_bf16x2(T[0], T[1]), pack_bf16x2(T[2], T[3]),
-                                               pack_bf16x2(T[4], T[5]), pack_bf16x2(T[6], T[7])));
+                    store_f32x8<WIDE>(sm.scratch, v0 + step, U);
                 }
             }
-            release();
+        } else {
+            // v and the outer step: v' = mu v + Delta; Theta' = Theta - eta (Delta + mu v')
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const unsigned char *slot = acquire();
+#pragma unroll
+                for (int rr = 0; rr < 2; ++rr) {
+                    const int r = 2 * half + rr;
+                    const unsigned step = (unsigned)(r * 32 + lane);
+                    const uint4 *p = reinterpret_cast<const uint4 *>(slot + (rr * 32 + lane) * 32);
+                    const uint4 a = p[0], b = p[1];
+                    float V[8] = {__uint_as_float(a.x), __uint_as_float(a.y), __uint_as_float(a.z),
+                                  __uint_as_float(a.w), __uint_as_float(b.x), __uint_as_float(b.y),
+                                  __uint_as_float(b.z), __uint_as_float(b.w)};
+                    float T[8];
+                    if (step < cnt && !rs.failed) {
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            const float delta = -((k & 1) ? acc[r][k >> 1].y : acc[r][k >> 1].x);
+                            const float vn = fmaf(mu, V[k], delta);
+                            const float u = heavy ? vn : fmaf(mu, vn, delta);
+                            const float tn = fmaf(-eta, u, -((k & 1) ? nT[r][k >> 1].y : nT[r][k >> 1].x));
+                            V[k] = vn;
+                            T[k] = tn;
+                            dsq = fmaf(delta, delta, dsq);
+                            tsq = fmaf(tn, tn, tsq);
+                            msq = fmaf(vn, vn, msq);
+                        }
+                        const unsigned vi = v0 + step;
+                        store_f32x8<WIDE>(sm.mom, vi, V);
+                        store_f32x8<WIDE>(sm.theta, vi, T);
+                        if (sm.out_bf16 != nullptr)
+                            st_stream16(reinterpret_cast<uint4 *>(sm.out_bf16) + vi,
+                                        make_uint4(pack_bf16x2(T[0], T[1]), pack_bf16x2(T[2], T[3]),
+                                                   pack_bf16x2(T[4], T[5]), pack_bf16x2(T[6], T[7])));
+                    }
+                }
+                release();
+            }
         }
         if (c.records != nullptr) {
             dsq = warp_sum(dsq);
@@ -291,8 +353,11 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
     }
 }
 
-// Kernel body of the staged merge (direct averaging, no per-learner norms).
-template <bool BF16>
+// Kernel body of the staged merge.  MODE is what this launch does with fragments
+// merged radial-directionally (kModeMerge for a plain launch); a fragment of kind
+// DD_MERGE_AVG is skipped by the norms and direction passes and gets the ordinary
+// fused merge in the apply pass, so one batch can mix both kinds.
+template <bool BF16, int MODE, bool PL>
 __device__ __forceinline__ void merge_body_tma(const DevFrag *frags, const Common &c)
 {
     __shared__ Smem sm;
@@ -312,33 +377,49 @@ __device__ __forceinline__ void merge_body_tma(const DevFrag *frags, const Commo
         __syncthreads();
         if (threadIdx.x < 32) {
             cur = find_frag(frags, cur < 0 ? 0 : cur + 1, c.P, tile);
-            load_header<kModeMerge>(frags + cur, cur, tile, c, sm);
+            if (MODE == kModeApply && frags[cur].kind == DD_MERGE_AVG)
+                load_header<kModeMerge>(frags + cur, cur, tile, c, sm);
+            else
+                load_header<MODE>(frags + cur, cur, tile, c, sm);
         }
         __syncthreads();
         cur = sm.frag;
         const unsigned long long tile_end = sm.tile_end;
         const unsigned long long mine = (tile_end - tile + G - 1) / G;      // this CTA's tiles in the fragment
-        if (sm.status == DD_STATUS_OK) {
-            if (!rs.failed) {
-                if (sm.wide) process_fragment_tma<BF16, true>(sm, c, tile, ring_base, bars, rs);
-                else process_fragment_tma<BF16, false>(sm, c, tile, ring_base, bars, rs);
-            }
+        const bool plain = MODE == kModeMerge || (MODE == kModeApply && sm.kind == DD_MERGE_AVG);
+        const bool worked_on = sm.status == DD_STATUS_OK && (plain || sm.kind == DD_MERGE_RDA);
+        if (worked_on) {
             const int rem = (int)(sm.n % kVec);
-            if (rem != 0 && warp == 0 && tile + (mine - 1) * G == tile_end - 1) {
-                float dsq = 0.0f, tsq = 0.0f, msq = 0.0f;
-                process_tail<BF16, false, kModeMerge>(sm, c, (sm.n / kVec) * kVec, rem, dsq, tsq, msq);
-                if (c.records != nullptr) {
-                    dsq = warp_sum(dsq);
-                    tsq = warp_sum(tsq);
-                    msq = warp_sum(msq);
-                    if (lane == 0) {
-                        sm.red[0][0] += (double)dsq;
-                        sm.red[0][1] += (double)tsq;
-                        sm.red[0][2] += (double)msq;
-                    }
+            const bool owns_tail = rem != 0 && warp == 0 && tile + (mine - 1) * G == tile_end - 1;
+            float dsq = 0.0f, tsq = 0.0f, msq = 0.0f;
+            if (plain) {
+                if (!rs.failed) {
+                    if (sm.wide) process_fragment_tma<BF16, true, kModeMerge, PL && MODE == kModeMerge>(sm, c, tile, ring_base, bars, rs);
+                    else process_fragment_tma<BF16, false, kModeMerge, PL && MODE == kModeMerge>(sm, c, tile, ring_base, bars, rs);
+                }
+                if (owns_tail)
+                    process_tail<BF16, PL && MODE == kModeMerge, kModeMerge>(sm, c, (sm.n / kVec) * kVec, rem, dsq, tsq, msq);
+            } else {
+                if (!rs.failed) {
+                    if (sm.wide) process_fragment_tma<BF16, true, MODE, PL>(sm, c, tile, ring_base, bars, rs);
+                    else process_fragment_tma<BF16, false, MODE, PL>(sm, c, tile, ring_base, bars, rs);
+                }
+                if (owns_tail) process_tail<BF16, PL, MODE>(sm, c, (sm.n / kVec) * kVec, rem, dsq, tsq, msq);
+            }
+            if (owns_tail && c.records != nullptr) {
+                dsq = warp_sum(dsq);
+                tsq = warp_sum(tsq);
+                msq = warp_sum(msq);
+                if (lane == 0) {
+                    sm.red[0][0] += (double)dsq;
+                    sm.red[0][1] += (double)tsq;
+                    sm.red[0][2] += (double)msq;
                 }
             }
-            if (c.records != nullptr) flush_fragment<false>(sm, c);
+            if (c.records != nullptr) {
+                if (plain) flush_fragment<PL && MODE == kModeMerge>(sm, c);
+                else flush_fragment<PL>(sm, c);
+            }
         }
         tile += mine * G;
     }
