@@ -443,3 +443,28 @@ def test_bounded_wait_expires_and_context_survives(dd, ctx):
     assert_record_matches(dd.read_records(rec_buf)[0], ref, per_learner=False)
     assert floor_rel_err(t_dev.cpu().numpy(), theta) <= TOL_STATE
     assert floor_rel_err(v_dev.cpu().numpy(), v) <= TOL_STATE
+
+
+def test_hand_worked_example_on_gpu(dd, ctx):
+    # the two-learner merge worked on paper in tests/golden/merge_hand_worked.txt; every
+    # intermediate is exact in binary32, so the GPU must reproduce it bit for bit
+    import os
+    g = {}
+    for line in open(os.path.join(os.path.dirname(__file__), "golden", "merge_hand_worked.txt")):
+        line = line.strip()
+        if line and not line.startswith("#"):
+            key, *vals = line.split()
+            g[key] = [float(x) for x in vals]
+    for flags, key in ((0, "theta_nesterov"), (dd.HEAVY_BALL, "theta_heavy")):
+        t = torch.tensor(g["theta"], dtype=torch.float32, device="cuda")
+        v = torch.tensor(g["momentum"], dtype=torch.float32, device="cuda")
+        L = [torch.tensor(g["learner0"], dtype=torch.float32, device="cuda"),
+             torch.tensor(g["learner1"], dtype=torch.float32, device="cuda")]
+        rec_buf = dd.new_records(1)
+        ctx.merge_fragment(t, v, L, [int(x) for x in g["tokens"]], 0b11, 2, g["eta"][0], g["mu"][0],
+                           flags=flags | dd.DIAG_PER_LEARNER, record=rec_buf)
+        torch.cuda.synchronize()
+        rec = dd.read_records(rec_buf)[0]
+        assert rec.w_hat == g["w_hat"] and rec.delta_sq == g["delta_sq"][0]
+        assert rec.delta_m_sq == g["delta_m_sq"]
+        assert v.cpu().tolist() == g["momentum_new"] and t.cpu().tolist() == g[key]

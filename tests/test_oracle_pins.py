@@ -461,3 +461,41 @@ def test_grace_controller_moving_average_closed_form():
     xi = 2.0 - 0.9 ** 5                         # 1 -> 2 with beta = 0.9 after 5 updates
     assert math.isclose(oracle.grace_controller_window(1.0, 0.5, 0.9, obs), 0.5 * xi, rel_tol=1e-12)
     assert oracle.grace_controller_window(2.0, 0.5, 0.9, []) == 0.0
+
+
+# ---- a merge worked by hand (tests/golden/merge_hand_worked.txt) -------------------------
+
+def _hand_worked():
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "merge_hand_worked.txt")
+    out = {}
+    for line in open(path):
+        line = line.strip()
+        if line and not line.startswith("#"):
+            key, *vals = line.split()
+            out[key] = [float(x) for x in vals]
+    return out
+
+
+def test_hand_worked_merge():
+    g = _hand_worked()
+    tokens = [int(t) for t in g["tokens"]]
+    for nesterov, key in ((True, "theta_nesterov"), (False, "theta_heavy")):
+        theta = np.array(g["theta"], dtype=np.float32)
+        v = np.array(g["momentum"], dtype=np.float32)
+        learners = [np.array(g["learner0"], dtype=np.float32), np.array(g["learner1"], dtype=np.float32)]
+        rec = oracle.merge_fragment(theta, v, learners, tokens, 0b11, 2, g["eta"][0], g["mu"][0],
+                                    nesterov=nesterov)
+        assert rec.w_hat == g["w_hat"]
+        np.testing.assert_array_equal(v, np.array(g["momentum_new"], dtype=np.float32))
+        np.testing.assert_array_equal(theta, np.array(g[key], dtype=np.float32))
+        assert rec.delta_sq == g["delta_sq"][0] and rec.delta_m_sq == g["delta_m_sq"]
+    # radial-directional merge of the same inputs, from the closed form in the fixture's header
+    theta = np.array(g["theta"], dtype=np.float32)
+    v = np.zeros(2, dtype=np.float32)
+    learners = [np.array(g["learner0"], dtype=np.float32), np.array(g["learner1"], dtype=np.float32)]
+    oracle.merge_fragment(theta, v, learners, tokens, 0b11, 2, 1.0, 0.0, merge=oracle.MERGE_RDA)
+    s5 = math.sqrt(5.0)
+    d = np.array([0.25 * 1 + 0.75 * (-1) / s5, 0.75 * 2 / s5])
+    expect = (0.25 + 0.75 * s5) * d / np.linalg.norm(d)
+    np.testing.assert_allclose(v, expect.astype(np.float32), rtol=1e-6)
