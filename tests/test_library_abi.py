@@ -108,3 +108,15 @@ def test_grace_controller_matches_oracle(dd):
         dd.GraceController(2.0, 1.0, 0.5)           # gamma must stay below 1
     with pytest.raises(dd.DDMergeError):
         dd.GraceController(2.0, 0.5, 0.5).observe(-1.0, 0.0, 0.0)
+
+
+def test_header_is_plain_c_and_links(dd, tmp_path):
+    import subprocess
+    pkg = os.path.join(ROOT, "paper_2604_21428_b200")
+    exe = str(tmp_path / "abi_smoke")
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic",
+                           "-I", os.path.join(ROOT, "include"), os.path.join(ROOT, "tests", "abi_smoke.c"),
+                           "-o", exe, "-L", pkg, "-lddmerge", "-lm", f"-Wl,-rpath,{pkg}"])
+    out = subprocess.run([exe], capture_output=True, text=True, timeout=60)
+    assert out.returncode == 0, (out.returncode, out.stderr)
+    assert out.stdout.split() == ["abi", "ok", str(dd.RECORD_BYTES), str(dd.MAX_LEARNERS)]
