@@ -232,10 +232,92 @@ def build_workload(w, device, rank_seed, out_bf16, resident="all"):
     return frags
 
 
+def run_replay(args):
+    """Second workload: the syncer loop itself.  A 1.34B-parameter dense decoder (24 layers,
+    d 2048, d_ff 8192) is cut into P = H = 24 balanced fragments by the library's planner;
+    8 bf16 learners, K = 1, grace window of a quarter step; every syncer step merges the
+    fragment that is due (one launch) and broadcasts it to the learners that are up, driven
+    by a seeded synthetic event tape.  One bench step = one syncer step."""
+    import torch
+
+    from paper_2604_21428_b200 import ddmerge as dd
+    from paper_2604_21428_b200 import synth
+    from paper_2604_21428_b200.replay import Syncer, TapeEntry
+
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    M, P, H, K = 8, 24, 24, 1
+    tensors = synth.dense_tensor_list(24, 2048, 8192, 32000)
+    frag_of, bits = dd.plan_fragments([16 * n for n, _ in tensors], None, P, dd.FRAG_BALANCED)
+    sizes = [b // 16 for b in bits]
+    offsets = list(range(P))
+    total_steps = args.warmup + args.steps
+    tape = synth.synthetic_tape(M, P, H, offsets, total_steps, seed=11)
+    theta = [torch.empty(n, dtype=torch.float32, device=device) for n in sizes]
+    mom = [torch.empty(n, dtype=torch.float32, device=device) for n in sizes]
+    learners = [[None] * P for _ in range(M)]
+    for p, n in enumerate(sizes):
+        copies = [torch.empty(n, dtype=torch.bfloat16, device=device) for _ in range(M)]
+        synth.fill_fragment_gpu(theta[p], mom[p], copies, seed=7000 + p)
+        for m in range(M):
+            learners[m][p] = copies[m]
+    ctx = dd.Context(0)
+    syncer = Syncer(ctx, theta, mom, H=H, offsets=offsets, K=K, outer_lr=synth.OUTER_LR,
+                    outer_mu=synth.OUTER_MU, learner_dtype=dd.BF16, flags=dd.DIAG_STATE)
+    stream = torch.cuda.current_stream()
+    entries = [TapeEntry(arrival_s=e["arrival_s"], tokens=e["tokens"], steps=e["steps"]) for e in tape]
+    for t in range(args.warmup):
+        syncer.step(t, entries[t], learners, grace_s=0.25, stream=stream, read_back=False)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    merged_params = merged_bytes = launches = 0
+    sampler.start()
+    ev0.record(stream)
+    for t in range(args.warmup, total_steps):
+        res = syncer.step(t, entries[t], learners, grace_s=0.25, stream=stream, read_back=False)
+        alive = sum(1 for a in entries[t].arrival_s if a != float("inf"))
+        for p in res.due:
+            s_p = sum(1 for m in range(M) if (res.mask >> m) & 1 and entries[t].tokens[p][m] > 0)
+            if s_p >= max(K, 1):
+                merged_params += sizes[p]
+                merged_bytes += sizes[p] * (2 * s_p + 16) + sizes[p] * (4 + 2 * alive)
+                launches += 2
+            else:
+                launches += 1
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    sampler.stop()
+    ms = ev0.elapsed_time(ev1)
+    peak, peak_kind = hbm_peak()
+    achieved = merged_bytes / (ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": merged_params / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": "tape24", "model_params": sum(sizes), "fragments": P, "H": H, "M": M,
+                   "K": K, "grace_s": 0.25, "fragment_elems_min_max": [min(sizes), max(sizes)],
+                   "planner": "balanced", "learner_dtype": "bf16",
+                   "l2": "inputs larger than L2 (no flush)"},
+        "clocks": sampler.summary(), "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_source": f"of {peak_kind}", "traffic": None,
+                     "algorithmic_bytes": merged_bytes,
+                     "note": "merge + broadcast launches of the syncer loop, host work included"},
+        "e2e": None, "cpu_baseline": None,
+    }
+    print(json.dumps(line), flush=True)
+    ctx.close()
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.workload == "tape24":
+        run_replay(args)
         return
 
     import numpy as np

@@ -53,8 +53,12 @@ class Syncer:
         return [p for p in range(self.P) if t % self.H == self.offsets[p]]
 
     def step(self, t: int, entry: TapeEntry, learner_fragments, grace_s: float = 0.0,
-             stream=None) -> StepResult:
-        """``learner_fragments[m][p]`` is learner m's device copy of fragment p (or None)."""
+             stream=None, read_back: bool = True) -> StepResult:
+        """``learner_fragments[m][p]`` is learner m's device copy of fragment p (or None).
+
+        ``read_back=False`` keeps the step asynchronous: the records stay on the device and
+        the decision to broadcast is taken from what the host already knows (enough
+        admitted learners with a positive token count), which is the kernel's own test."""
         res = StepResult(due=self.due(t))
         if not res.due:
             return res
@@ -76,11 +80,17 @@ class Syncer:
         else:
             self.ctx.merge_fragments_batched(frags, M, self.dtype, self.lr, self.mu,
                                              flags=self.flags, records=recs, stream=stream)
-        res.records = dd.read_records(recs, len(frags))
+        if read_back:
+            res.records = dd.read_records(recs, len(frags))
+            merged = [rec.status == dd.STATUS_OK for rec in res.records]
+        else:
+            need = max(self.K, 1)
+            merged = [sum(1 for m in range(M) if (res.mask >> m) & 1 and entry.tokens[p][m] > 0) >= need
+                      for p in res.due]
         # every learner that is alive receives the new fragment (and resets its counters)
         alive = sum(1 << m for m in range(M) if entry.arrival_s[m] != float("inf"))
-        for p, rec in zip(res.due, res.records):
-            if rec.status == dd.STATUS_OK and alive:
+        for p, ok in zip(res.due, merged):
+            if ok and alive:
                 self.ctx.broadcast_fragment(self.theta[p],
                                             [learner_fragments[m][p] for m in range(M)], alive,
                                             self.alpha, n=int(self.theta[p].numel()),

@@ -217,6 +217,16 @@ def fill_fragment_gpu(theta, momentum, learners, seed: int, chunk: int = 1 << 26
             t[lo:hi].copy_(noise)
 
 
+def dense_tensor_list(layers: int, d: int, d_ff: int, vocab: int):
+    """(element count, transformer layer or -1) for every tensor of a dense decoder, in
+    model order: embedding, per layer q k v o up down and two norm gains, final norm, head."""
+    tensors = [(vocab * d, -1)]
+    for l in range(layers):
+        tensors += [(d * d, l)] * 4 + [(d * d_ff, l)] * 2 + [(d, l)] * 2
+    tensors += [(d, -1), (vocab * d, -1)]
+    return tensors
+
+
 # ---- event tapes ------------------------------------------------------------------
 
 def synthetic_tape(M: int, P: int, H: int, offsets, steps_total: int, seed: int, *,
