@@ -123,7 +123,8 @@ int dd_destroy(dd_ctx *ctx);
  *   global, momentum  [device] float32[n], in/out
  *   learner_ptrs      [host]   M device pointers to learner_dtype[n]
  *   tokens, steps     [host]   uint64[M]; steps may be NULL; tokens[m] > 0 with
- *                              steps[m] == 0 is DD_ERR_INVALID_ARG
+ *                              steps[m] == 0, or participants' tokens summing past
+ *                              2^64 - 1, is DD_ERR_INVALID_ARG
  *   quorum_mask       bit m = learner m reported in time (bits >= M ignored)
  *   K                 minimum quorum, 0 <= K <= M (0 acts as 1)
  *   out_bf16          [device] optional bf16[n]: round-to-nearest-even copy of

@@ -146,7 +146,7 @@ def weights(tokens, steps, idx):
     st = lib.ddo_weights(_u64(tokens), None if steps is None else _u64(steps), idx_c, s, w_hat,
                          ctypes.byref(W))
     if st == INVALID:
-        raise ValueError("oracle: tokens > 0 with steps == 0")
+        raise ValueError("oracle: tokens > 0 with steps == 0, or token sum beyond 64 bits")
     return st, [float(w_hat[j]) for j in range(s)], float(W.value)
 
 

@@ -128,7 +128,11 @@ int ddo_weights(const uint64_t *tokens, const uint64_t *steps, const uint8_t *id
     int j;
     if (steps == NULL) {
         uint64_t Wi = 0;
-        for (j = 0; j < s; ++j) { w[j] = (double)tokens[idx[j]]; Wi += tokens[idx[j]]; }
+        for (j = 0; j < s; ++j) {
+            w[j] = (double)tokens[idx[j]];
+            if (Wi + tokens[idx[j]] < Wi) return DDO_INVALID;   /* the exact 64-bit sum would wrap */
+            Wi += tokens[idx[j]];
+        }
         W = (double)Wi;
     } else {
         for (j = 0; j < s; ++j) {

@@ -103,12 +103,15 @@ static int fill_fragment(DevFrag &d, float *global, float *momentum, void *out_b
     d.mask = M >= 64 ? mask : (mask & ((1ull << M) - 1ull));
     d.K = K;
     d.has_steps = steps != nullptr;
+    uint64_t token_sum = 0;
     for (int m = 0; m < M; ++m) {
         d.tokens[m] = tokens[m];
         d.steps[m] = steps ? steps[m] : 0;
         d.ptrs[m] = learner_ptrs[m];
         if (steps && tokens[m] > 0 && steps[m] == 0) return DD_ERR_INVALID_ARG;
         const bool takes_part = ((d.mask >> m) & 1ull) && tokens[m] > 0;
+        // the kernel sums the participants' token counts exactly, in 64 bits
+        if (takes_part && __builtin_add_overflow(token_sum, tokens[m], &token_sum)) return DD_ERR_INVALID_ARG;
         if (takes_part && n > 0) {
             const void *p = learner_ptrs[m];
             if (!p) return DD_ERR_INVALID_ARG;

@@ -122,11 +122,15 @@ static int fill(DevFrag &d, const dd_fragment_desc &f, int M, dd_dtype dtype)
     d.mask = M >= 64 ? f.quorum_mask : (f.quorum_mask & ((1ull << M) - 1ull));
     d.K = f.K;
     d.has_steps = f.steps != nullptr;
+    uint64_t token_sum = 0;
     for (int m = 0; m < M; ++m) {
         d.tokens[m] = f.tokens[m];
         d.steps[m] = f.steps ? f.steps[m] : 0;
         d.ptrs[m] = f.learner_ptrs[m];
         if (f.steps && f.tokens[m] > 0 && f.steps[m] == 0) return DD_ERR_INVALID_ARG;
+        if (((d.mask >> m) & 1ull) && f.tokens[m] > 0 &&
+            __builtin_add_overflow(token_sum, f.tokens[m], &token_sum))
+            return DD_ERR_INVALID_ARG;
         if (((d.mask >> m) & 1ull) && f.tokens[m] > 0 && n > 0) {
             const void *p = f.learner_ptrs[m];
             if (!p) return DD_ERR_INVALID_ARG;

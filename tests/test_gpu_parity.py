@@ -187,6 +187,12 @@ def test_quorum_not_met_and_zero_tokens(dd, ctx):
     assert rec.status == dd.STATUS_QUORUM_NOT_MET and rec.n_part == 0
 
 
+def test_huge_token_counts(dd, ctx):
+    run_case(dd, ctx, 9_000, 3, "bf16", [2**62, 2**61, 2**61 + 12345], 0b111, 3, seed=44, merges=1)
+    run_case(dd, ctx, 9_000, 3, "bf16", [2**40, 2**45, 2**50 + 1], 0b111, 3, seed=45, merges=1,
+             steps=[3, 2**20, 7])
+
+
 def test_steps_weighting(dd, ctx):
     tokens = [40960, 8192, 123456, 99999, 5]
     steps = [10, 1, 33, 7, 5]
@@ -342,6 +348,7 @@ def test_argument_validation(dd, ctx):
     assert rc_of(lambda: ctx.merge_fragment(t, v, [L[0], None, L[2]], [1, 1, 1], 7, 1, ETA, MU, **good)) == dd.ERR_INVALID_ARG
     assert rc_of(lambda: ctx.merge_fragment(t, v, L, [1, 1, 1], 7, 1, ETA, MU, steps=[1, 0, 1], **good)) == dd.ERR_INVALID_ARG
     assert rc_of(lambda: ctx.merge_fragment(t, v, L, [1, 1, 1], 7, 1, ETA, MU, flags=1 << 9, **good)) == dd.ERR_INVALID_ARG
+    assert rc_of(lambda: ctx.merge_fragment(t, v, L, [2**63, 2**63, 1], 7, 1, ETA, MU, **good)) == dd.ERR_INVALID_ARG
     assert rc_of(lambda: ctx.merge_fragment(t.data_ptr() + 4, v, L, [1, 1, 1], 7, 1, ETA, MU, n=n - 8, learner_dtype=dd.BF16)) == dd.ERR_ALIGNMENT
     assert rc_of(lambda: ctx.merge_fragment(t, v, [L[0], L[1].data_ptr() + 2, L[2]], [1, 1, 1], 7, 1, ETA, MU, n=n - 8, learner_dtype=dd.BF16)) == dd.ERR_ALIGNMENT
     assert rc_of(lambda: ctx.merge_fragment(t, t, L, [1, 1, 1], 7, 1, ETA, MU, **good)) == dd.ERR_ALIAS

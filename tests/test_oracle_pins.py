@@ -499,3 +499,13 @@ def test_hand_worked_merge():
     d = np.array([0.25 * 1 + 0.75 * (-1) / s5, 0.75 * 2 / s5])
     expect = (0.25 + 0.75 * s5) * d / np.linalg.norm(d)
     np.testing.assert_allclose(v, expect.astype(np.float32), rtol=1e-6)
+
+
+def test_huge_token_counts():
+    # counts far beyond 2^53: the integer sum stays exact, the weights stay normalised
+    big = [2**62, 2**61, 2**61 + 12345]
+    st, w_hat, W = oracle.weights(big, None, [0, 1, 2])
+    assert st == 0 and W == float(sum(big))
+    np.testing.assert_allclose(w_hat, [b / sum(big) for b in big], rtol=1e-15)
+    with pytest.raises(ValueError):
+        oracle.weights([2**63, 2**63], None, [0, 1])        # the exact sum would wrap
