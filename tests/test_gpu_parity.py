@@ -475,3 +475,30 @@ def test_hand_worked_example_on_gpu(dd, ctx):
         assert rec.w_hat == g["w_hat"] and rec.delta_sq == g["delta_sq"][0]
         assert rec.delta_m_sq == g["delta_m_sq"]
         assert v.cpu().tolist() == g["momentum_new"] and t.cpu().tolist() == g[key]
+
+
+def test_participation_and_weights_random_sweep(dd, ctx):
+    # 300 random (M, mask, tokens, steps, K): participant set, order, status bit-exact;
+    # weights bit-exact as float32 without steps, to 1 ulp-ish with steps (fp64 sum order is fixed)
+    rng = np.random.default_rng(2024)
+    n = 64
+    theta = torch.zeros(n, device="cuda")
+    mom = torch.zeros(n, device="cuda")
+    pool = [torch.full((n,), 0.01 * (m + 1), device="cuda", dtype=torch.bfloat16) for m in range(64)]
+    rec_buf = dd.new_records(1)
+    for trial in range(300):
+        M = int(rng.integers(1, 65))
+        tokens = [int(t) for t in rng.integers(0, 4, size=M) * rng.integers(1, 10**6, size=M)]
+        mask = int(rng.integers(0, 1 << 62)) | (int(rng.integers(0, 4)) << 62)
+        K = int(rng.integers(0, M + 1))
+        steps = None if trial % 2 else [int(x) for x in rng.integers(1, 1000, size=M)]
+        st, idx = oracle.participants(mask, tokens, K)
+        ctx.merge_fragment(theta, mom, pool[:M], tokens, mask, K, ETA, MU, n=n, learner_dtype=dd.BF16,
+                           steps=steps, record=rec_buf)
+        torch.cuda.synchronize()
+        rec = dd.read_records(rec_buf)[0]
+        assert (rec.status, rec.idx) == (st, idx), (trial, M, K)
+        if st == 0:
+            _, w_hat, W = oracle.weights(tokens, steps, idx)
+            assert rec.w_hat == [float(np.float32(w)) for w in w_hat], trial
+            assert abs(rec.w_total - W) <= 1e-15 * W
