@@ -101,7 +101,7 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
     unsigned char *const ring = ring_base + (size_t)warp * kTmaStages * kTmaChunk;
     unsigned long long *const bar = bars + warp * kTmaStages;
     const unsigned nfull = (unsigned)(sm.n / kVec);
-    const unsigned long long tile_end = sm.tile_end, tile_begin = sm.tile_begin;
+    const unsigned long long tile_begin = sm.tile_begin;
     const int s = sm.n_part;
     constexpr bool kHasV = MODE == kModeMerge || MODE == kModeApply;
     constexpr bool kNorms = PL || MODE == kModeNorms;
@@ -110,45 +110,41 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
     const float *const theta = sm.theta;
     const float *const mom = sm.mom;
 
-    // first step (of 8 elements) of the super-row warp `warp` has in tile t
-    auto first_step = [&](unsigned long long t) {
-        return ((unsigned)(t - tile_begin) * kWarps + (unsigned)warp) * (unsigned)(kSuperRow / kVec);
-    };
+    // This warp's super-rows in the fragment start at step v_first and are row_stride steps apart.
+    constexpr unsigned kRowSteps = kSuperRow / kVec;
+    const unsigned row_stride = G * (unsigned)(kTileElems / kVec);
+    const unsigned v_first = ((unsigned)(tile - tile_begin) * kWarps + (unsigned)warp) * kRowSteps;
 
     // ---- producer (lane 0): one piece per call ---------------------------------------
-    unsigned long long itile = tile;
+    unsigned iv0 = v_first;                    // first step of the super-row being requested
     int ipiece = 0;
     int outstanding = 0;
     auto issue = [&]() {
-        if (rs.failed || itile >= tile_end) return;
-        const unsigned v0 = first_step(itile);
-        if (v0 >= nfull) { itile = tile_end; return; }
+        if (rs.failed || iv0 >= nfull) return;
         if (lane == 0) {
-            const unsigned cnt = min(128u, nfull - v0);            // steps in this super-row
-            const void *src;
+            const unsigned cnt = min(kRowSteps, nfull - iv0);      // steps in this super-row
+            const char *src;
             unsigned bytes;
-            if (ipiece < 2 || ipiece >= 2 + nmid || MODE == kModeApply) {
-                // float32 operand (Theta, stored direction, v): halves of 64 steps x 32 B
-                const float *base = ipiece < 2 ? theta : (ipiece < 2 + nmid ? sm.scratch : mom);
-                const int half = ipiece < 2 ? ipiece : (ipiece < 2 + nmid ? ipiece - 2 : ipiece - 2 - nmid);
-                const unsigned nv = cnt > 64u * half ? min(64u, cnt - 64u * half) : 0u;
-                src = base + 8ull * (v0 + 64u * half);
-                bytes = nv * 32u;
-            } else if (BF16) {
-                src = reinterpret_cast<const char *>(sm.ptr[ipiece - 2]) + 16ull * v0;
+            if (BF16 && MODE != kModeApply && ipiece >= 2 && ipiece < 2 + nmid) {
+                src = reinterpret_cast<const char *>(sm.ptr[ipiece - 2]) + 16ull * iv0;
                 bytes = cnt * 16u;
             } else {
-                const int j = (ipiece - 2) >> 1, half = (ipiece - 2) & 1;
-                const unsigned nv = cnt > 64u * half ? min(64u, cnt - 64u * half) : 0u;
-                src = reinterpret_cast<const char *>(sm.ptr[j]) + 32ull * (v0 + 64u * half);
+                // float32 operand (Theta, fp32 learner copy, stored direction, v): two halves of 64 steps
+                const int q = ipiece < 2 ? ipiece : (ipiece < 2 + nmid ? ipiece - 2 : ipiece - 2 - nmid);
+                const void *base = ipiece < 2 ? (const void *)theta
+                                 : ipiece >= 2 + nmid ? (const void *)mom
+                                 : MODE == kModeApply ? (const void *)sm.scratch : sm.ptr[q >> 1];
+                const unsigned first = 64u * (unsigned)(q & 1);
+                const unsigned nv = cnt > first ? min(64u, cnt - first) : 0u;
+                src = reinterpret_cast<const char *>(base) + 32ull * (iv0 + first);
                 bytes = nv * 32u;
             }
             // (test hook) announce 16 bytes that no copy will deliver: the wait must expire
-            const unsigned phantom = (c.flags & DD_DEBUG_EXPIRE_WAIT) && itile == tile && ipiece == 0 ? 16u : 0u;
+            const unsigned phantom = (c.flags & DD_DEBUG_EXPIRE_WAIT) && iv0 == v_first && ipiece == 0 ? 16u : 0u;
             mbar_arrive_expect_tx(bar + rs.islot, bytes + phantom);
             if (bytes != 0) bulk_copy_g2s(ring + rs.islot * kTmaChunk, src, bytes, bar + rs.islot);
         }
-        if (++ipiece == npieces) { ipiece = 0; itile += G; }
+        if (++ipiece == npieces) { ipiece = 0; iv0 += row_stride; }
         if (++rs.islot == kTmaStages) rs.islot = 0;
         ++outstanding;
     };
@@ -174,10 +170,8 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
     const float eta = c.eta, mu = c.mu;
     const bool heavy = (c.flags & DD_HEAVY_BALL) != 0;
 #pragma unroll 1
-    for (unsigned long long ctile = tile; ctile < tile_end && !rs.failed; ctile += G) {
-        const unsigned v0 = first_step(ctile);
-        if (v0 >= nfull) break;
-        const unsigned cnt = min(128u, nfull - v0);
+    for (unsigned v0 = v_first; v0 < nfull && !rs.failed; v0 += row_stride) {
+        const unsigned cnt = min(kRowSteps, nfull - v0);
         float2 nT[4][4], acc[4][4];
         // Theta: two pieces of 64 steps; lane owns steps r*32 + lane, r = 0..3
 #pragma unroll
