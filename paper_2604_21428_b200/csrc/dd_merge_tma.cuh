@@ -42,24 +42,25 @@ __device__ __forceinline__ void mbar_init(unsigned long long *bar, unsigned coun
 }
 
 // The issuing thread's arrival plus the number of bytes the copies will deliver.
-__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long *bar, unsigned bytes)
+// (These take 32-bit shared-space addresses so that the per-piece code does no
+// generic-to-shared conversions.)
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned bar, unsigned bytes)
 {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
-                 :: "r"(smem_addr(bar)), "r"(bytes) : "memory");
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
 }
 
-__device__ __forceinline__ bool mbar_try_wait(unsigned long long *bar, unsigned parity)
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity)
 {
     unsigned ok;
     // The attempt suspends the thread until the phase completes or the hint expires.
     asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
                  " selp.u32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity), "r"(kWaitHintNs) : "memory");
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(kWaitHintNs) : "memory");
     return ok != 0;
 }
 
 // Bounded wait for one phase of a slot's barrier.
-__device__ __forceinline__ bool mbar_wait_bounded(unsigned long long *bar, unsigned parity)
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity)
 {
     for (int spins = 0; spins < kWaitLimit; ++spins)
         if (mbar_try_wait(bar, parity)) return true;
@@ -67,11 +68,10 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned long long *bar, unsig
 }
 
 // global -> this CTA's shared memory, 16-byte aligned on both sides, bytes % 16 == 0.
-__device__ __forceinline__ void bulk_copy_g2s(void *dst, const void *src, unsigned bytes,
-                                              unsigned long long *bar)
+__device__ __forceinline__ void bulk_copy_g2s(unsigned dst, const void *src, unsigned bytes, unsigned bar)
 {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 :: "r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+                 :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
 // Ring position of a warp; survives from one fragment to the next (the ring is
@@ -99,7 +99,9 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const unsigned G = gridDim.x;
     unsigned char *const ring = ring_base + (size_t)warp * kTmaStages * kTmaChunk;
-    unsigned long long *const bar = bars + warp * kTmaStages;
+    const unsigned ring_s = smem_addr(ring);                      // the same, as shared-space addresses
+    const unsigned bar_s = smem_addr(bars + warp * kTmaStages);
+    const bool expire_hook = (c.flags & DD_DEBUG_EXPIRE_WAIT) != 0;
     const unsigned nfull = (unsigned)(sm.n / kVec);
     const unsigned long long tile_begin = sm.tile_begin;
     const int s = sm.n_part;
@@ -140,9 +142,9 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
                 bytes = nv * 32u;
             }
             // (test hook) announce 16 bytes that no copy will deliver: the wait must expire
-            const unsigned phantom = (c.flags & DD_DEBUG_EXPIRE_WAIT) && iv0 == v_first && ipiece == 0 ? 16u : 0u;
-            mbar_arrive_expect_tx(bar + rs.islot, bytes + phantom);
-            if (bytes != 0) bulk_copy_g2s(ring + rs.islot * kTmaChunk, src, bytes, bar + rs.islot);
+            const unsigned phantom = expire_hook && iv0 == v_first && ipiece == 0 ? 16u : 0u;
+            mbar_arrive_expect_tx(bar_s + 8u * rs.islot, bytes + phantom);
+            if (bytes != 0) bulk_copy_g2s(ring_s + kTmaChunk * rs.islot, src, bytes, bar_s + 8u * rs.islot);
         }
         if (++ipiece == npieces) { ipiece = 0; iv0 += row_stride; }
         if (++rs.islot == kTmaStages) rs.islot = 0;
@@ -153,7 +155,7 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
         __syncwarp();                                              // the slot consumed last is free again
         if (!rs.failed) {
             issue();
-            const bool ok = mbar_wait_bounded(bar + rs.cslot, rs.cphase);
+            const bool ok = mbar_wait_bounded(bar_s + 8u * rs.cslot, rs.cphase);
             if (!__all_sync(0xffffffffu, ok)) rs.failed = true;    // the whole warp gives up together
         }
         return ring + rs.cslot * kTmaChunk;
@@ -339,7 +341,7 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
         // Give the copies still in flight a bounded chance to land before this
         // warp's slots can be reused or the CTA exits, and say what happened.
         for (int k = 0; k < outstanding; ++k) {
-            (void)mbar_wait_bounded(bar + rs.cslot, rs.cphase);
+            (void)mbar_wait_bounded(bar_s + 8u * rs.cslot, rs.cphase);
             if (++rs.cslot == kTmaStages) { rs.cslot = 0; rs.cphase ^= 1u; }
         }
         rs.islot = rs.cslot;
