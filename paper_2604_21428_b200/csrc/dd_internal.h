@@ -11,8 +11,8 @@ namespace ddm {
 constexpr int kThreads = 256;            // threads per CTA
 constexpr int kWarps = kThreads / 32;
 constexpr int kVec = 8;                  // elements one thread handles per step
-constexpr int kUnroll = 4;               // steps per tile
-constexpr int kTileElems = kThreads * kVec * kUnroll;   // 8192 elements per tile
+constexpr int kStepsPerLane = 4;         // 8-element steps a lane handles per warp round
+constexpr int kTileElems = kThreads * kVec * kStepsPerLane;   // 8192 elements per tile: 1024 per warp
 constexpr int kNumScalarDiag = 3;        // delta_sq, theta_sq, mom_sq
 constexpr unsigned long long kMaxFragmentElems = 1ull << 34;   // 8-element steps are indexed in 32 bits
 

@@ -1,21 +1,16 @@
-// Fused per-fragment merge kernel (sm_100a): participation -> weights -> outer
-// gradients -> weighted reduce -> outer optimizer step -> norm diagnostics, one
-// pass over HBM.  Algorithm 2 steps 2-3 with the Weight function of Section 3.2
-// and the weighted direct-averaging merge of the "Merging methods" appendix.
+// Building blocks of the fused per-fragment merge kernel (sm_100a): participation
+// -> weights -> outer gradients -> weighted reduce -> outer optimizer step -> norm
+// diagnostics, one pass over HBM.  Algorithm 2 steps 2-3 with the Weight function
+// of Section 3.2 and the weighted direct-averaging merge of the "Merging methods"
+// appendix.  This file holds the per-fragment header (participation and weights),
+// the ragged-tail code and the reduction of the diagnostics; the streaming part
+// is in dd_merge_tma.cuh.
 #pragma once
 
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
 #include "dd_internal.h"
-
-// Learner loads a thread issues back to back before it consumes them.
-#ifndef DD_BATCH_BF16
-#define DD_BATCH_BF16 8
-#endif
-#ifndef DD_BATCH_F32
-#define DD_BATCH_F32 4
-#endif
 
 namespace ddm {
 
@@ -242,134 +237,6 @@ __device__ __forceinline__ int find_frag(const DevFrag *frags, int lo, int P,
     return lo;
 }
 
-// ---- steps 3-5 for 8 consecutive elements --------------------------------------
-//
-// acc = sum_j w_hat_j (theta_j - Theta) = -Delta.  The difference is formed FIRST
-// (exact or nearly so when theta_j is close to Theta), then weighted: factoring
-// Theta out of the sum would lose ~|Theta|/|Delta| ulps.  `active` is false only
-// with per-learner diagnostics, where idle lanes still take part in the shuffles.
-template <bool BF16, bool PL, bool WIDE, int MODE>
-__device__ __forceinline__ void process_vec(Smem &sm, const Common &c, unsigned vi, bool active,
-                                            float &dsq, float &tsq, float &msq)
-{
-    constexpr int B = BF16 ? DD_BATCH_BF16 : DD_BATCH_F32;
-    const int s = sm.n_part;
-    float T[8], V[8];
-    float2 nT[4], acc[4];
-    if (!PL || active) {
-        load_f32x8<WIDE>(sm.theta, vi, T);
-    } else {
-#pragma unroll
-        for (int k = 0; k < 8; ++k) { T[k] = 0.0f; V[k] = 0.0f; }
-    }
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        nT[k] = make_float2(-T[2 * k], -T[2 * k + 1]);
-        acc[k] = make_float2(0.0f, 0.0f);
-    }
-
-    if (MODE != kModeApply) {
-#pragma unroll 1
-        for (int j0 = 0; j0 < s; j0 += B) {
-            uint4 r[BF16 ? B : 2 * B];
-#pragma unroll
-            for (int b = 0; b < B; ++b) {
-                if (j0 + b < s) {
-                    if (PL && !active) {
-                        if (BF16) r[b] = make_uint4(0u, 0u, 0u, 0u);
-                        else r[2 * b] = r[2 * b + 1] = make_uint4(0u, 0u, 0u, 0u);
-                    } else if (BF16) {
-                        r[b] = ld_stream16(reinterpret_cast<const uint4 *>(sm.ptr[j0 + b]) + vi);
-                    } else {
-                        const uint4 *p = reinterpret_cast<const uint4 *>(sm.ptr[j0 + b]) + 2ull * vi;
-                        r[2 * b] = ld_stream16(p);
-                        r[2 * b + 1] = ld_stream16(p + 1);
-                    }
-                }
-            }
-            // The momentum is needed only by the epilogue: fetch it behind the last batch.
-            if (MODE == kModeMerge && j0 + B >= s && (!PL || active)) load_f32x8<WIDE>(sm.mom, vi, V);
-#pragma unroll
-            for (int b = 0; b < B; ++b) {
-                if (j0 + b < s) {
-                    const float w = sm.w[j0 + b];
-                    const float2 w2 = make_float2(w, w);
-                    float2 x[4];
-                    if (BF16) {
-                        // element 2k sits in the low half of word k, element 2k+1 in the high half
-                        const unsigned word[4] = {r[b].x, r[b].y, r[b].z, r[b].w};
-#pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            x[k] = make_float2(__uint_as_float(word[k] << 16),
-                                               __uint_as_float(word[k] & 0xffff0000u));
-                    } else {
-                        x[0] = make_float2(__uint_as_float(r[2 * b].x), __uint_as_float(r[2 * b].y));
-                        x[1] = make_float2(__uint_as_float(r[2 * b].z), __uint_as_float(r[2 * b].w));
-                        x[2] = make_float2(__uint_as_float(r[2 * b + 1].x), __uint_as_float(r[2 * b + 1].y));
-                        x[3] = make_float2(__uint_as_float(r[2 * b + 1].z), __uint_as_float(r[2 * b + 1].w));
-                    }
-                    float q = 0.0f;
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const float2 d = __fadd2_rn(x[k], nT[k]);
-                        if (MODE != kModeNorms) acc[k] = __ffma2_rn(w2, d, acc[k]);
-                        if (PL) q = fmaf(d.x, d.x, fmaf(d.y, d.y, q));
-                    }
-                    if (PL) {
-                        q = warp_sum(q);
-                        if ((threadIdx.x & 31) == 0) sm.dm[threadIdx.x >> 5][j0 + b] += (double)q;
-                    }
-                }
-            }
-        }
-    }
-    if (PL && !active) return;
-    if (MODE == kModeNorms) return;
-
-    if (MODE == kModeDir) {
-        // the mean direction u = sum_j a_j (Theta - theta_j), kept for the apply pass
-        float U[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            U[k] = -((k & 1) ? acc[k >> 1].y : acc[k >> 1].x);
-            dsq = fmaf(U[k], U[k], dsq);
-        }
-        store_f32x8<WIDE>(sm.scratch, vi, U);
-        return;
-    }
-    if (MODE == kModeApply) {
-        float U[8];
-        load_f32x8<WIDE>(sm.scratch, vi, U);
-        load_f32x8<WIDE>(sm.mom, vi, V);
-        const float cs = sm.cscale;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) acc[k] = make_float2(-cs * U[2 * k], -cs * U[2 * k + 1]);
-    }
-
-    // Outer step: v' = mu v + Delta; Theta' = Theta - eta (Delta + mu v') (Nesterov)
-    // or Theta - eta v' (heavy ball).
-    const float eta = c.eta, mu = c.mu;
-    const bool heavy = (c.flags & DD_HEAVY_BALL) != 0;
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-        const float delta = -((k & 1) ? acc[k >> 1].y : acc[k >> 1].x);
-        const float vn = fmaf(mu, V[k], delta);
-        const float u = heavy ? vn : fmaf(mu, vn, delta);
-        const float tn = fmaf(-eta, u, -((k & 1) ? nT[k >> 1].y : nT[k >> 1].x));
-        V[k] = vn;
-        T[k] = tn;
-        dsq = fmaf(delta, delta, dsq);
-        tsq = fmaf(tn, tn, tsq);
-        msq = fmaf(vn, vn, msq);
-    }
-    store_f32x8<WIDE>(sm.mom, vi, V);
-    store_f32x8<WIDE>(sm.theta, vi, T);
-    if (sm.out_bf16 != nullptr)
-        st_stream16(reinterpret_cast<uint4 *>(sm.out_bf16) + vi,
-                    make_uint4(pack_bf16x2(T[0], T[1]), pack_bf16x2(T[2], T[3]),
-                               pack_bf16x2(T[4], T[5]), pack_bf16x2(T[6], T[7])));
-}
-
 // The ragged end of a fragment (n mod 8 elements), one element per lane of warp 0.
 template <bool BF16, bool PL, int MODE>
 __device__ __forceinline__ void process_tail(Smem &sm, const Common &c, unsigned long long first,
@@ -471,89 +338,6 @@ __device__ __forceinline__ void flush_fragment(Smem &sm, const Common &c)
         }
     }
     if (threadIdx.x == 0) c.tickets[p] = 0u;
-}
-
-// One tile (kTileElems elements of the current fragment).
-template <bool BF16, bool PL, bool WIDE, int MODE>
-__device__ __forceinline__ void process_tile(Smem &sm, const Common &c, unsigned long long tile)
-{
-    constexpr unsigned kTileSteps = kTileElems / kVec;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const unsigned nfull = (unsigned)(sm.n / kVec);                       // whole 8-element steps
-    const unsigned base = (unsigned)(tile - sm.tile_begin) * kTileSteps;
-    const unsigned end = min(base + kTileSteps, nfull);
-    float dsq = 0.0f, tsq = 0.0f, msq = 0.0f;
-    if (PL) {
-        // per-learner norms are warp-wide sums: the whole warp walks together
-        for (unsigned v0 = base + warp * 32; v0 < end; v0 += kThreads)
-            process_vec<BF16, true, WIDE, MODE>(sm, c, v0 + lane, v0 + lane < end, dsq, tsq, msq);
-    } else {
-        for (unsigned vi = base + threadIdx.x; vi < end; vi += kThreads)
-            process_vec<BF16, false, WIDE, MODE>(sm, c, vi, true, dsq, tsq, msq);
-    }
-    const int rem = (int)(sm.n % kVec);
-    if (rem != 0 && tile == sm.tile_end - 1 && warp == 0)
-        process_tail<BF16, PL, MODE>(sm, c, (unsigned long long)nfull * kVec, rem, dsq, tsq, msq);
-    if (c.records != nullptr && MODE != kModeNorms) {
-        // fp32 within a tile (at most 32 elements per thread), fp64 from here on
-        dsq = warp_sum(dsq);
-        tsq = warp_sum(tsq);
-        msq = warp_sum(msq);
-        if (lane == 0) {
-            sm.red[warp][0] += (double)dsq;
-            sm.red[warp][1] += (double)tsq;
-            sm.red[warp][2] += (double)msq;
-        }
-    }
-}
-
-// ---- the kernel body ----------------------------------------------------------
-//
-// MODE is what this launch does with fragments merged radial-directionally; a
-// fragment of kind DD_MERGE_AVG is skipped by the norms and direction passes and
-// gets the ordinary fused merge in the apply pass, so one batch can mix both.
-template <bool BF16, bool PL, int MODE>
-__device__ __forceinline__ void merge_body(const DevFrag *frags, const Common &c)
-{
-    __shared__ Smem sm;
-    const unsigned G = gridDim.x;
-    int cur = -1;
-    bool loaded = false;
-    auto worked_on = [&]() {
-        return sm.status == DD_STATUS_OK && (MODE == kModeMerge || MODE == kModeApply || sm.kind == DD_MERGE_RDA);
-    };
-
-    for (unsigned long long tile = blockIdx.x; tile < c.total_tiles; tile += G) {
-        if (!loaded || tile >= sm.tile_end) {                     // CTA-uniform
-            if (loaded && c.records != nullptr && worked_on()) {
-                if (MODE == kModeApply && sm.kind == DD_MERGE_AVG) flush_fragment<false>(sm, c);
-                else flush_fragment<PL>(sm, c);
-            }
-            __syncthreads();
-            if (threadIdx.x < 32) {
-                cur = find_frag(frags, cur < 0 ? 0 : cur + 1, c.P, tile);
-                if (MODE == kModeApply && frags[cur].kind == DD_MERGE_AVG)
-                    load_header<kModeMerge>(frags + cur, cur, tile, c, sm);
-                else
-                    load_header<MODE>(frags + cur, cur, tile, c, sm);
-            }
-            __syncthreads();
-            cur = sm.frag;
-            loaded = true;
-        }
-        if (!worked_on()) continue;
-        if (MODE == kModeApply && sm.kind == DD_MERGE_AVG) {
-            if (sm.wide) process_tile<BF16, false, true, kModeMerge>(sm, c, tile);
-            else process_tile<BF16, false, false, kModeMerge>(sm, c, tile);
-        } else {
-            if (sm.wide) process_tile<BF16, PL, true, MODE>(sm, c, tile);
-            else process_tile<BF16, PL, false, MODE>(sm, c, tile);
-        }
-    }
-    if (loaded && c.records != nullptr && worked_on()) {
-        if (MODE == kModeApply && sm.kind == DD_MERGE_AVG) flush_fragment<false>(sm, c);
-        else flush_fragment<PL>(sm, c);
-    }
 }
 
 }  // namespace ddm

@@ -14,7 +14,7 @@
 
 #include <cuda_runtime.h>
 
-#include "dd_merge_kernel.cuh"
+#include "dd_merge_tma.cuh"
 
 namespace ddm {
 namespace noalloc {
@@ -40,13 +40,13 @@ static __device__ __align__(256) unsigned char g_scratch[DD_NOALLOC_SCRATCH_BYTE
 __global__ void __launch_bounds__(kThreads, 2)
 merge_batched_noalloc_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ Common c)
 {
-    merge_body<true, false, kModeMerge>(frags, c);
+    merge_body_tma<true, kModeMerge, false>(frags, c);
 }
 
 __global__ void __launch_bounds__(kThreads, 2)
 merge_batched_noalloc_kernel_f32(const DevFrag *__restrict__ frags, const __grid_constant__ Common c)
 {
-    merge_body<false, false, kModeMerge>(frags, c);
+    merge_body_tma<false, kModeMerge, false>(frags, c);
 }
 
 struct DeviceState {
@@ -77,13 +77,21 @@ static int setup_current_device(DeviceState **out)
         }
         int sms = 0, occ_bf16 = 0, occ_f32 = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            // the warps' staging rings live in dynamic shared memory: opt in (this sets a
+            // function attribute; it allocates nothing)
+            cudaFuncSetAttribute(merge_batched_noalloc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kTmaRingBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(merge_batched_noalloc_kernel_f32, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kTmaRingBytes) != cudaSuccess ||
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_bf16, merge_batched_noalloc_kernel,
-                                                          kThreads, 0) != cudaSuccess ||
+                                                          kThreads, kTmaRingBytes) != cudaSuccess ||
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_f32, merge_batched_noalloc_kernel_f32,
-                                                          kThreads, 0) != cudaSuccess) {
+                                                          kThreads, kTmaRingBytes) != cudaSuccess) {
             (void)cudaGetLastError();
             return DD_ERR_CUDA;
         }
+        if (occ_bf16 > 2) occ_bf16 = 2;              // same launch shape as the ordinary entry points
+        if (occ_f32 > 2) occ_f32 = 2;
         const int g1 = sms * (occ_bf16 > 0 ? occ_bf16 : 1), g0 = sms * (occ_f32 > 0 ? occ_f32 : 1);
         st.grid[1] = g1 < kMaxCtas ? g1 : kMaxCtas;
         st.grid[0] = g0 < kMaxCtas ? g0 : kMaxCtas;
@@ -206,9 +214,9 @@ extern "C" int dd_merge_fragments_batched_noalloc(const dd_fragment_desc *descs,
         return DD_ERR_CUDA;
     }
     if (bf16)
-        merge_batched_noalloc_kernel<<<(unsigned)g, kThreads, 0, stream>>>(dev_frags, c);
+        merge_batched_noalloc_kernel<<<(unsigned)g, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
     else
-        merge_batched_noalloc_kernel_f32<<<(unsigned)g, kThreads, 0, stream>>>(dev_frags, c);
+        merge_batched_noalloc_kernel_f32<<<(unsigned)g, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
     if (cudaGetLastError() != cudaSuccess) return DD_ERR_CUDA;
     return DD_OK;
 }

@@ -502,3 +502,34 @@ def test_participation_and_weights_random_sweep(dd, ctx):
             _, w_hat, W = oracle.weights(tokens, steps, idx)
             assert rec.w_hat == [float(np.float32(w)) for w in w_hat], trial
             assert abs(rec.w_total - W) <= 1e-15 * W
+
+
+def test_two_contexts_on_two_streams(dd):
+    # Separate contexts own separate workspaces, so their launches may overlap on the GPU.
+    n, M = 400_003, 4
+    results = []
+    ctxs = [dd.Context(0), dd.Context(0)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    cases = []
+    for i in range(2):
+        theta, v, learners = synth.fragment_cpu(n, M, "bf16", 300 + i)
+        cases.append((theta, v, learners, torch.from_numpy(theta).cuda(), torch.from_numpy(v).cuda(),
+                      [to_torch_learner(a, "cuda") for a in learners], dd.new_records(1)))
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for i in range(2):
+            theta, v, learners, t_dev, v_dev, L, rec = cases[i]
+            ctxs[i].merge_fragment(t_dev, v_dev, L, [3, 1, 4, 1 + i], 0b1111, 2, ETA, MU,
+                                   flags=dd.DIAG_STATE, record=rec, stream=streams[i])
+    torch.cuda.synchronize()
+    for i in range(2):
+        theta, v, learners, t_dev, v_dev, L, rec = cases[i]
+        for rep in range(3):
+            ref = oracle.merge_fragment(theta, v, learners, [3, 1, 4, 1 + i], 0b1111, 2, ETA, MU)
+        got = dd.read_records(rec)[0]
+        assert got.status == 0 and got.idx == ref.idx
+        assert floor_rel_err(t_dev.cpu().numpy(), theta) <= 1e-4        # three merges without resync
+        assert float(np.max(np.abs(v_dev.cpu().numpy() - v))) <= 1e-7
+        assert abs(got.theta_sq - ref.theta_sq) <= 1e-4 * ref.theta_sq
+    for c in ctxs:
+        c.close()
