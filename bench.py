@@ -365,6 +365,46 @@ def main():
             ctx.merge_fragments_batched(frags, w.M, ldtype, eta, mu, flags=flags, records=records,
                                         stream=stream)
 
+    # ---- parity evidence on the buffers that are about to be timed: sampled windows of
+    # the very first merge (fresh state) against the oracle -----------------------------
+    parity = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and args.merge == "avg":
+        import oracle
+        f = frags[0]
+        n = f["n"]
+        win = min(1 << 16, n)
+        starts = sorted({0, max(0, (n - win) // 8 * 8), (n // 3) // 8 * 8, (2 * n // 3) // 8 * 8})
+        starts = [s0 for s0 in starts if s0 + win <= n]
+        part = [m for m in range(w.M) if (f["quorum_mask"] >> m) & 1 and f["tokens"][m] > 0]
+
+        def host_learner(t):
+            t = t.cpu()
+            return t.view(torch.int16).numpy().view(np.uint16).copy() if t.dtype == torch.bfloat16 \
+                else t.numpy().copy()
+
+        saved = [(f["global_"][s0:s0 + win].cpu().numpy().copy(),
+                  f["momentum"][s0:s0 + win].cpu().numpy().copy(),
+                  [host_learner(f["learners"][m][s0:s0 + win]) if m in part else None
+                   for m in range(w.M)]) for s0 in starts]
+        step()
+        torch.cuda.synchronize()
+        rec = dd.read_records(records)[0]
+        worst = {"t": 0.0, "v": 0.0}
+        exact = True
+        for s0, (t0, v0, ls) in zip(starts, saved):
+            ref = oracle.merge_fragment(t0, v0, ls, f["tokens"], f["quorum_mask"], f["K"], eta, mu)
+            exact &= (rec.status, rec.n_part, rec.idx) == (ref.status, ref.n_part, ref.idx)
+            exact &= rec.w_hat == [float(np.float32(x)) for x in ref.w_hat]
+            for got, want, which in ((f["global_"], t0, "t"), (f["momentum"], v0, "v")):
+                g = got[s0:s0 + win].cpu().numpy().astype(np.float64)
+                o = want.astype(np.float64)
+                rms = float(np.sqrt(np.mean(o * o))) or 1.0
+                worst[which] = max(worst[which], float(np.max(np.abs(g - o) / np.maximum(np.abs(o), rms))))
+        parity = {"windows": len(starts), "window_elems": win, "max_err_theta": worst["t"],
+                  "max_err_momentum": worst["v"], "tolerance": 1e-5,
+                  "participation_and_weights_bit_exact": bool(exact),
+                  "metric": "first merge: max |gpu - oracle| / max(|oracle|, rms(oracle))"}
+
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
@@ -499,6 +539,9 @@ def main():
         del h_learners, h_theta, h_mom
     else:
         line["e2e"] = None
+
+    if parity is not None:
+        line["parity"] = parity
 
     # ---- the oracle on the host cores, bounded sample of the same workload -----------
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -533,3 +533,20 @@ def test_two_contexts_on_two_streams(dd):
         assert abs(got.theta_sq - ref.theta_sq) <= 1e-4 * ref.theta_sq
     for c in ctxs:
         c.close()
+
+
+def test_random_shape_sweep(dd, ctx):
+    # 60 random (n, M, participants, dtype, alignment, flags, steps, output) combinations
+    rng = np.random.default_rng(77)
+    for trial in range(60):
+        n = int(rng.choice([rng.integers(1, 300), rng.integers(300, 9000), rng.integers(9000, 70000)]))
+        M = int(rng.integers(1, 13))
+        tokens = [int(t) for t in rng.integers(0, 3, size=M) * rng.integers(1, 5000, size=M)]
+        mask = int(rng.integers(0, 1 << M))
+        K = int(rng.integers(0, M + 1))
+        dtype = "bf16" if rng.random() < 0.6 else "f32"
+        flags = int(rng.choice([0, 1, 2, 4, 6, 7]))
+        steps = None if rng.random() < 0.5 else [int(x) for x in rng.integers(1, 50, size=M)]
+        run_case(dd, ctx, n, M, dtype, tokens, mask, K, seed=1000 + trial, steps=steps, flags=flags,
+                 merges=1, use_out=bool(rng.random() < 0.5), null_absent=bool(rng.random() < 0.5),
+                 shift=int(rng.choice([0, 4])))
