@@ -92,6 +92,15 @@ def _load():
         lib.ddo_apply_to_learner.restype = None
         lib.ddo_apply_to_learner.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p,
                                              ctypes.c_float, ctypes.c_size_t]
+        lib.ddo_quantize_int4.restype = None
+        lib.ddo_quantize_int4.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+                                          ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p]
+        lib.ddo_merge_fragment_int4.restype = ctypes.c_int
+        lib.ddo_merge_fragment_int4.argtypes = [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p),
+            ctypes.POINTER(ctypes.c_void_p), ctypes.c_int, u64p, u64p, ctypes.c_uint64, ctypes.c_int,
+            ctypes.c_float, ctypes.c_float, ctypes.c_int, ctypes.c_size_t, ctypes.c_void_p,
+            ctypes.POINTER(_Record)]
         lib.ddo_grace_window.restype = ctypes.c_double
         lib.ddo_grace_window.argtypes = [ctypes.c_double] * 5
         lib.ddo_select_quorum.restype = ctypes.c_int
@@ -228,3 +237,50 @@ def grace_controller_window(tau, gamma, beta, observations) -> float:
     if xs is None:
         return 0.0
     return grace_window(tau, xs[0], xs[1], xs[2], gamma)
+
+
+INT4_BLOCK = 128
+
+
+def quantize_int4(theta: np.ndarray, learner: np.ndarray):
+    """Outer gradient Theta - theta of one learner as int4 codes + one float32 scale per
+    128 elements.  Returns (codes uint8[ceil(n/2)], scales float32[ceil(n/128)])."""
+    lib = _load()
+    n = theta.size
+    assert theta.dtype == np.float32 and learner.size == n
+    codes = np.zeros((n + 1) // 2, dtype=np.uint8)
+    scales = np.zeros((n + INT4_BLOCK - 1) // INT4_BLOCK, dtype=np.float32)
+    lib.ddo_quantize_int4(theta.ctypes.data, learner.ctypes.data, int(learner.dtype == np.uint16), n,
+                          codes.ctypes.data, scales.ctypes.data)
+    return codes, scales
+
+
+def dequantize_int4(codes: np.ndarray, scales: np.ndarray, n: int) -> np.ndarray:
+    """(code - 8) * scale in float32, for tests."""
+    i = np.arange(n)
+    nib = (codes[i // 2] >> (4 * (i & 1))) & 15
+    return ((nib.astype(np.int32) - 8).astype(np.float32) * scales[i // INT4_BLOCK]).astype(np.float32)
+
+
+def merge_fragment_int4(theta: np.ndarray, v: np.ndarray, codes, scales, tokens, mask: int, K: int,
+                        eta: float, mu: float, *, steps=None, nesterov: bool = True,
+                        out_bf16: np.ndarray | None = None) -> Record:
+    """The merge with int4-compressed outer gradients, IN PLACE on theta and v."""
+    lib = _load()
+    M = len(codes)
+    n = theta.size
+    cp = (ctypes.c_void_p * M)(*[None if a is None else a.ctypes.data for a in codes])
+    sp = (ctypes.c_void_p * M)(*[None if a is None else a.ctypes.data for a in scales])
+    rec = _Record()
+    rc = lib.ddo_merge_fragment_int4(
+        theta.ctypes.data, v.ctypes.data, cp, sp, M, _u64(tokens),
+        None if steps is None else _u64(steps), ctypes.c_uint64(mask & (2**64 - 1)), K,
+        ctypes.c_float(eta), ctypes.c_float(mu), int(nesterov), n,
+        None if out_bf16 is None else out_bf16.ctypes.data, ctypes.byref(rec))
+    if rc != 0:
+        raise ValueError("oracle: invalid int4 merge arguments")
+    s = rec.n_part
+    return Record(status=rec.status, n_part=s, idx=[int(rec.idx[j]) for j in range(s)],
+                  w_hat=[float(rec.w_hat[j]) for j in range(s)], w_total=float(rec.w_total),
+                  delta_sq=float(rec.delta_sq), theta_sq=float(rec.theta_sq),
+                  mom_sq=float(rec.mom_sq), delta_m_sq=[0.0] * s)

@@ -270,6 +270,99 @@ void ddo_apply_to_learner(void *learner, int learner_is_bf16, const float *Theta
     }
 }
 
+/* ---- int4 compression of outer gradients (appendix "Outer gradients compression") ---- */
+
+/*
+ * The paper compresses outer gradients to 4 bits per value before they are merged
+ * but gives no quantiser.  PARITY UNPINNED BY THE PAPER; the reading used here:
+ * blocks of 128 consecutive elements, D = Theta - theta in float32, one float32
+ * scale = max|D| / 7 per block, code = round-half-even(D / scale) clamped to
+ * [-7, 7], stored as code + 8 in a nibble (even element in the low nibble).
+ * Every decision is taken in float32, the precision the kernel uses.
+ */
+#define DDO_INT4_BLOCK 128
+
+void ddo_quantize_int4(const float *Theta, const void *learner, int learner_is_bf16, size_t n,
+                       uint8_t *codes, float *scales)
+{
+    size_t b, i, nblocks = (n + DDO_INT4_BLOCK - 1) / DDO_INT4_BLOCK;
+    memset(codes, 0, (n + 1) / 2);
+    for (b = 0; b < nblocks; ++b) {
+        size_t lo = b * DDO_INT4_BLOCK, hi = lo + DDO_INT4_BLOCK < n ? lo + DDO_INT4_BLOCK : n;
+        float amax = 0.0f, scale;
+        for (i = lo; i < hi; ++i) {
+            float th = learner_is_bf16 ? ddo_bf16_to_f32(((const uint16_t *)learner)[i])
+                                       : ((const float *)learner)[i];
+            float d = Theta[i] - th;
+            float a = fabsf(d);
+            if (a > amax) amax = a;
+        }
+        scale = amax / 7.0f;
+        scales[b] = scale;
+        for (i = lo; i < hi; ++i) {
+            float th = learner_is_bf16 ? ddo_bf16_to_f32(((const uint16_t *)learner)[i])
+                                       : ((const float *)learner)[i];
+            float d = Theta[i] - th;
+            float q = scale > 0.0f ? rintf(d / scale) : 0.0f;
+            int code;
+            if (q > 7.0f) q = 7.0f;
+            if (q < -7.0f) q = -7.0f;
+            code = (int)q + 8;
+            codes[i / 2] |= (uint8_t)(code << (4 * (i & 1)));
+        }
+    }
+}
+
+/* Outer gradient of element i as the syncer sees it: (code - 8) * scale, in float32. */
+static double int4_at(const uint8_t *codes, const float *scales, size_t i)
+{
+    int code = (codes[i / 2] >> (4 * (i & 1))) & 15;
+    float d = (float)(code - 8) * scales[i / DDO_INT4_BLOCK];
+    return (double)d;
+}
+
+/*
+ * The merge of Algorithm 2 with compressed outer gradients: Delta = sum_m w_hat_m D^_m,
+ * then the same outer step.  Participation and weights exactly as ddo_merge_fragment.
+ */
+int ddo_merge_fragment_int4(float *Theta, float *v, const uint8_t *const *codes,
+                            const float *const *scales, int M, const uint64_t *tokens,
+                            const uint64_t *steps, uint64_t mask, int K, float eta, float mu,
+                            int nesterov, size_t n, uint16_t *out_bf16, ddo_record *rec)
+{
+    double w_hat[DDO_MAX_LEARNERS];
+    const double eta_d = (double)eta, mu_d = (double)mu;
+    size_t i;
+    int j, s, st;
+    memset(rec, 0, sizeof *rec);
+    st = ddo_participants(mask, tokens, M, K, rec->idx, &rec->n_part);
+    if (st == DDO_INVALID) return DDO_INVALID;
+    s = rec->n_part;
+    if (st != DDO_STATUS_OK) { rec->status = st; return 0; }
+    st = ddo_weights(tokens, steps, rec->idx, s, w_hat, &rec->w_total);
+    if (st == DDO_INVALID) return DDO_INVALID;
+    if (st != DDO_STATUS_OK) { rec->status = st; return 0; }
+    for (j = 0; j < s; ++j) {
+        rec->w_hat[j] = w_hat[j];
+        if (codes[rec->idx[j]] == NULL || scales[rec->idx[j]] == NULL) return DDO_INVALID;
+    }
+    for (i = 0; i < n; ++i) {
+        double d = 0.0, vn, u, Tn;
+        for (j = 0; j < s; ++j) d += w_hat[j] * int4_at(codes[rec->idx[j]], scales[rec->idx[j]], i);
+        vn = mu_d * (double)v[i] + d;
+        u = nesterov ? d + mu_d * vn : vn;
+        Tn = (double)Theta[i] - eta_d * u;
+        v[i] = (float)vn;
+        Theta[i] = (float)Tn;
+        if (out_bf16 != NULL) out_bf16[i] = ddo_bf16_rne((float)Tn);
+        rec->delta_sq += d * d;
+        rec->theta_sq += (double)Theta[i] * (double)Theta[i];
+        rec->mom_sq += (double)v[i] * (double)v[i];
+    }
+    rec->status = DDO_STATUS_OK;
+    return 0;
+}
+
 /* ---- quorum / grace window ("Adaptive Quorum Window", Section 3.2) --------- */
 
 /*

@@ -509,3 +509,61 @@ def test_huge_token_counts():
     np.testing.assert_allclose(w_hat, [b / sum(big) for b in big], rtol=1e-15)
     with pytest.raises(ValueError):
         oracle.weights([2**63, 2**63], None, [0, 1])        # the exact sum would wrap
+
+
+# ---- int4 compression of outer gradients (reading of this build; the paper gives no quantiser) ----
+
+def test_int4_quantiser_properties():
+    n = 1000                                           # 7 full blocks of 128 and a ragged one
+    theta, _, learners = _frag(n=n, M=2, dtype="bf16", seed=71)
+    codes, scales = oracle.quantize_int4(theta, learners[0])
+    d = theta - oracle.bf16_to_f32(learners[0])        # float32 differences
+    nib = np.concatenate([codes & 15, codes >> 4]).reshape(2, -1).T.reshape(-1)[:n]
+    assert nib.min() >= 1 and nib.max() <= 15          # codes -7..7 stored as code + 8
+    dq = oracle.dequantize_int4(codes, scales, n)
+    for b in range(len(scales)):
+        blk = slice(128 * b, min(n, 128 * (b + 1)))
+        amax = np.max(np.abs(d[blk]))
+        assert scales[b] == np.float32(amax) / np.float32(7.0)
+        # nearest-code rounding: error at most half a step; the largest element is hit exactly
+        assert np.max(np.abs(dq[blk] - d[blk])) <= 0.5 * scales[b] * (1 + 1e-6)
+        k = np.argmax(np.abs(d[blk]))
+        assert abs(int(nib[blk][k]) - 8) == 7
+    # quantising an already quantised gradient changes nothing
+    learner2 = (theta.astype(np.float64) - dq.astype(np.float64)).astype(np.float32)
+    d2 = theta - learner2
+    if np.array_equal(d2, dq):                         # only when Theta - (Theta - dq) is exact
+        codes2, scales2 = oracle.quantize_int4(theta, learner2)
+        np.testing.assert_array_equal(codes2, codes)
+    # an all-zero block has scale 0 and code 0 everywhere
+    codes0, scales0 = oracle.quantize_int4(theta, theta.copy())
+    assert np.all(scales0 == 0) and np.all((codes0 & 15) == 8) and np.all((codes0[: n // 2] >> 4) == 8)
+    # ties round to even: d / scale = 2.5 -> 2, 3.5 -> 4
+    t = np.zeros(128, dtype=np.float32)
+    l = np.zeros(128, dtype=np.float32)
+    l[0], l[1], l[2] = -7.0, -2.5, -3.5                # d = 7 (scale 1), 2.5, 3.5
+    c, s_ = oracle.quantize_int4(t, l)
+    assert s_[0] == 1.0 and (c[0] & 15) == 15 and (c[0] >> 4) == 10 and (c[1] & 15) == 12
+
+
+def test_int4_merge_equals_plain_merge_of_dequantised_gradients():
+    n, M = 3000, 4
+    theta, v, learners = _frag(n=n, M=M, dtype="bf16", seed=72)
+    v[:] = np.random.default_rng(1).normal(0, 1e-3, n).astype(np.float32)
+    tokens, mask = [10, 0, 30, 40], 0b1101
+    q = [oracle.quantize_int4(theta, a) for a in learners]
+    # a learner whose copy IS Theta - D^ reproduces the compressed gradient (up to one float32 rounding)
+    recon = [(theta.astype(np.float64) - oracle.dequantize_int4(c, s_, n)).astype(np.float32) for c, s_ in q]
+    t_a, v_a = theta.copy(), v.copy()
+    ra = oracle.merge_fragment_int4(t_a, v_a, [c for c, _ in q], [s_ for _, s_ in q], tokens, mask, 2,
+                                    0.7, 0.9)
+    t_b, v_b = theta.copy(), v.copy()
+    rb = oracle.merge_fragment(t_b, v_b, recon, tokens, mask, 2, 0.7, 0.9)
+    assert ra.idx == rb.idx == [0, 2, 3] and ra.w_hat == rb.w_hat
+    np.testing.assert_allclose(v_a, v_b, rtol=0, atol=2e-9)
+    np.testing.assert_allclose(t_a, t_b, rtol=0, atol=1.5e-8)          # an ulp of Theta at 0.1
+    # and it stays within half a quantisation step of the uncompressed merge
+    t_c, v_c = theta.copy(), v.copy()
+    oracle.merge_fragment(t_c, v_c, learners, tokens, mask, 2, 0.7, 0.9)
+    step = max(float(np.max(s_)) for _, s_ in q)
+    assert np.max(np.abs(v_a - v_c)) <= 0.5 * step * 1.001
