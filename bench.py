@@ -48,8 +48,9 @@ def parse_args():
     ap.add_argument("--cpu-sample", type=int, default=1 << 27,
                     help="elements of the workload the CPU oracle is timed on")
     ap.add_argument("--out-bf16", action="store_true", help="also write the bf16 broadcast copy")
-    ap.add_argument("--merge", choices=["avg", "rda"], default="avg",
-                    help="weighted direct averaging (the headline path) or radial-directional")
+    ap.add_argument("--merge", choices=["avg", "rda", "int4"], default="avg",
+                    help="weighted direct averaging (the headline path), radial-directional, or "
+                         "direct averaging of int4-compressed outer gradients")
     ap.add_argument("--resident", choices=["all", "participants"], default="all",
                     help="allocate every learner copy, or only those that take part")
     ap.add_argument("--sharding", choices=["replica", "range"], default="replica",
@@ -352,8 +353,28 @@ def main():
     eta, mu = synth.OUTER_LR, synth.OUTER_MU
     stream = torch.cuda.current_stream()
 
+    int4_codes = int4_scales = None
+    if args.merge == "int4":
+        # the learners' side, outside the timed region: compress every participant's outer gradient
+        assert w.P == 1, "--merge int4 takes a single-fragment workload"
+        f = frags[0]
+        n0 = f["n"]
+        int4_codes, int4_scales = [None] * w.M, [None] * w.M
+        for m in range(w.M):
+            if (f["quorum_mask"] >> m) & 1 and f["tokens"][m] > 0:
+                int4_codes[m] = torch.empty((n0 + 1) // 2, dtype=torch.uint8, device=device)
+                int4_scales[m] = torch.empty((n0 + 127) // 128, dtype=torch.float32, device=device)
+                ctx.quantize_outer_gradient_int4(f["global_"], f["learners"][m], int4_codes[m],
+                                                 int4_scales[m], n=n0, learner_dtype=ldtype)
+        torch.cuda.synchronize()
+
     def step():
-        if args.merge == "rda":
+        if args.merge == "int4":
+            f = frags[0]
+            ctx.merge_fragment_int4(f["global_"], f["momentum"], int4_codes, int4_scales, f["tokens"],
+                                    f["quorum_mask"], f["K"], eta, mu, n=f["n"], flags=flags,
+                                    out_bf16=f["out_bf16"], record=records, stream=stream)
+        elif args.merge == "rda":
             ctx.merge_fragments_batched_rda(frags, w.M, ldtype, eta, mu, flags=flags,
                                             records=records, stream=stream)
         elif w.P == 1:
@@ -450,6 +471,9 @@ def main():
     value = ddist.whole_job_rate(job_params, args.steps, 1, max_ms)
     alg_bytes = w.algorithmic_bytes(out_bf16=args.out_bf16)
     launches_per_step = 1
+    if args.merge == "int4":
+        alg_bytes = sum(int(n * (w.participants(p) * (0.5 + 4.0 / 128.0) + 16))
+                        for p, n in enumerate(w.fragment_sizes))
     if args.merge == "rda":
         # learner copies and Theta are read twice (norms, direction), the direction is
         # written and read back once: 2 (s b + 4) + 24 bytes per parameter

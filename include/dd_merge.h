@@ -207,6 +207,36 @@ int dd_merge_fragments_batched_rda(dd_ctx *ctx, const dd_fragment_desc *descs, i
                                    size_t scratch_elems, void *cuda_stream);
 
 /*
+ * int4 compression of outer gradients (Appendix "Outer gradients compression": 16 -> 4
+ * bits per value before the merge, comparable quality; 2 and 1 bit are not).  The paper
+ * prints no quantiser; this library's reading, fixed here so that both ends agree:
+ *   - blocks of DD_INT4_BLOCK consecutive elements, the last one possibly shorter;
+ *   - D = Theta - theta_m in float32; scale = max|D| / 7 (float32), one per block;
+ *   - code = D / scale rounded to nearest (ties to even), clamped to [-7, 7]; a block of
+ *     zeros has scale 0 and codes 0;
+ *   - element i's code + 8 sits in nibble (i & 1) of byte i / 2 (even element low).
+ *
+ * dd_quantize_outer_gradient_int4 is the learner side:
+ *   global [device] float32[n]; learner [device] learner_dtype[n];
+ *   codes [device] (n + 1) / 2 bytes, 2-byte aligned; scales [device] float32[ceil(n / 128)].
+ *
+ * dd_merge_fragment_int4 is dd_merge_fragment with the outer gradients arriving
+ * compressed: Delta = sum_{m in S} w^_m (code_m - 8) scale_m, same outer step, same
+ * participation, weights, record and errors.  code_ptrs / scale_ptrs are host arrays
+ * of M device pointers (16- and 4-byte aligned).  DD_DIAG_PER_LEARNER is not offered.
+ * Bytes per merged parameter: s (1/2 + 4/128) + 16.
+ */
+#define DD_INT4_BLOCK 128
+int dd_quantize_outer_gradient_int4(dd_ctx *ctx, const float *global, const void *learner,
+                                    dd_dtype learner_dtype, size_t n, uint8_t *codes, float *scales,
+                                    void *cuda_stream);
+int dd_merge_fragment_int4(dd_ctx *ctx, float *global, float *momentum,
+                           const uint8_t *const *code_ptrs, const float *const *scale_ptrs, int M,
+                           const uint64_t *tokens, const uint64_t *steps, uint64_t quorum_mask,
+                           int K, float outer_lr, float outer_mu, uint32_t flags, size_t n,
+                           void *out_bf16, dd_merge_record *record, void *cuda_stream);
+
+/*
  * The same update for a fragment whose operands live in HOST memory -- the
  * paper's syncer pulls each learner's fragment from that learner's host RAM and
  * keeps the global state off the accelerators (Section 4, system overview).

@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libddmerge.so")
-SOURCES = ["dd_merge.cu", "dd_host_stream.cu", "dd_noalloc.cu", "dd_broadcast.cu", "dd_host.cpp"]
+SOURCES = ["dd_merge.cu", "dd_host_stream.cu", "dd_noalloc.cu", "dd_broadcast.cu", "dd_int4.cu", "dd_host.cpp"]
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
     "--shared", "-Xcompiler", "-fPIC", "-Xptxas", "-v", "-cudart", "static",

@@ -73,4 +73,14 @@ inline int cuda_fail(dd_ctx *ctx, cudaError_t e, const char *where)
 
 void host_pipe_destroy(dd_ctx *ctx);
 
+// Shared by the entry points (defined in dd_merge.cu).
+// Validates one fragment's arguments and fills its device descriptor (tile range excluded);
+// learner_bytes is the size of one learner buffer, for the overlap checks.
+int fill_fragment(DevFrag &d, float *global, float *momentum, void *out_bf16,
+                  const void *const *learner_ptrs, const uint64_t *tokens, const uint64_t *steps,
+                  uint64_t mask, int K, uint64_t n, int M, size_t learner_bytes);
+int check_common(const dd_ctx *ctx, int M, dd_dtype dtype, float lr, float mu, uint32_t flags);
+// Grows the diagnostics workspace to P x nq x grid partial sums (and P tickets).
+int ensure_workspace(dd_ctx *ctx, size_t P, size_t nq, size_t grid);
+
 }  // namespace ddm

@@ -81,17 +81,16 @@ static bool overlaps(const void *a, size_t abytes, const void *b, size_t bbytes)
 static bool misaligned(const void *p) { return ((uintptr_t)p & 15u) != 0; }
 
 // Validates one fragment and fills its device descriptor (tile range excluded).
-static int fill_fragment(DevFrag &d, float *global, float *momentum, void *out_bf16,
-                         const void *const *learner_ptrs, const uint64_t *tokens,
-                         const uint64_t *steps, uint64_t mask, int K, uint64_t n, int M,
-                         dd_dtype dtype)
+int fill_fragment(DevFrag &d, float *global, float *momentum, void *out_bf16,
+                  const void *const *learner_ptrs, const uint64_t *tokens, const uint64_t *steps,
+                  uint64_t mask, int K, uint64_t n, int M, size_t learner_bytes)
 {
     if (!learner_ptrs || !tokens) return DD_ERR_INVALID_ARG;
     if (K < 0 || K > M) return DD_ERR_INVALID_ARG;
     if (n > 0 && (!global || !momentum)) return DD_ERR_INVALID_ARG;
     if (n > kMaxFragmentElems) return DD_ERR_TOO_LARGE;
     if (misaligned(global) || misaligned(momentum) || misaligned(out_bf16)) return DD_ERR_ALIGNMENT;
-    const size_t lb = (dtype == DD_BF16 ? 2u : 4u) * (size_t)n;
+    const size_t lb = learner_bytes;
     if (overlaps(global, 4 * n, momentum, 4 * n) || overlaps(global, 4 * n, out_bf16, 2 * n) ||
         overlaps(momentum, 4 * n, out_bf16, 2 * n))
         return DD_ERR_ALIAS;
@@ -124,13 +123,18 @@ static int fill_fragment(DevFrag &d, float *global, float *momentum, void *out_b
     return DD_OK;
 }
 
+static size_t learner_bytes_of(dd_dtype dtype, uint64_t n)
+{
+    return (dtype == DD_BF16 ? 2u : 4u) * (size_t)n;
+}
+
 static unsigned long long tiles_of(uint64_t n)
 {
     const unsigned long long t = (n + kTileElems - 1) / kTileElems;
     return t ? t : 1;       // an empty fragment still owns one (empty) tile so its record is written
 }
 
-static int check_common(const dd_ctx *ctx, int M, dd_dtype dtype, float lr, float mu, uint32_t flags)
+int check_common(const dd_ctx *ctx, int M, dd_dtype dtype, float lr, float mu, uint32_t flags)
 {
     if (!ctx) return DD_ERR_INVALID_ARG;
     if (M > DD_MAX_LEARNERS) return DD_ERR_TOO_MANY_LEARNERS;
@@ -144,7 +148,7 @@ static int check_common(const dd_ctx *ctx, int M, dd_dtype dtype, float lr, floa
 
 // Grows the diagnostics workspace; growth waits for the device to drain because
 // kernels in flight may still use the old one.
-static int ensure_workspace(dd_ctx *ctx, size_t P, size_t nq, size_t grid)
+int ensure_workspace(dd_ctx *ctx, size_t P, size_t nq, size_t grid)
 {
     const size_t need = P * nq * grid;
     if (need > ctx->partials_cap) {
@@ -273,7 +277,7 @@ extern "C" int dd_merge_fragment(dd_ctx *ctx, float *global, float *momentum,
     if (rc != DD_OK) return rc;
     DevFrag frag;
     rc = fill_fragment(frag, global, momentum, out_bf16, learner_ptrs, tokens, steps, quorum_mask, K,
-                       n, M, learner_dtype);
+                       n, M, learner_bytes_of(learner_dtype, n));
     if (rc != DD_OK) return rc;
     if (n == 0 && record == nullptr) return DD_OK;
     frag.tile_begin = 0;
@@ -327,7 +331,7 @@ extern "C" int dd_merge_fragments_batched(dd_ctx *ctx, const dd_fragment_desc *d
     for (int p = 0; p < P; ++p) {
         const dd_fragment_desc &d = descs[p];
         rc = fill_fragment(slot.host[p], d.global, d.momentum, d.out_bf16, d.learner_ptrs, d.tokens,
-                           d.steps, d.quorum_mask, d.K, d.n, M, learner_dtype);
+                           d.steps, d.quorum_mask, d.K, d.n, M, learner_bytes_of(learner_dtype, d.n));
         if (rc != DD_OK) return rc;
         slot.host[p].tile_begin = tile;
         tile += tiles_of(d.n);
@@ -436,7 +440,7 @@ extern "C" int dd_merge_fragments_batched_rda(dd_ctx *ctx, const dd_fragment_des
         const dd_fragment_desc &d = descs[p];
         DevFrag &f = slot.host[p];
         rc = fill_fragment(f, d.global, d.momentum, d.out_bf16, d.learner_ptrs, d.tokens, d.steps,
-                           d.quorum_mask, d.K, d.n, M, learner_dtype);
+                           d.quorum_mask, d.K, d.n, M, learner_bytes_of(learner_dtype, d.n));
         if (rc != DD_OK) return rc;
         f.kind = (!merge_kinds || merge_kinds[p] == DD_MERGE_RDA) ? DD_MERGE_RDA : DD_MERGE_AVG;
         if (f.kind == DD_MERGE_RDA) {

@@ -28,6 +28,7 @@ EXPORTS = (
     "dd_create", "dd_destroy", "dd_merge_fragment", "dd_merge_fragments_batched",
     "dd_merge_fragment_host", "dd_merge_fragments_batched_noalloc",
     "dd_merge_fragment_rda", "dd_merge_fragments_batched_rda",
+    "dd_quantize_outer_gradient_int4", "dd_merge_fragment_int4",
     "dd_broadcast_fragment", "dd_grace_controller_init", "dd_grace_controller_observe",
     "dd_grace_controller_window", "dd_plan_fragments", "dd_select_quorum", "dd_grace_window", "dd_status_string", "dd_last_cuda_error",
     "dd_launch_geometry",
@@ -102,6 +103,12 @@ def _load() -> ctypes.CDLL:
         vp, ctypes.POINTER(CFragmentDesc), ctypes.c_int, ctypes.c_int, ctypes.c_int,
         ctypes.c_float, ctypes.c_float, ctypes.c_uint32, ctypes.POINTER(ctypes.c_uint8), vp, vp,
         ctypes.c_size_t, vp]
+    lib.dd_quantize_outer_gradient_int4.restype = ctypes.c_int
+    lib.dd_quantize_outer_gradient_int4.argtypes = [vp, vp, vp, ctypes.c_int, ctypes.c_size_t, vp, vp, vp]
+    lib.dd_merge_fragment_int4.restype = ctypes.c_int
+    lib.dd_merge_fragment_int4.argtypes = [
+        vp, vp, vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.c_int, u64p, u64p, ctypes.c_uint64,
+        ctypes.c_int, ctypes.c_float, ctypes.c_float, ctypes.c_uint32, ctypes.c_size_t, vp, vp, vp]
     lib.dd_merge_fragment_host.restype = ctypes.c_int
     lib.dd_merge_fragment_host.argtypes = [
         vp, vp, vp, ctypes.POINTER(vp), ctypes.c_int, ctypes.c_int, u64p, u64p, ctypes.c_uint64,
@@ -304,6 +311,35 @@ class Context:
             self._h, _ptr(global_), ptrs, M, learner_dtype,
             ctypes.c_uint64(apply_mask & (2**64 - 1)), ctypes.c_float(alpha), ctypes.c_size_t(n),
             _stream_handle(stream)))
+
+    def quantize_outer_gradient_int4(self, global_, learner, codes, scales, *, n: int | None = None,
+                                     learner_dtype: int | None = None, stream=None) -> None:
+        """``dd_quantize_outer_gradient_int4``: ``codes`` uint8[(n+1)//2], ``scales``
+        float32[ceil(n/128)], both device tensors written in place."""
+        if n is None:
+            n = int(global_.numel())
+        if learner_dtype is None:
+            learner_dtype = _infer_dtype([learner])
+        self._check(lib.dd_quantize_outer_gradient_int4(
+            self._h, _ptr(global_), _ptr(learner), learner_dtype, ctypes.c_size_t(n), _ptr(codes),
+            _ptr(scales), _stream_handle(stream)))
+
+    def merge_fragment_int4(self, global_, momentum, codes, scales, tokens, quorum_mask: int, K: int,
+                            outer_lr: float, outer_mu: float, *, n: int | None = None, steps=None,
+                            flags: int = 0, out_bf16=None, record=None, stream=None) -> None:
+        """``dd_merge_fragment_int4``: ``codes`` / ``scales`` are lists of M device tensors
+        (or None for absent learners)."""
+        M = len(codes)
+        if n is None:
+            n = int(global_.numel())
+        cp = (ctypes.c_void_p * M)(*[_ptr(t) for t in codes])
+        sp = (ctypes.c_void_p * M)(*[_ptr(t) for t in scales])
+        self._check(lib.dd_merge_fragment_int4(
+            self._h, _ptr(global_), _ptr(momentum), cp, sp, M, _u64_array(tokens),
+            None if steps is None else _u64_array(steps),
+            ctypes.c_uint64(quorum_mask & (2**64 - 1)), int(K), ctypes.c_float(outer_lr),
+            ctypes.c_float(outer_mu), ctypes.c_uint32(flags), ctypes.c_size_t(n), _ptr(out_bf16),
+            _ptr(record), _stream_handle(stream)))
 
     def merge_fragment_host(self, global_, momentum, learners, tokens, quorum_mask: int, K: int,
                             outer_lr: float, outer_mu: float, *, n: int | None = None,
