@@ -26,23 +26,43 @@ quantize_int4_kernel(const float *__restrict__ theta, const void *__restrict__ l
                      unsigned long long n, unsigned char *__restrict__ codes, float *__restrict__ scales)
 {
     const int lane = threadIdx.x & 31;
+    const bool vec_ok = (((unsigned long long)theta | (unsigned long long)learner) & 15ull) == 0;
     const unsigned long long nblocks = (n + kInt4Block - 1) / kInt4Block;
     const unsigned long long warps = (unsigned long long)gridDim.x * (blockDim.x >> 5);
     for (unsigned long long b = (unsigned long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
          b < nblocks; b += warps) {
         const unsigned long long e0 = b * kInt4Block + 4ull * lane;
-        float d[4];
+        float d[4], T[4], th[4];
         float amax = 0.0f;
+        if (vec_ok && e0 + 3 < n) {
+            // 16 bytes of Theta and 8 (bf16) or 16 (fp32) bytes of the learner copy per lane
+            const float4 t4 = __ldcs(reinterpret_cast<const float4 *>(theta + e0));
+            T[0] = t4.x; T[1] = t4.y; T[2] = t4.z; T[3] = t4.w;
+            if (BF16) {
+                const uint2 w = __ldcs(reinterpret_cast<const uint2 *>(
+                    reinterpret_cast<const uint16_t *>(learner) + e0));
+                th[0] = __uint_as_float(w.x << 16); th[1] = __uint_as_float(w.x & 0xffff0000u);
+                th[2] = __uint_as_float(w.y << 16); th[3] = __uint_as_float(w.y & 0xffff0000u);
+            } else {
+                const float4 l4 = __ldcs(reinterpret_cast<const float4 *>(
+                    reinterpret_cast<const float *>(learner) + e0));
+                th[0] = l4.x; th[1] = l4.y; th[2] = l4.z; th[3] = l4.w;
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const unsigned long long e = e0 + k;
+                T[k] = th[k] = 0.0f;
+                if (e < n) {
+                    T[k] = theta[e];
+                    th[k] = BF16 ? __uint_as_float((unsigned)reinterpret_cast<const uint16_t *>(learner)[e] << 16)
+                                 : reinterpret_cast<const float *>(learner)[e];
+                }
+            }
+        }
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            const unsigned long long e = e0 + k;
-            float th = 0.0f, T = 0.0f;
-            if (e < n) {
-                T = theta[e];
-                th = BF16 ? __uint_as_float((unsigned)reinterpret_cast<const uint16_t *>(learner)[e] << 16)
-                          : reinterpret_cast<const float *>(learner)[e];
-            }
-            d[k] = __fsub_rn(T, th);
+            d[k] = __fsub_rn(T[k], th[k]);
             amax = fmaxf(amax, fabsf(d[k]));
         }
 #pragma unroll
