@@ -529,14 +529,26 @@ def main():
         f = frags[0]
         n = f["n"]
         part = [m for m in range(w.M) if (f["quorum_mask"] >> m) & 1 and f["tokens"][m] > 0]
+        # Page-locked host memory is bounded: every rank of the node pins its own buffers, so
+        # with several ranks (or little free host memory) the end-to-end leg streams a leading
+        # slice of the fragment instead of all of it.
+        esz0 = 2 if w.learner_dtype == "bf16" else 4
+        per_elem = len(part) * esz0 + 8
+        try:
+            avail = next(int(l.split()[1]) * 1024 for l in open("/proc/meminfo") if l.startswith("MemAvailable"))
+        except Exception:
+            avail = 64 << 30
+        local_world = int(os.environ.get("LOCAL_WORLD_SIZE", str(world)))
+        budget = int(0.4 * avail / max(local_world, 1))
+        n = max(8, min(n, budget // per_elem) // 8 * 8)
         h_theta = torch.empty(n, dtype=torch.float32, pin_memory=True)
         h_mom = torch.empty(n, dtype=torch.float32, pin_memory=True)
-        h_theta.copy_(f["global_"])
-        h_mom.copy_(f["momentum"])
+        h_theta.copy_(f["global_"][:n])
+        h_mom.copy_(f["momentum"][:n])
         h_learners = [None] * w.M
         for m in part:
             h_learners[m] = torch.empty(n, dtype=f["learners"][m].dtype, pin_memory=True)
-            h_learners[m].copy_(f["learners"][m])
+            h_learners[m].copy_(f["learners"][m][:n])
         esz = 2 if w.learner_dtype == "bf16" else 4
         h2d = n * (len(part) * esz + 8)
         d2h = n * 8 + dd.RECORD_BYTES
@@ -554,10 +566,11 @@ def main():
         dt = time.perf_counter() - t0
         assert rec.status == 0
         dt_max = ddist.max_over_ranks(dt, device=device)
-        e2e_params = job_params            # every rank streams its own copy / its own range
+        # every rank streams its own copy (or its own range) of n elements per step
+        e2e_params = n * world
         line["e2e"] = {"value": e2e_params * args.e2e_steps / dt_max, "unit": UNIT,
                        "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                       "steps": args.e2e_steps,
+                       "steps": args.e2e_steps, "elements_per_rank_step": n,
                        "path": "dd_merge_fragment_host: pinned host buffers, chunked H2D -> "
                                "kernel -> D2H pipeline, blocking"}
         del h_learners, h_theta, h_mom
