@@ -602,6 +602,19 @@ def main():
             "sample": f"first {ns} elements of fragment 0 of {w.name}, {len(part)} participating "
                       f"{w.learner_dtype} learners, one merge, {dt:.1f} s, single thread of "
                       f"{os.cpu_count()} host cores"}
+        # Beside it, because the paper's own syncer is a CPU program: the same element loop
+        # spread over all host cores (OpenMP; not the checked oracle, a timing baseline only).
+        try:
+            cores = len(os.sched_getaffinity(0))
+            t0 = time.perf_counter()
+            oracle.merge_fragment_all_cores(theta, mom, learners, f["tokens"], f["quorum_mask"], f["K"],
+                                            eta, mu)
+            dt_all = time.perf_counter() - t0
+            line["cpu_baseline"]["all_cores"] = {"value": ns / dt_all, "unit": UNIT, "cores": cores,
+                                                 "kind": "oracle element loop under OpenMP",
+                                                 "seconds": dt_all}
+        except Exception as exc:      # no OpenMP runtime on the box: the oracle figure stands alone
+            line["cpu_baseline"]["all_cores"] = {"unavailable": str(exc)[:120]}
     elif rank == 0:
         line["cpu_baseline"] = None
 

@@ -284,3 +284,44 @@ def merge_fragment_int4(theta: np.ndarray, v: np.ndarray, codes, scales, tokens,
                   w_hat=[float(rec.w_hat[j]) for j in range(s)], w_total=float(rec.w_total),
                   delta_sq=float(rec.delta_sq), theta_sq=float(rec.theta_sq),
                   mom_sq=float(rec.mom_sq), delta_m_sq=[0.0] * s)
+
+
+# ---- all-cores CPU baseline (benchmark only; not the checked oracle) ---------------------
+
+_PAR_SRC = os.path.join(_HERE, "dd_cpu_parallel.c")
+_PAR_LIB = os.path.join(_HERE, "libdd_cpu_parallel.so")
+_par = None
+
+
+def build_parallel(force: bool = False) -> str:
+    if force or not os.path.exists(_PAR_LIB) or os.path.getmtime(_PAR_LIB) < os.path.getmtime(_PAR_SRC):
+        tmp = _PAR_LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared", "-Wall",
+                               "-ffp-contract=off", "-o", tmp, _PAR_SRC])
+        os.replace(tmp, _PAR_LIB)
+    return _PAR_LIB
+
+
+def merge_fragment_all_cores(theta, v, learners, tokens, mask, K, eta, mu, *, nesterov=True):
+    """The direct-averaging merge with the element loop spread over all host cores
+    (OpenMP).  Participation and weights come from the single-threaded oracle.
+    Returns ||Delta||^2, or None when the quorum is not met."""
+    global _par
+    if _par is None:
+        _par = ctypes.CDLL(build_parallel())
+        _par.ddp_merge_fragment.restype = ctypes.c_double
+        _par.ddp_merge_fragment.argtypes = [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p),
+            ctypes.POINTER(ctypes.c_double), ctypes.c_int, ctypes.c_int, ctypes.c_float,
+            ctypes.c_float, ctypes.c_int, ctypes.c_size_t]
+    st, idx = participants(mask, tokens, K)
+    if st != STATUS_OK:
+        return None
+    _, w_hat, _ = weights(tokens, None, idx)
+    chosen = [learners[m] for m in idx]
+    is_bf16 = chosen[0].dtype == np.uint16
+    ptrs = (ctypes.c_void_p * len(idx))(*[a.ctypes.data for a in chosen])
+    wh = (ctypes.c_double * len(idx))(*w_hat)
+    return float(_par.ddp_merge_fragment(theta.ctypes.data, v.ctypes.data, ptrs, wh, len(idx),
+                                         int(is_bf16), ctypes.c_float(eta), ctypes.c_float(mu),
+                                         int(nesterov), theta.size))

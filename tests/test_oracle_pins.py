@@ -567,3 +567,17 @@ def test_int4_merge_equals_plain_merge_of_dequantised_gradients():
     oracle.merge_fragment(t_c, v_c, learners, tokens, mask, 2, 0.7, 0.9)
     step = max(float(np.max(s_)) for _, s_ in q)
     assert np.max(np.abs(v_a - v_c)) <= 0.5 * step * 1.001
+
+
+def test_all_cores_baseline_agrees_with_the_oracle():
+    # the OpenMP loop is only a timing baseline, but it must compute the same merge
+    theta, v, learners = _frag(n=50_001, M=5, dtype="bf16", seed=81)
+    tokens, mask = [10, 20, 0, 40, 50], 0b11101
+    t_a, v_a = theta.copy(), v.copy()
+    ref = oracle.merge_fragment(t_a, v_a, learners, tokens, mask, 2, 0.7, 0.9)
+    t_b, v_b = theta.copy(), v.copy()
+    dsq = oracle.merge_fragment_all_cores(t_b, v_b, learners, tokens, mask, 2, 0.7, 0.9)
+    np.testing.assert_array_equal(t_a, t_b)
+    np.testing.assert_array_equal(v_a, v_b)
+    assert abs(dsq - ref.delta_sq) <= 1e-12 * ref.delta_sq
+    assert oracle.merge_fragment_all_cores(t_b, v_b, learners, tokens, mask, 5, 0.7, 0.9) is None
