@@ -485,7 +485,7 @@ def main():
     slowest = sorted(range(len(per_launch_ms)), key=lambda k: -per_launch_ms[k])[:3]
     achieved = alg_bytes / (avg_launch_ms * 1e-3) / 1e9
     peak, peak_kind = hbm_peak()
-    traffic_pp = NCU_TRAFFIC_BYTES_PER_PARAM.get(args.workload)
+    traffic_pp = NCU_TRAFFIC_BYTES_PER_PARAM.get(args.workload) if args.merge == "avg" else None
     roofline = {
         "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
         "frac": achieved / peak, "peak_source": f"of {peak_kind}",
