@@ -15,6 +15,7 @@
 namespace ddm {
 
 constexpr int kInt4Block = DD_INT4_BLOCK;     // elements per scale
+constexpr int kInt4Batch = 8;                 // participants whose loads a thread keeps in flight
 
 // ---- learner side: quantise Theta - theta ---------------------------------------------
 //
@@ -99,7 +100,7 @@ struct ScalePtrs {
     const float *p[DD_MAX_LEARNERS];
 };
 
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 3)
 merge_int4_kernel(const __grid_constant__ DevFrag frag, const __grid_constant__ ScalePtrs sp,
                   const __grid_constant__ Common c)
 {
@@ -127,23 +128,38 @@ merge_int4_kernel(const __grid_constant__ DevFrag frag, const __grid_constant__ 
 #pragma unroll
         for (int k = 0; k < 8; ++k) acc[k] = make_float2(0.0f, 0.0f);
         const unsigned long long blk = vi / (kInt4Block / 16);
-#pragma unroll 2
-        for (int j = 0; j < s; ++j) {
-            const uint2 words = __ldcs(reinterpret_cast<const uint2 *>(sm.ptr[j]) + vi);
-            const float ws = sm.w[j] * __ldg(sptr[j] + blk);
-            const float2 ws2 = make_float2(ws, ws);
-            // nibble -> float without integer conversions: even nibbles in the bytes of `lo`, odd
-            // ones in `hi`; a byte permute drops each under the exponent of 2^23, giving 2^23 +
-            // code + 8, and one packed add removes 2^23 + 8.
+        // kInt4Batch participants at a time: all their loads are issued before the first is used
+#pragma unroll 1
+        for (int j0 = 0; j0 < s; j0 += kInt4Batch) {
+            uint2 words[kInt4Batch];
+            float ws[kInt4Batch];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const unsigned word = h ? words.y : words.x;
-                const unsigned lo = word & 0x0f0f0f0fu, hi = (word >> 4) & 0x0f0f0f0fu;
+            for (int b = 0; b < kInt4Batch; ++b) {
+                if (j0 + b < s) {
+                    words[b] = __ldcs(reinterpret_cast<const uint2 *>(sm.ptr[j0 + b]) + vi);
+                    ws[b] = __ldg(sptr[j0 + b] + blk);
+                }
+            }
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const float2 m = make_float2(__uint_as_float(__byte_perm(lo, 0x4b000000u, 0x7650u + k)),
-                                                 __uint_as_float(__byte_perm(hi, 0x4b000000u, 0x7650u + k)));
-                    acc[4 * h + k] = __ffma2_rn(ws2, __fadd2_rn(m, minus_c), acc[4 * h + k]);
+            for (int b = 0; b < kInt4Batch; ++b) {
+                if (j0 + b < s) {
+                    const float w = sm.w[j0 + b] * ws[b];
+                    const float2 ws2 = make_float2(w, w);
+                    // nibble -> float without integer conversions: even nibbles in the bytes of `lo`,
+                    // odd ones in `hi`; a byte permute drops each under the exponent of 2^23, giving
+                    // 2^23 + code + 8, and one packed add removes 2^23 + 8.
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const unsigned word = h ? words[b].y : words[b].x;
+                        const unsigned lo = word & 0x0f0f0f0fu, hi = (word >> 4) & 0x0f0f0f0fu;
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const float2 m = make_float2(
+                                __uint_as_float(__byte_perm(lo, 0x4b000000u, 0x7650u + k)),
+                                __uint_as_float(__byte_perm(hi, 0x4b000000u, 0x7650u + k)));
+                            acc[4 * h + k] = __ffma2_rn(ws2, __fadd2_rn(m, minus_c), acc[4 * h + k]);
+                        }
+                    }
                 }
             }
         }
@@ -264,7 +280,7 @@ extern "C" int dd_merge_fragment_int4(dd_ctx *ctx, float *global, float *momentu
     if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
     const unsigned long long nvec = (n + 15) / 16;
     unsigned long long grid = (nvec + 255) / 256;
-    const unsigned long long cap = (unsigned long long)ctx->sm_count * 4;   // 64 registers: 4 CTAs of 256 threads per SM
+    const unsigned long long cap = (unsigned long long)ctx->sm_count * 3;   // 3 CTAs of 256 threads per SM
     if (grid > cap) grid = cap;
     if (grid == 0) grid = 1;
     frag.tile_begin = 0;
