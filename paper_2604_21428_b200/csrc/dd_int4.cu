@@ -15,6 +15,7 @@
 namespace ddm {
 
 constexpr int kInt4Block = DD_INT4_BLOCK;     // elements per scale
+constexpr int kQuantUnroll = 4;               // blocks a warp of the quantiser loads before it reduces
 constexpr int kInt4Batch = 8;                 // participants whose loads a thread keeps in flight
 
 // ---- learner side: quantise Theta - theta ---------------------------------------------
@@ -30,8 +31,49 @@ quantize_int4_kernel(const float *__restrict__ theta, const void *__restrict__ l
     const bool vec_ok = (((unsigned long long)theta | (unsigned long long)learner) & 15ull) == 0;
     const unsigned long long nblocks = (n + kInt4Block - 1) / kInt4Block;
     const unsigned long long warps = (unsigned long long)gridDim.x * (blockDim.x >> 5);
-    for (unsigned long long b = (unsigned long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-         b < nblocks; b += warps) {
+    unsigned long long b = (unsigned long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    // Whole blocks, kQuantUnroll at a time: every load is issued before the first reduction.
+    if (vec_ok) {
+        for (; b + (kQuantUnroll - 1) * warps < n / kInt4Block; b += kQuantUnroll * warps) {
+            float4 t4[kQuantUnroll];
+            float4 l4[kQuantUnroll];
+#pragma unroll
+            for (int u = 0; u < kQuantUnroll; ++u) {
+                const unsigned long long e0 = (b + u * warps) * kInt4Block + 4ull * lane;
+                t4[u] = __ldcs(reinterpret_cast<const float4 *>(theta + e0));
+                if (BF16) {
+                    const uint2 w = __ldcs(reinterpret_cast<const uint2 *>(
+                        reinterpret_cast<const uint16_t *>(learner) + e0));
+                    l4[u] = make_float4(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xffff0000u),
+                                        __uint_as_float(w.y << 16), __uint_as_float(w.y & 0xffff0000u));
+                } else {
+                    l4[u] = __ldcs(reinterpret_cast<const float4 *>(
+                        reinterpret_cast<const float *>(learner) + e0));
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kQuantUnroll; ++u) {
+                const float d[4] = {__fsub_rn(t4[u].x, l4[u].x), __fsub_rn(t4[u].y, l4[u].y),
+                                    __fsub_rn(t4[u].z, l4[u].z), __fsub_rn(t4[u].w, l4[u].w)};
+                float amax = fmaxf(fmaxf(fabsf(d[0]), fabsf(d[1])), fmaxf(fabsf(d[2]), fabsf(d[3])));
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+                const float scale = __fdiv_rn(amax, 7.0f);
+                if (lane == 0) scales[b + u * warps] = scale;
+                unsigned packed = 0;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    float q = scale > 0.0f ? rintf(__fdiv_rn(d[k], scale)) : 0.0f;
+                    q = fminf(fmaxf(q, -7.0f), 7.0f);
+                    packed |= (unsigned)((int)q + 8) << (4 * k);
+                }
+                *reinterpret_cast<unsigned short *>(codes + ((b + u * warps) * kInt4Block + 4ull * lane) / 2) =
+                    (unsigned short)packed;
+            }
+        }
+    }
+    // the remaining blocks (and every block when the inputs are not 16-byte aligned), one at a time
+    for (; b < nblocks; b += warps) {
         const unsigned long long e0 = b * kInt4Block + 4ull * lane;
         float d[4], T[4], th[4];
         float amax = 0.0f;
