@@ -27,9 +27,13 @@ if ROOT not in sys.path:
 METRIC = "merged_params_per_sec"
 UNIT = "params/s"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per merged parameter of the merge
-# kernel, from the ncu capture summarised under profiles/ (None until captured).
-NCU_TRAFFIC_BYTES_PER_PARAM = {"scale500m": 63.04}
+# dram__bytes_read.sum + dram__bytes_write.sum per merged parameter and merge, from the ncu
+# captures summarised under profiles/ (absent: not captured for that merge kind and workload).
+# The radial-directional figure is the sum of its three passes.
+NCU_TRAFFIC_BYTES_PER_PARAM = {
+    ("avg", "scale500m"): 63.04, ("avg", "dense150m"): 27.73, ("avg", "dense1b3"): 41.61,
+    ("avg", "moe4b"): 41.50, ("rda", "scale500m"): 124.8, ("int4", "scale500m"): 26.24,
+}
 
 
 def parse_args():
@@ -485,7 +489,7 @@ def main():
     slowest = sorted(range(len(per_launch_ms)), key=lambda k: -per_launch_ms[k])[:3]
     achieved = alg_bytes / (avg_launch_ms * 1e-3) / 1e9
     peak, peak_kind = hbm_peak()
-    traffic_pp = NCU_TRAFFIC_BYTES_PER_PARAM.get(args.workload) if args.merge == "avg" else None
+    traffic_pp = None if args.out_bf16 else NCU_TRAFFIC_BYTES_PER_PARAM.get((args.merge, args.workload))
     roofline = {
         "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
         "frac": achieved / peak, "peak_source": f"of {peak_kind}",
