@@ -60,7 +60,8 @@ def _run(name, n_windows, merges):
     from paper_2604_21428_b200 import ddmerge as dd
 
     w = synth.workload(name)
-    need = w.algorithmic_bytes() + 8 * w.total_params
+    # resident: the participants' copies, Theta and v (the algorithmic bytes count Theta and v twice)
+    need = w.algorithmic_bytes() - 8 * w.total_params
     free, _ = torch.cuda.mem_get_info()
     if free < need + (4 << 30):
         pytest.skip(f"needs {need >> 30} GiB of device memory, {free >> 30} GiB free")
@@ -129,3 +130,11 @@ def test_scale500m_full_size_sampled():
 
 def test_dense150m_full_size_batched_sampled():
     _run("dense150m", n_windows=4, merges=2)
+
+
+def test_dense1b3_full_size_batched_sampled():
+    _run("dense1b3", n_windows=2, merges=1)
+
+
+def test_moe4b_full_size_batched_sampled():
+    _run("moe4b", n_windows=1, merges=1)
