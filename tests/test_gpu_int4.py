@@ -39,7 +39,8 @@ def _quantize_gpu(dd, ctx, theta, learner, dtype):
     return codes[: (n + 1) // 2], scales[: (n + 127) // 128]
 
 
-@pytest.mark.parametrize("n", [1, 2, 3, 5, 127, 128, 129, 1000, 8192, 100_003])
+# the largest size spans the four-blocks-at-a-time loop, the one-block loop and a ragged last block
+@pytest.mark.parametrize("n", [1, 2, 3, 5, 127, 128, 129, 1000, 8192, 100_003, 4_000_037])
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 def test_quantiser_bit_exact(dd, ctx, n, dtype):
     theta, _, learners = synth.fragment_cpu(n, 1, dtype, 900 + n % 13)
@@ -54,7 +55,8 @@ def test_quantiser_bit_exact(dd, ctx, n, dtype):
     np.testing.assert_array_equal(codes.cpu().numpy(), ref_codes)
 
 
-@pytest.mark.parametrize("n", [5, 8, 1023, 8192 * 2 + 3, 150_001])
+# the largest size gives every thread of the persistent grid more than one 16-element step
+@pytest.mark.parametrize("n", [5, 8, 1023, 8192 * 2 + 3, 150_001, 4_000_037])
 def test_int4_merge(dd, ctx, n):
     M = 6
     tokens, mask, K = [100, 200, 0, 400, 500, 50], 0b111101, 3
