@@ -161,6 +161,23 @@ def test_scale_shape_scaled(dd, ctx):
     assert rec.n_part == 24
 
 
+@pytest.mark.parametrize("dtype,flags", [("bf16", 4), ("f32", 4 | 2)])
+def test_several_tiles_per_cta_element_by_element(dd, ctx, dtype, flags):
+    # 2 x 296 CTAs' worth of 8192-element tiles plus a ragged rest: every CTA of the persistent
+    # grid walks more than one tile and its ring wraps many times; checked on every element
+    n = 2 * 296 * 8192 + 3 * 8192 + 5
+    run_case(dd, ctx, n, 3, dtype, [700, 0, 900], 0b111, 2, seed=77, flags=flags, merges=1)
+
+
+def test_batched_large_fragments_element_by_element(dd, ctx):
+    # CTAs cross fragment boundaries in mid-stream: tile counts that are not multiples of the grid
+    sizes = [3_000_017, 1_500_001, 8, 2_000_003]
+    M = 3
+    tokens = np.array([[5, 7, 9], [1, 0, 4], [3, 3, 3], [9, 8, 0]])
+    _batched_case(dd, ctx, sizes, M, "bf16", tokens, [0b111, 0b101, 0b110, 0b011], 2, seed=21,
+                  flags=dd.DIAG_STATE | dd.DIAG_PER_LEARNER, merges=1)
+
+
 def test_masked_learners_are_never_read(dd, ctx):
     # absent learners: NaN payloads, then null pointers
     run_case(dd, ctx, 20_001, 6, "bf16", [9, 9, 0, 9, 9, 9], 0b101011, 2, seed=8, poison_absent=True)

@@ -79,6 +79,11 @@ def test_rda_sizes(dd, ctx, n, dtype):
     _case(dd, ctx, n, 5, dtype, [100, 200, 0, 400, 500], 0b11101, 2, seed=n % 89)
 
 
+def test_rda_several_tiles_per_cta(dd, ctx):
+    # every pass walks more than one tile per CTA; all elements against the oracle
+    _case(dd, ctx, 2 * 296 * 8192 + 8192 + 3, 3, "bf16", [700, 0, 900], 0b111, 2, seed=31, merges=1)
+
+
 def test_rda_workload_shapes(dd, ctx):
     w = synth.workload("dense150m")
     rec = _case(dd, ctx, 150_003, w.M, "bf16", w.tokens[1].tolist(), w.masks[1], w.K, seed=3,
