@@ -138,3 +138,57 @@ def test_dense1b3_full_size_batched_sampled():
 
 def test_moe4b_full_size_batched_sampled():
     _run("moe4b", n_windows=1, merges=1)
+
+
+def test_scale500m_full_size_int4_sampled():
+    """The compressed merge at the size and participant count bench.py --merge int4 times:
+    every participant's copy is generated, quantised on the GPU and dropped; the oracle
+    quantises and merges the sampled windows (block aligned) from the saved inputs."""
+    from paper_2604_21428_b200 import ddmerge as dd
+
+    w = synth.workload("scale500m")
+    n = w.fragment_sizes[0]
+    free, _ = torch.cuda.mem_get_info()
+    if free < (24 << 30):
+        pytest.skip("needs 24 GiB of device memory")
+    dev = torch.device("cuda", 0)
+    tokens = [int(x) for x in w.tokens[0]]
+    mask, K = w.masks[0], w.K
+    part = [m for m in range(w.M) if (mask >> m) & 1 and tokens[m] > 0]
+    rng = np.random.default_rng(4321)
+    windows = [(lo - lo % 128, lo - lo % 128 + WINDOW) for lo, _ in _windows(n, 4, rng)]
+    g = torch.Generator(device=dev).manual_seed(77)
+    theta = torch.randn(n, generator=g, device=dev) * synth.THETA_STD
+    mom = torch.randn(n, generator=g, device=dev) * 1e-3
+    ctx = dd.Context(0)
+    codes, scales, saved_l = [None] * w.M, [None] * w.M, [None] * w.M
+    for m in part:
+        learner = (theta + torch.randn(n, generator=g, device=dev) * synth.LEARNER_NOISE_STD).to(torch.bfloat16)
+        codes[m] = torch.empty((n + 1) // 2, dtype=torch.uint8, device=dev)
+        scales[m] = torch.empty((n + 127) // 128, dtype=torch.float32, device=dev)
+        ctx.quantize_outer_gradient_int4(theta, learner, codes[m], scales[m])
+        saved_l[m] = [_to_host_learner(learner[lo:hi]) for lo, hi in windows]
+        del learner
+    saved = [(theta[lo:hi].cpu().numpy().copy(), mom[lo:hi].cpu().numpy().copy()) for lo, hi in windows]
+    records = dd.new_records(1, device=dev)
+    ctx.merge_fragment_int4(theta, mom, codes, scales, tokens, mask, K, ETA, MU, n=n,
+                            flags=dd.DIAG_STATE, record=records)
+    torch.cuda.synchronize()
+    rec = dd.read_records(records)[0]
+    for k, (lo, hi) in enumerate(windows):
+        t0, v0 = saved[k]
+        q = [oracle.quantize_int4(t0, saved_l[m][k]) if m in part else None for m in range(w.M)]
+        # the quantiser is bit-exact: codes and scales of the window as the GPU wrote them
+        for m in part:
+            np.testing.assert_array_equal(codes[m][lo // 2:hi // 2].cpu().numpy(), q[m][0])
+            np.testing.assert_array_equal(scales[m][lo // 128:hi // 128].cpu().numpy().view(np.uint32),
+                                          q[m][1].view(np.uint32))
+        ref = oracle.merge_fragment_int4(t0, v0, [None if x is None else x[0] for x in q],
+                                         [None if x is None else x[1] for x in q], tokens, mask, K, ETA, MU)
+        assert (rec.status, rec.n_part, rec.idx) == (ref.status, ref.n_part, ref.idx)
+        assert rec.w_hat == [float(np.float32(x)) for x in ref.w_hat]
+        assert floor_rel_err(theta[lo:hi].cpu().numpy(), t0) <= TOL_STATE
+        assert floor_rel_err(mom[lo:hi].cpu().numpy(), v0) <= TOL_STATE
+    assert abs(rec.theta_sq - _sq(theta)) <= TOL_NORM * rec.theta_sq
+    assert abs(rec.mom_sq - _sq(mom)) <= TOL_NORM * rec.mom_sq
+    ctx.close()
