@@ -192,3 +192,70 @@ def test_scale500m_full_size_int4_sampled():
     assert abs(rec.theta_sq - _sq(theta)) <= TOL_NORM * rec.theta_sq
     assert abs(rec.mom_sq - _sq(mom)) <= TOL_NORM * rec.mom_sq
     ctx.close()
+
+
+def test_scale500m_full_size_rda_properties():
+    """The radial-directional merge at bench size.  Its result depends on whole-fragment norms,
+    so the oracle cannot take a window; what is checked holds at any size: per-participant
+    norms against float64 device reductions, ||Delta|| = sum_m w_m ||Delta_m|| (the defining
+    property of the merge), and on sampled windows v' - mu v = Delta = c u, u the weighted mean
+    of unit directions and c the factor that whole-fragment float64 reductions fix."""
+    from paper_2604_21428_b200 import ddmerge as dd
+
+    w = synth.workload("scale500m")
+    n = w.fragment_sizes[0]
+    free, _ = torch.cuda.mem_get_info()
+    if free < (36 << 30):
+        pytest.skip("needs 36 GiB of device memory")
+    dev = torch.device("cuda", 0)
+    tokens = [int(x) for x in w.tokens[0]]
+    mask, K = w.masks[0], w.K
+    part = [m for m in range(w.M) if (mask >> m) & 1 and tokens[m] > 0]
+    theta = torch.empty(n, dtype=torch.float32, device=dev)
+    mom = torch.empty(n, dtype=torch.float32, device=dev)
+    learners = [torch.empty(n, dtype=torch.bfloat16, device=dev) if m in part else None for m in range(w.M)]
+    synth.fill_fragment_gpu(theta, mom, learners, seed=99)
+    mom.normal_(0.0, 1e-3, generator=torch.Generator(device=dev).manual_seed(5))
+    chunk = 1 << 25
+    norms = []
+    for m in part:
+        acc = 0.0
+        for lo in range(0, n, chunk):
+            d = theta[lo:lo + chunk].double() - learners[m][lo:lo + chunk].double()
+            acc += float((d * d).sum())
+        norms.append(acc ** 0.5)
+    st, idx = oracle.participants(mask, tokens, K)
+    _, w_hat, _ = oracle.weights(tokens, None, idx)
+    wf = [float(np.float32(x)) for x in w_hat]
+    u_sq = 0.0                                           # ||sum_j w_j Delta_j / ||Delta_j|| ||^2
+    for lo in range(0, n, chunk):
+        T = theta[lo:lo + chunk].double()
+        u = torch.zeros_like(T)
+        for j, m in enumerate(part):
+            u += (wf[j] / norms[j]) * (T - learners[m][lo:lo + chunk].double())
+        u_sq += float((u * u).sum())
+    radial = sum(wf[j] * norms[j] for j in range(len(part)))
+    c_expected = radial / u_sq ** 0.5
+    rng = np.random.default_rng(99)
+    windows = _windows(n, 3, rng)
+    saved = [(theta[lo:hi].double().cpu().numpy(), mom[lo:hi].double().cpu().numpy(),
+              [learners[m][lo:hi].double().cpu().numpy() for m in part]) for lo, hi in windows]
+    ctx = dd.Context(0)
+    records = dd.new_records(1, device=dev)
+    ctx.merge_fragment_rda(theta, mom, learners, tokens, mask, K, ETA, MU, n=n, learner_dtype=dd.BF16,
+                           flags=dd.DIAG_STATE, record=records)
+    torch.cuda.synchronize()
+    rec = dd.read_records(records)[0]
+    assert (rec.status, rec.n_part, rec.idx) == (st, len(idx), list(idx))
+    assert rec.w_hat == wf
+    for j in range(len(part)):
+        assert abs(rec.delta_m_sq[j] - norms[j] ** 2) <= TOL_NORM * norms[j] ** 2
+    assert abs(rec.delta_sq ** 0.5 - radial) <= 1e-5 * radial
+    for (lo, hi), (t0, v0, ls) in zip(windows, saved):
+        u = sum(wf[j] / norms[j] * (t0 - ls[j]) for j in range(len(part)))
+        delta = mom[lo:hi].double().cpu().numpy() - MU * v0           # v' = mu v + Delta
+        # Delta = c u with one factor for the whole fragment, fixed by the norms
+        assert floor_rel_err(delta, c_expected * u) <= 1e-4
+    assert abs(rec.theta_sq - _sq(theta)) <= TOL_NORM * rec.theta_sq
+    assert abs(rec.mom_sq - _sq(mom)) <= TOL_NORM * rec.mom_sq
+    ctx.close()
