@@ -55,18 +55,34 @@ quantize_int4_kernel(const float *__restrict__ theta, const void *__restrict__ l
             for (int u = 0; u < kQuantUnroll; ++u) {
                 const float d[4] = {__fsub_rn(t4[u].x, l4[u].x), __fsub_rn(t4[u].y, l4[u].y),
                                     __fsub_rn(t4[u].z, l4[u].z), __fsub_rn(t4[u].w, l4[u].w)};
+                // |d| is never NaN here (fmaxf drops it), so the maximum of the bit patterns is the maximum
                 float amax = fmaxf(fmaxf(fabsf(d[0]), fabsf(d[1])), fmaxf(fabsf(d[2]), fabsf(d[3])));
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+                amax = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(amax)));
                 const float scale = __fdiv_rn(amax, 7.0f);
                 if (lane == 0) scales[b + u * warps] = scale;
-                unsigned packed = 0;
+                // round(d / scale) without a division per element: q0 = d * (1 / scale) is within
+                // 1.1e-6 of the correctly rounded quotient (|quotient| <= 7), so both round to the same
+                // integer unless q0 is that close to a half-integer; those elements, and blocks whose
+                // scale is so small or large that the reciprocal leaves the normal range, take the
+                // exact division.  The codes equal rint(fdiv(d, scale)) in every case.
+                const bool fast = scale >= 1e-30f && scale <= 1e30f;
+                const float rcp = __frcp_rn(scale);
+                float q[4];
+                bool exact = !fast;
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    float q = scale > 0.0f ? rintf(__fdiv_rn(d[k], scale)) : 0.0f;
-                    q = fminf(fmaxf(q, -7.0f), 7.0f);
-                    packed |= (unsigned)((int)q + 8) << (4 * k);
+                    const float q0 = d[k] * rcp;
+                    q[k] = rintf(q0);
+                    exact |= !(fabsf(q0 - q[k]) <= 0.5f - 4e-6f);
                 }
+                if (exact) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) q[k] = scale > 0.0f ? rintf(__fdiv_rn(d[k], scale)) : 0.0f;
+                }
+                unsigned packed = 0;
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    packed |= (unsigned)((int)fminf(fmaxf(q[k], -7.0f), 7.0f) + 8) << (4 * k);
                 *reinterpret_cast<unsigned short *>(codes + ((b + u * warps) * kInt4Block + 4ull * lane) / 2) =
                     (unsigned short)packed;
             }

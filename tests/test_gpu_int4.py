@@ -55,6 +55,34 @@ def test_quantiser_bit_exact(dd, ctx, n, dtype):
     np.testing.assert_array_equal(codes.cpu().numpy(), ref_codes)
 
 
+def test_quantiser_near_ties_and_extreme_scales(dd, ctx):
+    """Outer gradients placed on, and one to three ulps beside, the half-integer multiples of
+    the block scale -- where rint(d / scale) decides between two codes -- and blocks whose
+    scale is tiny, huge or zero.  Codes must still equal the oracle's bit for bit."""
+    rng = np.random.default_rng(2024)
+    nblocks = 40_000                                    # enough for the four-blocks-at-a-time loop
+    n = nblocks * 128
+    sc = np.exp(rng.uniform(np.log(1e-6), np.log(1e3), size=nblocks)).astype(np.float32)
+    sc[::7] = 1.0                                       # exact ties: d = k + 1/2
+    sc[1::97] = np.float32(1e-36)
+    sc[2::97] = np.float32(3e33)
+    sc[3::97] = np.float32(1e-41)                       # subnormal scale
+    k = rng.integers(-7, 7, size=(nblocks, 128)).astype(np.float32)
+    ulps = rng.integers(-3, 4, size=(nblocks, 128)).astype(np.float32)
+    d = (k + np.float32(0.5)) * sc[:, None]
+    d = (d * (np.float32(1.0) + ulps * np.float32(2.0 ** -23))).astype(np.float32)
+    d[:, 0] = np.float32(7.0) * sc                      # fixes the block maximum, hence the scale
+    d[5::97] = 0.0                                      # all-zero blocks
+    learner = (-d).reshape(-1).astype(np.float32)       # Theta = 0: Theta - theta = d exactly
+    theta = np.zeros(n, dtype=np.float32)
+    ref_codes, ref_scales = oracle.quantize_int4(theta, learner)
+    codes, scales = _quantize_gpu(dd, ctx, theta, learner, "f32")
+    np.testing.assert_array_equal(scales.cpu().numpy().view(np.uint32), ref_scales.view(np.uint32))
+    np.testing.assert_array_equal(codes.cpu().numpy(), ref_codes)
+    # the stress is real: both neighbouring codes occur among elements built from the same k
+    assert len(np.unique(ref_codes)) > 100
+
+
 # the largest size gives every thread of the persistent grid more than one 16-element step
 @pytest.mark.parametrize("n", [5, 8, 1023, 8192 * 2 + 3, 150_001, 4_000_037])
 def test_int4_merge(dd, ctx, n):
