@@ -1,6 +1,7 @@
 // The streaming part of the fused merge: operands are staged through shared
 // memory by bulk asynchronous copies (cp.async.bulk: the TMA engine, no tensor
-// map, no multicast).  A warp owns a private ring of kTmaStages slots of 2 KB.  Its lane 0
+// map, every copy addressed to this CTA alone).  A warp owns a private ring of
+// kTmaStages slots of 2 KB.  Its lane 0
 // asks the copy engine for the next 2 KB piece -- 1024 bf16 elements of one
 // learner copy, or 512 floats of Theta / v -- up to kTmaStages-1 pieces ahead of
 // the piece the warp is consuming, each piece signalling its own mbarrier.  The
