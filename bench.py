@@ -372,7 +372,7 @@ def main():
                                                  int4_scales[m], n=n0, learner_dtype=ldtype)
         torch.cuda.synchronize()
 
-    def step():
+    def step(stream=stream):
         if args.merge == "int4":
             f = frags[0]
             ctx.merge_fragment_int4(f["global_"], f["momentum"], int4_codes, int4_scales, f["tokens"],
@@ -471,6 +471,31 @@ def main():
         cold_ms = {"median": statistics.median(cold), "min": min(cold), "max": max(cold)}
         del flush
 
+    # A single small fragment is launch-bound from Python (the host needs longer to issue a
+    # merge than the GPU to run it): the same calls captured once into a CUDA graph and
+    # replayed give the device-bound time per merge.  The library call is capture-safe
+    # (one kernel launch, no allocation or synchronisation once the workspace exists).
+    graph_ms = None
+    if cold_ms is not None and w.P == 1 and args.merge == "avg":
+        side = torch.cuda.Stream(device=device)
+        graph = torch.cuda.CUDAGraph()
+        reps = 50
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                for _ in range(reps):
+                    step(side)
+        torch.cuda.synchronize()
+        times = []
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(8):
+            e0.record()
+            graph.replay()
+            e1.record()
+            e1.synchronize()
+            times.append(e0.elapsed_time(e1) / reps)
+        graph_ms = {"median": statistics.median(times[3:]), "min": min(times[3:]), "merges_per_graph": reps}
+        del graph
+
     params_per_step = w.total_params
     value = ddist.whole_job_rate(job_params, args.steps, 1, max_ms)
     alg_bytes = w.algorithmic_bytes(out_bf16=args.out_bf16)
@@ -501,6 +526,8 @@ def main():
                       "slowest_steps": slowest},
         "frac_of_nominal_8TBs": achieved / 8000.0,
     }
+    if graph_ms is not None:
+        roofline["ms_per_merge_cuda_graph_replay"] = graph_ms
     if cold_ms is not None:
         roofline["kernel_ms_l2_flushed"] = cold_ms
         roofline["achieved_l2_flushed"] = alg_bytes / (cold_ms["median"] * 1e-3) / 1e9
