@@ -130,6 +130,11 @@ int dd_destroy(dd_ctx *ctx);
  *   out_bf16          [device] optional bf16[n]: round-to-nearest-even copy of
  *                     Theta' (the payload broadcast back to the learners)
  *   record            [device] optional; without it no diagnostics are computed
+ *
+ * The call enqueues one kernel on cuda_stream and returns.  The first call that
+ * passes a record allocates the context's workspace; from then on the call
+ * neither allocates nor synchronises, so it may be recorded into a CUDA graph by
+ * stream capture (host arrays are consumed before it returns).
  */
 int dd_merge_fragment(dd_ctx *ctx, float *global, float *momentum,
                       const void *const *learner_ptrs, int M, dd_dtype learner_dtype,

@@ -567,3 +567,33 @@ def test_random_shape_sweep(dd, ctx):
         run_case(dd, ctx, n, M, dtype, tokens, mask, K, seed=1000 + trial, steps=steps, flags=flags,
                  merges=1, use_out=bool(rng.random() < 0.5), null_absent=bool(rng.random() < 0.5),
                  shift=int(rng.choice([0, 4])))
+
+
+def test_cuda_graph_capture_and_replay(dd, ctx):
+    """The single-fragment call is capture-safe once the context has its workspace: captured into a
+    CUDA graph and replayed, it gives the oracle's result, replay after replay."""
+    n, M = 40_003, 4
+    tokens, mask, K = [5, 0, 7, 9], 0b1101, 2
+    theta, v, learners = synth.fragment_cpu(n, M, "bf16", 321)
+    t_dev, v_dev = torch.from_numpy(theta).cuda(), torch.from_numpy(v).cuda()
+    l_dev = [to_torch_learner(a, "cuda") for a in learners]
+    rec_buf = dd.new_records(1)
+    ctx.merge_fragment(t_dev, v_dev, l_dev, tokens, mask, K, ETA, MU, flags=dd.DIAG_STATE, record=rec_buf)
+    torch.cuda.synchronize()                                 # workspace exists from here on
+    ref = oracle.merge_fragment(theta, v, learners, tokens, mask, K, ETA, MU)
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            ctx.merge_fragment(t_dev, v_dev, l_dev, tokens, mask, K, ETA, MU, flags=dd.DIAG_STATE,
+                               record=rec_buf, stream=side)
+    for _ in range(3):
+        t_dev.copy_(torch.from_numpy(synth.fragment_cpu(n, M, "bf16", 321)[0]))
+        v_dev.zero_()
+        rec_buf.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        got = dd.read_records(rec_buf)[0]
+        assert_record_matches(got, ref, diag_state=True, per_learner=False)
+        assert floor_rel_err(t_dev.cpu().numpy(), theta) <= TOL_STATE
+        assert floor_rel_err(v_dev.cpu().numpy(), v) <= TOL_STATE
