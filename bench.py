@@ -372,6 +372,10 @@ def main():
                                                  int4_scales[m], n=n0, learner_dtype=ldtype)
         torch.cuda.synchronize()
 
+    # the same buffers are merged every step: marshal their addresses and counts once
+    packed_ptrs = dd.pack_pointers(frags[0]["learners"]) if w.P == 1 else None
+    packed_tokens = dd.pack_u64(frags[0]["tokens"]) if w.P == 1 else None
+
     def step(stream=stream):
         if args.merge == "int4":
             f = frags[0]
@@ -383,7 +387,7 @@ def main():
                                             records=records, stream=stream)
         elif w.P == 1:
             f = frags[0]
-            ctx.merge_fragment(f["global_"], f["momentum"], f["learners"], f["tokens"],
+            ctx.merge_fragment(f["global_"], f["momentum"], packed_ptrs, packed_tokens,
                                f["quorum_mask"], f["K"], eta, mu, n=f["n"], learner_dtype=ldtype,
                                flags=flags, out_bf16=f["out_bf16"], record=records, stream=stream)
         else:

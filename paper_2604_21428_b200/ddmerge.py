@@ -179,7 +179,25 @@ def _ptr(x) -> int | None:
 
 
 def _u64_array(values):
+    if isinstance(values, ctypes.Array):
+        return values
     return (ctypes.c_uint64 * len(values))(*[int(v) for v in values])
+
+
+def pack_pointers(tensors):
+    """The addresses of ``tensors`` (tensors / ints / None) as a C array.  Every entry point that
+    takes a list of learner buffers also takes this array, which saves the per-call marshalling
+    when the same buffers are merged again and again (pass ``learner_dtype`` explicitly then)."""
+    return (ctypes.c_void_p * len(tensors))(*[_ptr(t) for t in tensors])
+
+
+def pack_u64(values):
+    """Token or step counts as a C array of uint64 (accepted wherever a list of counts is)."""
+    return (ctypes.c_uint64 * len(values))(*[int(v) for v in values])
+
+
+def _pointer_array(learners):
+    return learners if isinstance(learners, ctypes.Array) else pack_pointers(learners)
 
 
 def _stream_handle(stream) -> int | None:
@@ -256,7 +274,7 @@ class Context:
             n = int(global_.numel())
         if learner_dtype is None:
             learner_dtype = _infer_dtype(learners)
-        ptrs = (ctypes.c_void_p * M)(*[_ptr(t) for t in learners])
+        ptrs = _pointer_array(learners)
         self._check(lib.dd_merge_fragment(
             self._h, _ptr(global_), _ptr(momentum), ptrs, M, learner_dtype, _u64_array(tokens),
             None if steps is None else _u64_array(steps),
@@ -274,7 +292,7 @@ class Context:
             n = int(global_.numel())
         if learner_dtype is None:
             learner_dtype = _infer_dtype(learners)
-        ptrs = (ctypes.c_void_p * M)(*[_ptr(t) for t in learners])
+        ptrs = _pointer_array(learners)
         self._check(lib.dd_merge_fragment_rda(
             self._h, _ptr(global_), _ptr(momentum), ptrs, M, learner_dtype, _u64_array(tokens),
             None if steps is None else _u64_array(steps),
@@ -306,7 +324,7 @@ class Context:
             n = int(global_.numel())
         if learner_dtype is None:
             learner_dtype = _infer_dtype(learners)
-        ptrs = (ctypes.c_void_p * M)(*[_ptr(t) for t in learners])
+        ptrs = _pointer_array(learners)
         self._check(lib.dd_broadcast_fragment(
             self._h, _ptr(global_), ptrs, M, learner_dtype,
             ctypes.c_uint64(apply_mask & (2**64 - 1)), ctypes.c_float(alpha), ctypes.c_size_t(n),
@@ -353,7 +371,7 @@ class Context:
             n = int(global_.numel())
         if learner_dtype is None:
             learner_dtype = _infer_dtype(learners)
-        ptrs = (ctypes.c_void_p * M)(*[_ptr(t) for t in learners])
+        ptrs = _pointer_array(learners)
         rec = CRecord()
         self._check(lib.dd_merge_fragment_host(
             self._h, _ptr(global_), _ptr(momentum), ptrs, M, learner_dtype, _u64_array(tokens),
@@ -420,6 +438,8 @@ def merge_fragments_batched_noalloc(fragments, M: int, learner_dtype: int, outer
 
 def _infer_dtype(learners) -> int:
     import torch
+    if isinstance(learners, ctypes.Array):
+        raise ValueError("learner_dtype must be given with a packed pointer array")
     for t in learners:
         if t is not None and not isinstance(t, int):
             return BF16 if t.dtype == torch.bfloat16 else F32

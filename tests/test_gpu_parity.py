@@ -597,3 +597,27 @@ def test_cuda_graph_capture_and_replay(dd, ctx):
         assert_record_matches(got, ref, diag_state=True, per_learner=False)
         assert floor_rel_err(t_dev.cpu().numpy(), theta) <= TOL_STATE
         assert floor_rel_err(v_dev.cpu().numpy(), v) <= TOL_STATE
+
+
+def test_packed_pointer_and_count_arrays(dd, ctx):
+    """Pre-marshalled learner addresses and token counts give the same merge as lists."""
+    n, M = 20_001, 5
+    tokens, mask, K = [3, 0, 8, 1, 6], 0b11101, 2
+    theta, v, learners = synth.fragment_cpu(n, M, "bf16", 55)
+    ref = oracle.merge_fragment(theta.copy(), v.copy(), learners, tokens, mask, K, ETA, MU)
+    l_dev = [to_torch_learner(a, "cuda") for a in learners]
+    results = []
+    for packed in (False, True):
+        t_dev, v_dev = torch.from_numpy(theta).cuda(), torch.from_numpy(v).cuda()
+        rec_buf = dd.new_records(1)
+        ls = dd.pack_pointers(l_dev) if packed else l_dev
+        tk = dd.pack_u64(tokens) if packed else tokens
+        ctx.merge_fragment(t_dev, v_dev, ls, tk, mask, K, ETA, MU, n=n, learner_dtype=dd.BF16,
+                           flags=dd.DIAG_STATE, record=rec_buf)
+        torch.cuda.synchronize()
+        results.append((t_dev.cpu(), v_dev.cpu(), dd.read_records(rec_buf)[0]))
+    assert torch.equal(results[0][0], results[1][0]) and torch.equal(results[0][1], results[1][1])
+    assert results[0][2].idx == results[1][2].idx == ref.idx
+    with pytest.raises(ValueError):
+        ctx.merge_fragment(results[0][0].cuda(), results[0][1].cuda(), dd.pack_pointers(l_dev), tokens,
+                           mask, K, ETA, MU, n=n)
