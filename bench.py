@@ -52,6 +52,8 @@ def parse_args():
     ap.add_argument("--cpu-sample", type=int, default=1 << 27,
                     help="elements of the workload the CPU oracle is timed on")
     ap.add_argument("--out-bf16", action="store_true", help="also write the bf16 broadcast copy")
+    ap.add_argument("--unfused-push", action="store_true",
+                    help="tape24: separate merge and broadcast launches instead of the fused push")
     ap.add_argument("--merge", choices=["avg", "rda", "int4"], default="avg",
                     help="weighted direct averaging (the headline path), radial-directional, or "
                          "direct averaging of int4-compressed outer gradients")
@@ -268,7 +270,8 @@ def run_replay(args):
             learners[m][p] = copies[m]
     ctx = dd.Context(0)
     syncer = Syncer(ctx, theta, mom, H=H, offsets=offsets, K=K, outer_lr=synth.OUTER_LR,
-                    outer_mu=synth.OUTER_MU, learner_dtype=dd.BF16, flags=dd.DIAG_STATE)
+                    outer_mu=synth.OUTER_MU, learner_dtype=dd.BF16, flags=dd.DIAG_STATE,
+                    fused_push=not args.unfused_push)
     stream = torch.cuda.current_stream()
     entries = [TapeEntry(arrival_s=e["arrival_s"], tokens=e["tokens"], steps=e["steps"]) for e in tape]
     for t in range(args.warmup):
@@ -286,10 +289,13 @@ def run_replay(args):
             s_p = sum(1 for m in range(M) if (res.mask >> m) & 1 and entries[t].tokens[p][m] > 0)
             if s_p >= max(K, 1):
                 merged_params += sizes[p]
-                merged_bytes += sizes[p] * (2 * s_p + 16) + sizes[p] * (4 + 2 * alive)
-                launches += 2
-            else:
-                launches += 1
+                # merge (read s copies, Theta, v; write Theta', v') + push (write the alive copies);
+                # the unfused form reads Theta' once more in its broadcast launch
+                merged_bytes += sizes[p] * (2 * s_p + 16) + sizes[p] * (2 * alive)
+                if not syncer.fused_push:
+                    merged_bytes += sizes[p] * 4
+                    launches += 1
+            launches += 1
     ev1.record(stream)
     torch.cuda.synchronize()
     sampler.stop()
@@ -309,7 +315,8 @@ def run_replay(args):
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": f"of {peak_kind}", "traffic": None,
                      "algorithmic_bytes": merged_bytes,
-                     "note": "merge + broadcast launches of the syncer loop, host work included"},
+                     "note": ("merge and push fused in one launch per syncer step" if syncer.fused_push else
+                              "merge + broadcast launches of the syncer loop") + ", host work included"},
         "e2e": None, "cpu_baseline": None,
     }
     print(json.dumps(line), flush=True)

@@ -168,6 +168,33 @@ int dd_merge_fragments_batched(dd_ctx *ctx, const dd_fragment_desc *descs, int P
                                void *cuda_stream);
 
 /*
+ * Merge and push in one pass.  Algorithm 2 ends a fragment's synchronisation by sending
+ * the new global fragment to every learner, which overwrites its copy (alpha = 0 in the
+ * learner-side mixing of the Appendix).  When the learner copies the syncer reads are also
+ * the buffers the learners resume from, these calls do both: every learner m with bit m of
+ * push_mask set has its copy replaced by Theta' rounded to learner_dtype (round to
+ * nearest even for bf16), in the same kernel that merges, so Theta' is not read back a
+ * second time.  A learner may be pushed to without being merged (it was late or down) and
+ * merged without being pushed to.  If the quorum is not met nothing is pushed.
+ *
+ *   learner_ptrs[m] of a pushed learner is written: it must be non-NULL, 16-byte aligned
+ *   and must not overlap global, momentum, out_bf16, or the copy of another learner that
+ *   is read or pushed (DD_ERR_ALIAS).  Bits of push_mask at or above M are ignored.
+ * Everything else is as in dd_merge_fragment / dd_merge_fragments_batched;
+ * push_masks is a host array of P masks.
+ */
+int dd_merge_fragment_push(dd_ctx *ctx, float *global, float *momentum,
+                           void *const *learner_ptrs, int M, dd_dtype learner_dtype,
+                           const uint64_t *tokens, const uint64_t *steps,
+                           uint64_t quorum_mask, int K, float outer_lr, float outer_mu,
+                           uint32_t flags, size_t n, uint64_t push_mask, void *out_bf16,
+                           dd_merge_record *record, void *cuda_stream);
+int dd_merge_fragments_batched_push(dd_ctx *ctx, const dd_fragment_desc *descs,
+                                    const uint64_t *push_masks, int P, int M,
+                                    dd_dtype learner_dtype, float outer_lr, float outer_mu,
+                                    uint32_t flags, dd_merge_record *records, void *cuda_stream);
+
+/*
  * Radial-directional averaging (RDA, Appendix "Merging methods"): the merged outer
  * gradient keeps the weighted mean NORM of the per-learner outer gradients
  * D_m = Theta - theta_m and takes the direction of their weighted mean direction,

@@ -31,6 +31,8 @@ struct alignas(16) DevFrag {
     float *scratch;                      // radial-directional merge: n floats for the mean direction
     int kind;                            // DD_MERGE_AVG or DD_MERGE_RDA
     int pad_;
+    unsigned long long push_mask;        // learners whose copy is overwritten with Theta' (fused push)
+    unsigned long long pad2_;
     const void *ptrs[DD_MAX_LEARNERS];
     unsigned long long tokens[DD_MAX_LEARNERS];
     unsigned long long steps[DD_MAX_LEARNERS];

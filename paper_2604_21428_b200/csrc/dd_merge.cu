@@ -128,6 +128,28 @@ static size_t learner_bytes_of(dd_dtype dtype, uint64_t n)
     return (dtype == DD_BF16 ? 2u : 4u) * (size_t)n;
 }
 
+// Fused push: marks the learners whose copy the merge overwrites with Theta'.  Their
+// pointers are written through, so each must be a valid, aligned buffer of its own.
+static int set_push(DevFrag &d, const void *const *learner_ptrs, uint64_t push_mask, int M, uint64_t n,
+                    size_t lb)
+{
+    const uint64_t pm = M >= 64 ? push_mask : (push_mask & ((1ull << M) - 1ull));
+    for (int m = 0; m < M && n > 0; ++m) {
+        if (!((pm >> m) & 1ull)) continue;
+        const void *p = learner_ptrs[m];
+        if (!p) return DD_ERR_INVALID_ARG;
+        if (misaligned(p)) return DD_ERR_ALIGNMENT;
+        if (overlaps(p, lb, d.theta, 4 * n) || overlaps(p, lb, d.mom, 4 * n) || overlaps(p, lb, d.out_bf16, 2 * n))
+            return DD_ERR_ALIAS;
+        for (int k = 0; k < m; ++k)        // two pushed (or read) copies sharing memory would race
+            if (learner_ptrs[k] && (((pm >> k) & 1ull) || (((d.mask >> k) & 1ull) && d.tokens[k] > 0)) &&
+                overlaps(p, lb, learner_ptrs[k], lb))
+                return DD_ERR_ALIAS;
+    }
+    d.push_mask = pm;
+    return DD_OK;
+}
+
 static unsigned long long tiles_of(uint64_t n)
 {
     const unsigned long long t = (n + kTileElems - 1) / kTileElems;
@@ -266,12 +288,12 @@ extern "C" int dd_destroy(dd_ctx *ctx)
     return DD_OK;
 }
 
-extern "C" int dd_merge_fragment(dd_ctx *ctx, float *global, float *momentum,
-                                 const void *const *learner_ptrs, int M, dd_dtype learner_dtype,
-                                 const uint64_t *tokens, const uint64_t *steps,
-                                 uint64_t quorum_mask, int K, float outer_lr, float outer_mu,
-                                 uint32_t flags, size_t n, void *out_bf16,
-                                 dd_merge_record *record, void *cuda_stream)
+static int merge_fragment_impl(dd_ctx *ctx, float *global, float *momentum,
+                               const void *const *learner_ptrs, int M, dd_dtype learner_dtype,
+                               const uint64_t *tokens, const uint64_t *steps,
+                               uint64_t quorum_mask, int K, float outer_lr, float outer_mu,
+                               uint32_t flags, size_t n, uint64_t push_mask, void *out_bf16,
+                               dd_merge_record *record, void *cuda_stream)
 {
     int rc = check_common(ctx, M, learner_dtype, outer_lr, outer_mu, flags);
     if (rc != DD_OK) return rc;
@@ -279,6 +301,10 @@ extern "C" int dd_merge_fragment(dd_ctx *ctx, float *global, float *momentum,
     rc = fill_fragment(frag, global, momentum, out_bf16, learner_ptrs, tokens, steps, quorum_mask, K,
                        n, M, learner_bytes_of(learner_dtype, n));
     if (rc != DD_OK) return rc;
+    if (push_mask) {
+        rc = set_push(frag, learner_ptrs, push_mask, M, n, learner_bytes_of(learner_dtype, n));
+        if (rc != DD_OK) return rc;
+    }
     if (n == 0 && record == nullptr) return DD_OK;
     frag.tile_begin = 0;
     frag.tile_end = tiles_of(n);
@@ -308,10 +334,33 @@ extern "C" int dd_merge_fragment(dd_ctx *ctx, float *global, float *momentum,
     return DD_OK;
 }
 
-extern "C" int dd_merge_fragments_batched(dd_ctx *ctx, const dd_fragment_desc *descs, int P, int M,
-                                          dd_dtype learner_dtype, float outer_lr, float outer_mu,
-                                          uint32_t flags, dd_merge_record *records,
-                                          void *cuda_stream)
+extern "C" int dd_merge_fragment(dd_ctx *ctx, float *global, float *momentum,
+                                 const void *const *learner_ptrs, int M, dd_dtype learner_dtype,
+                                 const uint64_t *tokens, const uint64_t *steps,
+                                 uint64_t quorum_mask, int K, float outer_lr, float outer_mu,
+                                 uint32_t flags, size_t n, void *out_bf16,
+                                 dd_merge_record *record, void *cuda_stream)
+{
+    return merge_fragment_impl(ctx, global, momentum, learner_ptrs, M, learner_dtype, tokens, steps,
+                               quorum_mask, K, outer_lr, outer_mu, flags, n, 0, out_bf16, record,
+                               cuda_stream);
+}
+
+extern "C" int dd_merge_fragment_push(dd_ctx *ctx, float *global, float *momentum,
+                                      void *const *learner_ptrs, int M, dd_dtype learner_dtype,
+                                      const uint64_t *tokens, const uint64_t *steps,
+                                      uint64_t quorum_mask, int K, float outer_lr, float outer_mu,
+                                      uint32_t flags, size_t n, uint64_t push_mask, void *out_bf16,
+                                      dd_merge_record *record, void *cuda_stream)
+{
+    return merge_fragment_impl(ctx, global, momentum, learner_ptrs, M, learner_dtype, tokens, steps,
+                               quorum_mask, K, outer_lr, outer_mu, flags, n, push_mask, out_bf16, record,
+                               cuda_stream);
+}
+
+static int merge_batched_impl(dd_ctx *ctx, const dd_fragment_desc *descs, const uint64_t *push_masks,
+                              int P, int M, dd_dtype learner_dtype, float outer_lr, float outer_mu,
+                              uint32_t flags, dd_merge_record *records, void *cuda_stream)
 {
     int rc = check_common(ctx, M, learner_dtype, outer_lr, outer_mu, flags);
     if (rc != DD_OK) return rc;
@@ -333,6 +382,11 @@ extern "C" int dd_merge_fragments_batched(dd_ctx *ctx, const dd_fragment_desc *d
         rc = fill_fragment(slot.host[p], d.global, d.momentum, d.out_bf16, d.learner_ptrs, d.tokens,
                            d.steps, d.quorum_mask, d.K, d.n, M, learner_bytes_of(learner_dtype, d.n));
         if (rc != DD_OK) return rc;
+        if (push_masks && push_masks[p]) {
+            rc = set_push(slot.host[p], d.learner_ptrs, push_masks[p], M, d.n,
+                          learner_bytes_of(learner_dtype, d.n));
+            if (rc != DD_OK) return rc;
+        }
         slot.host[p].tile_begin = tile;
         tile += tiles_of(d.n);
         slot.host[p].tile_end = tile;
@@ -365,6 +419,26 @@ extern "C" int dd_merge_fragments_batched(dd_ctx *ctx, const dd_fragment_desc *d
     slot.used = true;
     ctx->next_slot = (ctx->next_slot + 1) % kSlots;
     return DD_OK;
+}
+
+extern "C" int dd_merge_fragments_batched(dd_ctx *ctx, const dd_fragment_desc *descs, int P, int M,
+                                          dd_dtype learner_dtype, float outer_lr, float outer_mu,
+                                          uint32_t flags, dd_merge_record *records,
+                                          void *cuda_stream)
+{
+    return merge_batched_impl(ctx, descs, nullptr, P, M, learner_dtype, outer_lr, outer_mu, flags, records,
+                              cuda_stream);
+}
+
+extern "C" int dd_merge_fragments_batched_push(dd_ctx *ctx, const dd_fragment_desc *descs,
+                                               const uint64_t *push_masks, int P, int M,
+                                               dd_dtype learner_dtype, float outer_lr, float outer_mu,
+                                               uint32_t flags, dd_merge_record *records,
+                                               void *cuda_stream)
+{
+    if (P > 0 && !push_masks) return DD_ERR_INVALID_ARG;
+    return merge_batched_impl(ctx, descs, push_masks, P, M, learner_dtype, outer_lr, outer_mu, flags,
+                              records, cuda_stream);
 }
 
 namespace ddm {

@@ -40,6 +40,8 @@ struct Smem {
     int kind;                            // DD_MERGE_AVG / DD_MERGE_RDA of this fragment
     float *scratch;                      // RDA: the mean direction u
     float cscale;                        // RDA apply: Delta = cscale * u
+    void *push[DD_MAX_LEARNERS];         // copies that receive Theta' (compacted)
+    int n_push;
     double red[kWarps][kNumScalarDiag];  // per-warp ||Delta||^2, ||Theta'||^2, ||v'||^2 of this fragment
     double dm[kWarps][DD_MAX_LEARNERS];  // per-warp per-participant ||Theta-theta_m||^2
 };
@@ -164,7 +166,15 @@ __device__ __forceinline__ void load_header(const DevFrag *f, int p, unsigned lo
                                      : (!(W > 0.0) ? DD_STATUS_ZERO_WEIGHT : DD_STATUS_OK);
     if (p0) { sm.idx[j0] = (unsigned char)m0; sm.w[j0] = (float)(w0 / W); sm.ptr[j0] = f->ptrs[m0]; }
     if (p1) { sm.idx[j1] = (unsigned char)m1; sm.w[j1] = (float)(w1 / W); sm.ptr[j1] = f->ptrs[m1]; }
+    // learners that receive Theta' in their own dtype: compacted like the participants
+    const unsigned long long pm = f->push_mask;
+    const bool q0 = m0 < M && ((pm >> m0) & 1ull), q1 = m1 < M && ((pm >> m1) & 1ull);
+    const unsigned pb0 = __ballot_sync(0xffffffffu, q0);
+    const unsigned pb1 = __ballot_sync(0xffffffffu, q1);
+    if (q0) sm.push[__popc(pb0 & lt)] = const_cast<void *>(f->ptrs[m0]);
+    if (q1) sm.push[__popc(pb0) + __popc(pb1 & lt)] = const_cast<void *>(f->ptrs[m1]);
     if (lane == 0) {
+        sm.n_push = __popc(pb0) + __popc(pb1);
         sm.theta = f->theta;
         sm.mom = f->mom;
         sm.out_bf16 = f->out_bf16;
@@ -276,6 +286,10 @@ __device__ __forceinline__ void process_tail(Smem &sm, const Common &c, unsigned
     sm.mom[e] = vn;
     sm.theta[e] = tn;
     if (sm.out_bf16 != nullptr) sm.out_bf16[e] = (uint16_t)(pack_bf16x2(tn, 0.0f) & 0xffffu);
+    for (int q = 0; q < sm.n_push; ++q) {
+        if (BF16) reinterpret_cast<uint16_t *>(sm.push[q])[e] = (uint16_t)(pack_bf16x2(tn, 0.0f) & 0xffffu);
+        else reinterpret_cast<float *>(sm.push[q])[e] = tn;
+    }
     dsq = fmaf(delta, delta, dsq);
     tsq = fmaf(tn, tn, tsq);
     msq = fmaf(vn, vn, msq);

@@ -171,6 +171,7 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
 
     const float eta = c.eta, mu = c.mu;
     const bool heavy = (c.flags & DD_HEAVY_BALL) != 0;
+    const int n_push = sm.n_push;
 #pragma unroll 1
     for (unsigned v0 = v_first; v0 < nfull && !rs.failed; v0 += row_stride) {
         const unsigned cnt = min(kRowSteps, nfull - v0);
@@ -316,10 +317,20 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
                         const unsigned vi = v0 + step;
                         store_f32x8<WIDE>(sm.mom, vi, V);
                         store_f32x8<WIDE>(sm.theta, vi, T);
-                        if (sm.out_bf16 != nullptr)
-                            st_stream16(reinterpret_cast<uint4 *>(sm.out_bf16) + vi,
-                                        make_uint4(pack_bf16x2(T[0], T[1]), pack_bf16x2(T[2], T[3]),
-                                                   pack_bf16x2(T[4], T[5]), pack_bf16x2(T[6], T[7])));
+                        if (sm.out_bf16 != nullptr || (BF16 && n_push > 0)) {
+                            const uint4 packed = make_uint4(pack_bf16x2(T[0], T[1]), pack_bf16x2(T[2], T[3]),
+                                                            pack_bf16x2(T[4], T[5]), pack_bf16x2(T[6], T[7]));
+                            if (sm.out_bf16 != nullptr)
+                                st_stream16(reinterpret_cast<uint4 *>(sm.out_bf16) + vi, packed);
+                            // fused push: Theta' replaces the selected learners' copies (in place: this
+                            // warp has already consumed these elements of every copy it reads)
+                            if (BF16)
+                                for (int q = 0; q < n_push; ++q)
+                                    st_stream16(reinterpret_cast<uint4 *>(sm.push[q]) + vi, packed);
+                        }
+                        if (!BF16)
+                            for (int q = 0; q < n_push; ++q)
+                                store_f32x8<false>(reinterpret_cast<float *>(sm.push[q]), vi, T);
                     }
                 }
                 release();

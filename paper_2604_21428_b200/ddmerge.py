@@ -26,6 +26,7 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libddmerge
 
 EXPORTS = (
     "dd_create", "dd_destroy", "dd_merge_fragment", "dd_merge_fragments_batched",
+    "dd_merge_fragment_push", "dd_merge_fragments_batched_push",
     "dd_merge_fragment_host", "dd_merge_fragments_batched_noalloc",
     "dd_merge_fragment_rda", "dd_merge_fragments_batched_rda",
     "dd_quantize_outer_gradient_int4", "dd_merge_fragment_int4",
@@ -93,6 +94,15 @@ def _load() -> ctypes.CDLL:
     lib.dd_merge_fragments_batched.restype = ctypes.c_int
     lib.dd_merge_fragments_batched.argtypes = [
         vp, ctypes.POINTER(CFragmentDesc), ctypes.c_int, ctypes.c_int, ctypes.c_int,
+        ctypes.c_float, ctypes.c_float, ctypes.c_uint32, vp, vp]
+    lib.dd_merge_fragment_push.restype = ctypes.c_int
+    lib.dd_merge_fragment_push.argtypes = [
+        vp, vp, vp, ctypes.POINTER(vp), ctypes.c_int, ctypes.c_int, u64p, u64p, ctypes.c_uint64,
+        ctypes.c_int, ctypes.c_float, ctypes.c_float, ctypes.c_uint32, ctypes.c_size_t, ctypes.c_uint64,
+        vp, vp, vp]
+    lib.dd_merge_fragments_batched_push.restype = ctypes.c_int
+    lib.dd_merge_fragments_batched_push.argtypes = [
+        vp, ctypes.POINTER(CFragmentDesc), u64p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
         ctypes.c_float, ctypes.c_float, ctypes.c_uint32, vp, vp]
     lib.dd_merge_fragment_rda.restype = ctypes.c_int
     lib.dd_merge_fragment_rda.argtypes = [
@@ -281,6 +291,37 @@ class Context:
             ctypes.c_uint64(quorum_mask & (2**64 - 1)), int(K), ctypes.c_float(outer_lr),
             ctypes.c_float(outer_mu), ctypes.c_uint32(flags), ctypes.c_size_t(n), _ptr(out_bf16),
             _ptr(record), _stream_handle(stream)))
+
+    def merge_fragment_push(self, global_, momentum, learners, tokens, quorum_mask: int, K: int,
+                            outer_lr: float, outer_mu: float, push_mask: int, *, n: int | None = None,
+                            learner_dtype: int | None = None, steps=None, flags: int = 0,
+                            out_bf16=None, record=None, stream=None) -> None:
+        """``dd_merge_fragment_push``: the merge, and Theta' written over the copies of the
+        learners in ``push_mask`` in the same pass."""
+        M = len(learners)
+        if n is None:
+            n = int(global_.numel())
+        if learner_dtype is None:
+            learner_dtype = _infer_dtype(learners)
+        ptrs = _pointer_array(learners)
+        self._check(lib.dd_merge_fragment_push(
+            self._h, _ptr(global_), _ptr(momentum), ptrs, M, learner_dtype, _u64_array(tokens),
+            None if steps is None else _u64_array(steps),
+            ctypes.c_uint64(quorum_mask & (2**64 - 1)), int(K), ctypes.c_float(outer_lr),
+            ctypes.c_float(outer_mu), ctypes.c_uint32(flags), ctypes.c_size_t(n),
+            ctypes.c_uint64(push_mask & (2**64 - 1)), _ptr(out_bf16), _ptr(record),
+            _stream_handle(stream)))
+
+    def merge_fragments_batched_push(self, fragments, push_masks, M: int, learner_dtype: int,
+                                     outer_lr: float, outer_mu: float, *, flags: int = 0, records=None,
+                                     stream=None) -> None:
+        """``dd_merge_fragments_batched_push``: ``push_masks`` holds one mask per fragment."""
+        P = len(fragments)
+        descs, _keep = _pack_descs(fragments, M)
+        self._check(lib.dd_merge_fragments_batched_push(
+            self._h, descs, _u64_array([int(x) & (2**64 - 1) for x in push_masks]), P, M, learner_dtype,
+            ctypes.c_float(outer_lr), ctypes.c_float(outer_mu), ctypes.c_uint32(flags), _ptr(records),
+            _stream_handle(stream)))
 
     def merge_fragment_rda(self, global_, momentum, learners, tokens, quorum_mask: int, K: int,
                            outer_lr: float, outer_mu: float, *, n: int | None = None,

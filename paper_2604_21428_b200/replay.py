@@ -5,8 +5,10 @@ per-(learner, fragment) token / step counters it carried -- exactly what the
 paper's deterministic replay records ("participant subsets and token
 weightings").  ``Syncer.step`` turns one tape entry into library calls: quorum
 selection with the grace window, ONE batched merge launch over the fragments that
-are due, and the broadcast of the updated fragments to the learners that are
-alive.  All arithmetic happens in libddmerge; this module only sequences calls.
+are due, and the push of the updated fragments to the learners that are alive --
+inside the merge launch when the learners simply take the new fragment (alpha = 0,
+plain averaging), as a broadcast launch per fragment otherwise.  All arithmetic
+happens in libddmerge; this module only sequences calls.
 """
 from __future__ import annotations
 
@@ -35,7 +37,7 @@ class Syncer:
 
     def __init__(self, ctx: "dd.Context", global_fragments, momentum_fragments, *, H: int,
                  offsets, K: int, outer_lr: float, outer_mu: float, learner_dtype: int,
-                 merge_kinds=None, alpha: float = 0.0, flags: int = 0):
+                 merge_kinds=None, alpha: float = 0.0, flags: int = 0, fused_push: bool = True):
         self.ctx = ctx
         self.theta = list(global_fragments)
         self.mom = list(momentum_fragments)
@@ -46,6 +48,7 @@ class Syncer:
         self.kinds = list(merge_kinds) if merge_kinds is not None else [dd.MERGE_AVG] * self.P
         self.alpha = float(alpha)
         self.flags = int(flags)
+        self.fused_push = bool(fused_push)
         self._records = dd.new_records(self.P, device=self.theta[0].device)
 
     def due(self, t: int):
@@ -73,26 +76,33 @@ class Syncer:
                               quorum_mask=res.mask, K=self.K, n=int(self.theta[p].numel())))
         recs = self._records[: len(frags) * dd.RECORD_BYTES]
         kinds = [self.kinds[p] for p in res.due]
-        if any(k == dd.MERGE_RDA for k in kinds):
+        # every learner that is alive receives the new fragment (and resets its counters)
+        alive = sum(1 << m for m in range(M) if entry.arrival_s[m] != float("inf"))
+        has_rda = any(k == dd.MERGE_RDA for k in kinds)
+        fused = self.fused_push and self.alpha == 0.0 and not has_rda and alive != 0
+        if has_rda:
             self.ctx.merge_fragments_batched_rda(frags, M, self.dtype, self.lr, self.mu,
                                                  merge_kinds=kinds, flags=self.flags, records=recs,
                                                  stream=stream)
+        elif fused:
+            # merge and push in one launch; a fragment whose quorum is not met pushes nothing
+            self.ctx.merge_fragments_batched_push(frags, [alive] * len(frags), M, self.dtype, self.lr,
+                                                  self.mu, flags=self.flags, records=recs, stream=stream)
         else:
             self.ctx.merge_fragments_batched(frags, M, self.dtype, self.lr, self.mu,
                                              flags=self.flags, records=recs, stream=stream)
         if read_back:
             res.records = dd.read_records(recs, len(frags))
             merged = [rec.status == dd.STATUS_OK for rec in res.records]
-        else:
+        elif not fused:
             need = max(self.K, 1)
             merged = [sum(1 for m in range(M) if (res.mask >> m) & 1 and entry.tokens[p][m] > 0) >= need
                       for p in res.due]
-        # every learner that is alive receives the new fragment (and resets its counters)
-        alive = sum(1 << m for m in range(M) if entry.arrival_s[m] != float("inf"))
-        for p, ok in zip(res.due, merged):
-            if ok and alive:
-                self.ctx.broadcast_fragment(self.theta[p],
-                                            [learner_fragments[m][p] for m in range(M)], alive,
-                                            self.alpha, n=int(self.theta[p].numel()),
-                                            learner_dtype=self.dtype, stream=stream)
+        if not fused:
+            for p, ok in zip(res.due, merged):
+                if ok and alive:
+                    self.ctx.broadcast_fragment(self.theta[p],
+                                                [learner_fragments[m][p] for m in range(M)], alive,
+                                                self.alpha, n=int(self.theta[p].numel()),
+                                                learner_dtype=self.dtype, stream=stream)
         return res

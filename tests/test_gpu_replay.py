@@ -24,8 +24,8 @@ def _to_host(t):
     return t.view(torch.int16).numpy().view(np.uint16).copy() if t.dtype == torch.bfloat16 else t.numpy().copy()
 
 
-@pytest.mark.parametrize("use_rda", [False, True])
-def test_replay_matches_oracle(use_rda):
+@pytest.mark.parametrize("use_rda,fused", [(False, True), (False, False), (True, True)])
+def test_replay_matches_oracle(use_rda, fused):
     from paper_2604_21428_b200 import ddmerge as dd
     from paper_2604_21428_b200.replay import Syncer, TapeEntry
 
@@ -49,7 +49,7 @@ def test_replay_matches_oracle(use_rda):
 
     ctx = dd.Context(0)
     syncer = Syncer(ctx, d_theta, d_mom, H=H, offsets=offsets, K=K, outer_lr=eta, outer_mu=mu,
-                    learner_dtype=dd.BF16, merge_kinds=kinds, flags=dd.DIAG_STATE)
+                    learner_dtype=dd.BF16, merge_kinds=kinds, flags=dd.DIAG_STATE, fused_push=fused)
     drift = np.random.default_rng(17)
     merged = 0
     for t, e in enumerate(tape):
@@ -69,6 +69,10 @@ def test_replay_matches_oracle(use_rda):
                 for m in range(M):
                     if math.isfinite(e["arrival_s"][m]):
                         oracle.apply_to_learner(h_learn[m][p], h_theta[p], 0.0)
+            # the push reached exactly the learners that are alive (fused into the merge or not)
+            for m in range(M):
+                same = np.mean(_to_host(d_learn[m][p]) == h_learn[m][p])
+                assert same > 0.995, (t, p, m, same)
         # ---- learners move on: identical drift on both sides ---------------------------
         for m in range(M):
             for p, n in enumerate(sizes):
