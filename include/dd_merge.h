@@ -239,6 +239,18 @@ int dd_merge_fragments_batched_rda(dd_ctx *ctx, const dd_fragment_desc *descs, i
                                    size_t scratch_elems, void *cuda_stream);
 
 /*
+ * The batched radial-directional merge with the push of dd_merge_fragment_push: the apply
+ * pass, which no longer reads the learner copies, overwrites those selected by
+ * push_masks[p] (host array of P masks) with Theta'.  Same rules for pushed copies.
+ */
+int dd_merge_fragments_batched_rda_push(dd_ctx *ctx, const dd_fragment_desc *descs,
+                                        const uint64_t *push_masks, int P, int M,
+                                        dd_dtype learner_dtype, float outer_lr, float outer_mu,
+                                        uint32_t flags, const uint8_t *merge_kinds,
+                                        dd_merge_record *records, float *scratch, size_t scratch_elems,
+                                        void *cuda_stream);
+
+/*
  * int4 compression of outer gradients (Appendix "Outer gradients compression": 16 -> 4
  * bits per value before the merge, comparable quality; 2 and 1 bit are not).  The paper
  * prints no quantiser; this library's reading, fixed here so that both ends agree:

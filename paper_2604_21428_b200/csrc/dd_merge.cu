@@ -457,12 +457,10 @@ static size_t round_up8(size_t n) { return (n + 7) / 8 * 8; }
 
 }  // namespace ddm
 
-extern "C" int dd_merge_fragments_batched_rda(dd_ctx *ctx, const dd_fragment_desc *descs, int P,
-                                              int M, dd_dtype learner_dtype, float outer_lr,
-                                              float outer_mu, uint32_t flags,
-                                              const uint8_t *merge_kinds, dd_merge_record *records,
-                                              float *scratch, size_t scratch_elems,
-                                              void *cuda_stream)
+static int rda_batched_impl(dd_ctx *ctx, const dd_fragment_desc *descs, const uint64_t *push_masks,
+                            int P, int M, dd_dtype learner_dtype, float outer_lr, float outer_mu,
+                            uint32_t flags, const uint8_t *merge_kinds, dd_merge_record *records,
+                            float *scratch, size_t scratch_elems, void *cuda_stream)
 {
     int rc = check_common(ctx, M, learner_dtype, outer_lr, outer_mu, flags);
     if (rc != DD_OK) return rc;
@@ -516,6 +514,10 @@ extern "C" int dd_merge_fragments_batched_rda(dd_ctx *ctx, const dd_fragment_des
         rc = fill_fragment(f, d.global, d.momentum, d.out_bf16, d.learner_ptrs, d.tokens, d.steps,
                            d.quorum_mask, d.K, d.n, M, learner_bytes_of(learner_dtype, d.n));
         if (rc != DD_OK) return rc;
+        if (push_masks && push_masks[p]) {      // written by the apply pass, after the passes that read
+            rc = set_push(f, d.learner_ptrs, push_masks[p], M, d.n, learner_bytes_of(learner_dtype, d.n));
+            if (rc != DD_OK) return rc;
+        }
         f.kind = (!merge_kinds || merge_kinds[p] == DD_MERGE_RDA) ? DD_MERGE_RDA : DD_MERGE_AVG;
         if (f.kind == DD_MERGE_RDA) {
             f.scratch = next_scratch;
@@ -556,6 +558,30 @@ extern "C" int dd_merge_fragments_batched_rda(dd_ctx *ctx, const dd_fragment_des
     slot.used = true;
     ctx->next_slot = (ctx->next_slot + 1) % kSlots;
     return DD_OK;
+}
+
+extern "C" int dd_merge_fragments_batched_rda(dd_ctx *ctx, const dd_fragment_desc *descs, int P,
+                                              int M, dd_dtype learner_dtype, float outer_lr,
+                                              float outer_mu, uint32_t flags,
+                                              const uint8_t *merge_kinds, dd_merge_record *records,
+                                              float *scratch, size_t scratch_elems,
+                                              void *cuda_stream)
+{
+    return rda_batched_impl(ctx, descs, nullptr, P, M, learner_dtype, outer_lr, outer_mu, flags, merge_kinds,
+                            records, scratch, scratch_elems, cuda_stream);
+}
+
+extern "C" int dd_merge_fragments_batched_rda_push(dd_ctx *ctx, const dd_fragment_desc *descs,
+                                                   const uint64_t *push_masks, int P, int M,
+                                                   dd_dtype learner_dtype, float outer_lr,
+                                                   float outer_mu, uint32_t flags,
+                                                   const uint8_t *merge_kinds, dd_merge_record *records,
+                                                   float *scratch, size_t scratch_elems,
+                                                   void *cuda_stream)
+{
+    if (P > 0 && !push_masks) return DD_ERR_INVALID_ARG;
+    return rda_batched_impl(ctx, descs, push_masks, P, M, learner_dtype, outer_lr, outer_mu, flags,
+                            merge_kinds, records, scratch, scratch_elems, cuda_stream);
 }
 
 extern "C" int dd_merge_fragment_rda(dd_ctx *ctx, float *global, float *momentum,

@@ -26,7 +26,7 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libddmerge
 
 EXPORTS = (
     "dd_create", "dd_destroy", "dd_merge_fragment", "dd_merge_fragments_batched",
-    "dd_merge_fragment_push", "dd_merge_fragments_batched_push",
+    "dd_merge_fragment_push", "dd_merge_fragments_batched_push", "dd_merge_fragments_batched_rda_push",
     "dd_merge_fragment_host", "dd_merge_fragments_batched_noalloc",
     "dd_merge_fragment_rda", "dd_merge_fragments_batched_rda",
     "dd_quantize_outer_gradient_int4", "dd_merge_fragment_int4",
@@ -111,6 +111,11 @@ def _load() -> ctypes.CDLL:
     lib.dd_merge_fragments_batched_rda.restype = ctypes.c_int
     lib.dd_merge_fragments_batched_rda.argtypes = [
         vp, ctypes.POINTER(CFragmentDesc), ctypes.c_int, ctypes.c_int, ctypes.c_int,
+        ctypes.c_float, ctypes.c_float, ctypes.c_uint32, ctypes.POINTER(ctypes.c_uint8), vp, vp,
+        ctypes.c_size_t, vp]
+    lib.dd_merge_fragments_batched_rda_push.restype = ctypes.c_int
+    lib.dd_merge_fragments_batched_rda_push.argtypes = [
+        vp, ctypes.POINTER(CFragmentDesc), u64p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
         ctypes.c_float, ctypes.c_float, ctypes.c_uint32, ctypes.POINTER(ctypes.c_uint8), vp, vp,
         ctypes.c_size_t, vp]
     lib.dd_quantize_outer_gradient_int4.restype = ctypes.c_int
@@ -343,17 +348,23 @@ class Context:
 
     def merge_fragments_batched_rda(self, fragments, M: int, learner_dtype: int, outer_lr: float,
                                     outer_mu: float, *, merge_kinds=None, flags: int = 0,
-                                    records=None, scratch=None, stream=None) -> None:
+                                    records=None, scratch=None, stream=None, push_masks=None) -> None:
         """``dd_merge_fragments_batched_rda``: ``merge_kinds`` is a list of MERGE_AVG /
-        MERGE_RDA per fragment (None = all RDA); ``scratch`` an optional float32 tensor."""
+        MERGE_RDA per fragment (None = all RDA); ``scratch`` an optional float32 tensor.
+        With ``push_masks`` (one mask per fragment): ``dd_merge_fragments_batched_rda_push``."""
         P = len(fragments)
         descs, _keep = _pack_descs(fragments, M)
         kinds = None if merge_kinds is None else (ctypes.c_uint8 * P)(*[int(k) for k in merge_kinds])
-        self._check(lib.dd_merge_fragments_batched_rda(
-            self._h, descs, P, M, learner_dtype, ctypes.c_float(outer_lr), ctypes.c_float(outer_mu),
-            ctypes.c_uint32(flags), kinds, _ptr(records), _ptr(scratch),
-            ctypes.c_size_t(0 if scratch is None else int(scratch.numel())),
-            _stream_handle(stream)))
+        tail = (ctypes.c_uint32(flags), kinds, _ptr(records), _ptr(scratch),
+                ctypes.c_size_t(0 if scratch is None else int(scratch.numel())), _stream_handle(stream))
+        if push_masks is None:
+            self._check(lib.dd_merge_fragments_batched_rda(
+                self._h, descs, P, M, learner_dtype, ctypes.c_float(outer_lr), ctypes.c_float(outer_mu),
+                *tail))
+        else:
+            self._check(lib.dd_merge_fragments_batched_rda_push(
+                self._h, descs, _u64_array([int(x) & (2**64 - 1) for x in push_masks]), P, M,
+                learner_dtype, ctypes.c_float(outer_lr), ctypes.c_float(outer_mu), *tail))
 
     def broadcast_fragment(self, global_, learners, apply_mask: int, alpha: float = 0.0, *,
                            n: int | None = None, learner_dtype: int | None = None,

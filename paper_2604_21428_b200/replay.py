@@ -6,8 +6,8 @@ paper's deterministic replay records ("participant subsets and token
 weightings").  ``Syncer.step`` turns one tape entry into library calls: quorum
 selection with the grace window, ONE batched merge launch over the fragments that
 are due, and the push of the updated fragments to the learners that are alive --
-inside the merge launch when the learners simply take the new fragment (alpha = 0,
-plain averaging), as a broadcast launch per fragment otherwise.  All arithmetic
+inside the merge launch when the learners simply take the new fragment (alpha = 0),
+as a broadcast launch per fragment otherwise.  All arithmetic
 happens in libddmerge; this module only sequences calls.
 """
 from __future__ import annotations
@@ -79,11 +79,12 @@ class Syncer:
         # every learner that is alive receives the new fragment (and resets its counters)
         alive = sum(1 << m for m in range(M) if entry.arrival_s[m] != float("inf"))
         has_rda = any(k == dd.MERGE_RDA for k in kinds)
-        fused = self.fused_push and self.alpha == 0.0 and not has_rda and alive != 0
+        fused = self.fused_push and self.alpha == 0.0 and alive != 0
         if has_rda:
             self.ctx.merge_fragments_batched_rda(frags, M, self.dtype, self.lr, self.mu,
                                                  merge_kinds=kinds, flags=self.flags, records=recs,
-                                                 stream=stream)
+                                                 stream=stream,
+                                                 push_masks=[alive] * len(frags) if fused else None)
         elif fused:
             # merge and push in one launch; a fragment whose quorum is not met pushes nothing
             self.ctx.merge_fragments_batched_push(frags, [alive] * len(frags), M, self.dtype, self.lr,

@@ -149,3 +149,33 @@ def test_push_argument_validation(dd, ctx):
     # bits at or above M are ignored
     ctx.merge_fragment_push(t_dev, v_dev, l_dev, tokens, 0b111, 1, ETA, MU, 0b1000, n=n, learner_dtype=dd.BF16)
     torch.cuda.synchronize()
+
+
+def test_batched_rda_and_push_equals_rda_then_broadcast(dd, ctx):
+    # mixed batch (one plain-average fragment, two radial-directional): the fused push against the
+    # library's own merge followed by broadcasts, which the other tests tie to the oracle
+    sizes = [30_007, 8192 * 2 + 1, 100_003]
+    M = 5
+    kinds = [dd.MERGE_AVG, dd.MERGE_RDA, dd.MERGE_RDA]
+    masks, pushes = [0b11011, 0b10111, 0b01110], [0b11111, 0b01001, 0b10110]
+    tokens = [[5, 9, 2, 7, 3], [4, 4, 8, 1, 6], [2, 3, 5, 7, 11]]
+
+    def make():
+        fr = []
+        for p, n in enumerate(sizes):
+            theta, v, learners = synth.fragment_cpu(n, M, "bf16", 900 + p)
+            fr.append(dict(global_=torch.from_numpy(theta).cuda(), momentum=torch.from_numpy(v).cuda(),
+                           learners=[to_torch_learner(a, "cuda") for a in learners], tokens=tokens[p],
+                           quorum_mask=masks[p], K=2, n=n))
+        return fr
+
+    a, b = make(), make()
+    ctx.merge_fragments_batched_rda(a, M, dd.BF16, ETA, MU, merge_kinds=kinds, push_masks=pushes)
+    ctx.merge_fragments_batched_rda(b, M, dd.BF16, ETA, MU, merge_kinds=kinds)
+    for p in range(len(sizes)):
+        ctx.broadcast_fragment(b[p]["global_"], b[p]["learners"], pushes[p], 0.0)
+    torch.cuda.synchronize()
+    for p in range(len(sizes)):
+        assert torch.equal(a[p]["global_"], b[p]["global_"]) and torch.equal(a[p]["momentum"], b[p]["momentum"])
+        for m in range(M):
+            assert torch.equal(a[p]["learners"][m], b[p]["learners"][m]), (p, m)

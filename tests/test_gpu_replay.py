@@ -24,7 +24,7 @@ def _to_host(t):
     return t.view(torch.int16).numpy().view(np.uint16).copy() if t.dtype == torch.bfloat16 else t.numpy().copy()
 
 
-@pytest.mark.parametrize("use_rda,fused", [(False, True), (False, False), (True, True)])
+@pytest.mark.parametrize("use_rda,fused", [(False, True), (False, False), (True, True), (True, False)])
 def test_replay_matches_oracle(use_rda, fused):
     from paper_2604_21428_b200 import ddmerge as dd
     from paper_2604_21428_b200.replay import Syncer, TapeEntry
