@@ -353,6 +353,9 @@ def main():
         w = synth.scaled(w, args.scale, align=8)
     job_params = w.total_params * (world if args.sharding == "replica" else 1)
     if args.sharding == "range" and world > 1:
+        if args.merge == "rda":
+            raise SystemExit("--merge rda needs whole-fragment norms between its passes: "
+                             "run it with --sharding replica")
         w.fragment_sizes = [hi - lo for lo, hi in
                             (ddist.shard_range(n, rank, world) for n in w.fragment_sizes)]
     frags = build_workload(w, device, rank, args.out_bf16, args.resident)
