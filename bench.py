@@ -247,6 +247,8 @@ def run_replay(args):
     by a seeded synthetic event tape.  One bench step = one syncer step."""
     import torch
 
+    from paper_2604_21428_b200 import build as lib_build
+    lib_build.build()            # no-op when libddmerge.so is newer than its sources
     from paper_2604_21428_b200 import ddmerge as dd
     from paper_2604_21428_b200 import synth
     from paper_2604_21428_b200.replay import Syncer, TapeEntry
@@ -336,6 +338,8 @@ def main():
     import torch
     import torch.distributed as dist
 
+    from paper_2604_21428_b200 import build as lib_build
+    lib_build.build()            # no-op when libddmerge.so is newer than its sources
     from paper_2604_21428_b200 import ddmerge as dd
     from paper_2604_21428_b200 import dist as ddist
     from paper_2604_21428_b200 import synth
