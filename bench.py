@@ -256,7 +256,10 @@ def run_replay(args):
     torch.cuda.set_device(0)
     device = torch.device("cuda", 0)
     M, P, H, K = 8, 24, 24, 1
-    tensors = synth.dense_tensor_list(24, 2048, 8192, 32000)
+    d_model = 2048
+    if args.scale != 1.0:            # a smaller model of the same shape (profiling captures)
+        d_model = max(64, int(2048 * args.scale ** 0.5) // 64 * 64)
+    tensors = synth.dense_tensor_list(24, d_model, 4 * d_model, 32000)
     frag_of, bits = dd.plan_fragments([16 * n for n, _ in tensors], None, P, dd.FRAG_BALANCED)
     sizes = [b // 16 for b in bits]
     offsets = list(range(P))
@@ -309,7 +312,8 @@ def run_replay(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
-        "config": {"workload": "tape24", "model_params": sum(sizes), "fragments": P, "H": H, "M": M,
+        "config": {"workload": "tape24" if args.scale == 1.0 else f"tape24@{args.scale:g}",
+                   "model_params": sum(sizes), "d_model": d_model, "fragments": P, "H": H, "M": M,
                    "K": K, "grace_s": 0.25, "fragment_elems_min_max": [min(sizes), max(sizes)],
                    "planner": "balanced", "learner_dtype": "bf16",
                    "l2": "inputs larger than L2 (no flush)"},
