@@ -259,3 +259,47 @@ def test_scale500m_full_size_rda_properties():
     assert abs(rec.theta_sq - _sq(theta)) <= TOL_NORM * rec.theta_sq
     assert abs(rec.mom_sq - _sq(mom)) <= TOL_NORM * rec.mom_sq
     ctx.close()
+
+
+def test_fragment_beyond_32_bit_offsets():
+    """One fragment of 2^32 + 24,581 elements (17 GB of Theta, 17 GB of v, one participating bf16
+    copy, merged and pushed to): element indices pass 2^32 and byte offsets pass 2^32, 2^33 and
+    2^34.  Windows sit on each of those boundaries; the oracle merges them from inputs saved
+    before the launch."""
+    from paper_2604_21428_b200 import ddmerge as dd
+
+    n = (1 << 32) + 3 * 8192 + 5
+    free, _ = torch.cuda.mem_get_info()
+    if free < 10 * n + (6 << 30):
+        pytest.skip("needs 46 GiB of device memory")
+    dev = torch.device("cuda", 0)
+    theta = torch.empty(n, dtype=torch.float32, device=dev)
+    mom = torch.empty(n, dtype=torch.float32, device=dev)
+    copy = torch.empty(n, dtype=torch.bfloat16, device=dev)
+    synth.fill_fragment_gpu(theta, mom, [copy], seed=4242)
+    learners = [None, copy]                              # learner 0 is absent: null pointer
+    tokens, mask, K = [0, 12345], 0b10, 1
+    half = WINDOW // 2
+    centres = [half, 1 << 29, 1 << 30, 1 << 31, (1 << 32) - 8192, 1 << 32, n - half]
+    starts = [max(0, min(n - WINDOW, c - half)) for c in centres]
+    windows = [(lo, lo + WINDOW) for lo in starts]
+    saved = [(theta[lo:hi].cpu().numpy().copy(), mom[lo:hi].cpu().numpy().copy(),
+              [None, _to_host_learner(copy[lo:hi])]) for lo, hi in windows]
+    ctx = dd.Context(0)
+    records = dd.new_records(1, device=dev)
+    # merged and pushed in one launch: the copy is overwritten with Theta' (bf16) in place
+    ctx.merge_fragment_push(theta, mom, learners, tokens, mask, K, ETA, MU, 0b10, n=n,
+                            learner_dtype=dd.BF16, flags=dd.DIAG_STATE, record=records)
+    torch.cuda.synchronize()
+    rec = dd.read_records(records)[0]
+    assert (rec.status, rec.n_part, rec.idx[:1]) == (0, 1, [1])
+    for (lo, hi), (t0, v0, ls) in zip(windows, saved):
+        oracle.merge_fragment(t0, v0, ls, tokens, mask, K, ETA, MU)
+        e_t = floor_rel_err(theta[lo:hi].cpu().numpy(), t0)
+        e_v = floor_rel_err(mom[lo:hi].cpu().numpy(), v0)
+        assert e_t <= TOL_STATE and e_v <= TOL_STATE, (lo, e_t, e_v)
+        oracle.apply_to_learner(ls[1], t0, 0.0)
+        assert np.mean(_to_host_learner(copy[lo:hi]) == ls[1]) > 0.999, lo
+    assert abs(rec.theta_sq - _sq(theta)) <= TOL_NORM * rec.theta_sq
+    assert abs(rec.mom_sq - _sq(mom)) <= TOL_NORM * rec.mom_sq
+    ctx.close()
