@@ -303,3 +303,47 @@ def test_fragment_beyond_32_bit_offsets():
     assert abs(rec.theta_sq - _sq(theta)) <= TOL_NORM * rec.theta_sq
     assert abs(rec.mom_sq - _sq(mom)) <= TOL_NORM * rec.mom_sq
     ctx.close()
+
+
+def test_int4_fragment_beyond_32_bit_offsets():
+    """The quantiser and the compressed merge on 2^32 + 12,421 elements: windows on the element
+    index 2^32 and on the byte-offset boundaries of Theta / v (2^32 ... 2^34) and of the codes."""
+    from paper_2604_21428_b200 import ddmerge as dd
+
+    n = (1 << 32) + 97 * 128 + 5
+    free, _ = torch.cuda.mem_get_info()
+    if free < 11 * n + (6 << 30):
+        pytest.skip("needs 50 GiB of device memory")
+    dev = torch.device("cuda", 0)
+    theta = torch.empty(n, dtype=torch.float32, device=dev)
+    mom = torch.empty(n, dtype=torch.float32, device=dev)
+    copy = torch.empty(n, dtype=torch.bfloat16, device=dev)
+    synth.fill_fragment_gpu(theta, mom, [copy], seed=777)
+    codes = torch.empty((n + 1) // 2, dtype=torch.uint8, device=dev)
+    scales = torch.empty((n + 127) // 128, dtype=torch.float32, device=dev)
+    ctx = dd.Context(0)
+    ctx.quantize_outer_gradient_int4(theta, copy, codes, scales)
+    half = WINDOW // 2
+    centres = [half, 1 << 30, 1 << 31, 1 << 32, n]
+    starts = [max(0, min(n - WINDOW, c - half)) // 128 * 128 for c in centres]
+    windows = [(lo, min(n, lo + WINDOW + 128)) for lo in starts]      # the last one ends on the ragged block
+    saved = [(theta[lo:hi].cpu().numpy().copy(), mom[lo:hi].cpu().numpy().copy(),
+              _to_host_learner(copy[lo:hi])) for lo, hi in windows]
+    del copy
+    tokens, mask, K = [777], 0b1, 1
+    records = dd.new_records(1, device=dev)
+    ctx.merge_fragment_int4(theta, mom, [codes], [scales], tokens, mask, K, ETA, MU, n=n,
+                            flags=dd.DIAG_STATE, record=records)
+    torch.cuda.synchronize()
+    rec = dd.read_records(records)[0]
+    assert (rec.status, rec.n_part) == (0, 1)
+    for (lo, hi), (t0, v0, l0) in zip(windows, saved):
+        q_codes, q_scales = oracle.quantize_int4(t0, l0)
+        np.testing.assert_array_equal(codes[lo // 2:(hi + 1) // 2].cpu().numpy(), q_codes)
+        np.testing.assert_array_equal(scales[lo // 128:(hi + 127) // 128].cpu().numpy().view(np.uint32),
+                                      q_scales.view(np.uint32))
+        oracle.merge_fragment_int4(t0, v0, [q_codes], [q_scales], tokens, mask, K, ETA, MU)
+        assert floor_rel_err(theta[lo:hi].cpu().numpy(), t0) <= TOL_STATE, lo
+        assert floor_rel_err(mom[lo:hi].cpu().numpy(), v0) <= TOL_STATE, lo
+    assert abs(rec.theta_sq - _sq(theta)) <= TOL_NORM * rec.theta_sq
+    ctx.close()
