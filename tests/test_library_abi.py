@@ -120,3 +120,30 @@ def test_header_is_plain_c_and_links(dd, tmp_path):
     out = subprocess.run([exe], capture_output=True, text=True, timeout=60)
     assert out.returncode == 0, (out.returncode, out.stderr)
     assert out.stdout.split() == ["abi", "ok", str(dd.RECORD_BYTES), str(dd.MAX_LEARNERS)]
+
+
+def test_missing_library_fails_loudly(tmp_path):
+    """Without libddmerge.so the binding refuses to import: there is no CPU fallback to fall
+    through to.  (A copy of the package without the built library, in a child interpreter.)"""
+    import shutil
+    import subprocess
+    import sys
+
+    pkg = os.path.join(ROOT, "paper_2604_21428_b200")
+    dst = tmp_path / "paper_2604_21428_b200"
+    shutil.copytree(pkg, dst, ignore=shutil.ignore_patterns("*.so", "*.so.*", "__pycache__", "csrc"))
+    proc = subprocess.run([sys.executable, "-c", "from paper_2604_21428_b200 import ddmerge"],
+                          cwd=tmp_path, capture_output=True, text=True,
+                          env={**os.environ, "PYTHONPATH": str(tmp_path)})
+    assert proc.returncode != 0
+    assert "libddmerge.so is missing" in proc.stderr and "no CPU fallback" in proc.stderr
+
+
+def test_product_package_never_imports_the_oracle():
+    """The oracle is test infrastructure: nothing under the package names it."""
+    pkg = os.path.join(ROOT, "paper_2604_21428_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h", ".cpp")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "import oracle" not in text and "from oracle" not in text and "dd_oracle" not in text, f
