@@ -621,3 +621,25 @@ def test_packed_pointer_and_count_arrays(dd, ctx):
     with pytest.raises(ValueError):
         ctx.merge_fragment(results[0][0].cuda(), results[0][1].cuda(), dd.pack_pointers(l_dev), tokens,
                            mask, K, ETA, MU, n=n)
+
+
+def test_bitwise_reproducible_run_to_run(dd, ctx):
+    """Same inputs, same bits: every element has one owner and the norms are reduced in a fixed
+    order (per-CTA partials added by the last CTA in CTA order), whatever the CTA timing."""
+    n, M = 2 * 296 * 8192 + 4099, 6
+    tokens, mask, K = [11, 7, 0, 5, 9, 13], 0b111011, 3
+    theta, v, learners = synth.fragment_cpu(n, M, "bf16", 404)
+    l_dev = [to_torch_learner(a, "cuda") for a in learners]
+    first = None
+    for rep in range(12):
+        t_dev, v_dev = torch.from_numpy(theta).cuda(), torch.from_numpy(v).cuda()
+        out = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+        rec_buf = dd.new_records(1)
+        ctx.merge_fragment(t_dev, v_dev, l_dev, tokens, mask, K, ETA, MU,
+                           flags=dd.DIAG_STATE | dd.DIAG_PER_LEARNER, out_bf16=out, record=rec_buf)
+        torch.cuda.synchronize()
+        got = (t_dev, v_dev, out.view(torch.int16), rec_buf.clone())
+        if first is None:
+            first = got
+        else:
+            assert all(torch.equal(a, b) for a, b in zip(first, got)), rep
