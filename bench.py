@@ -361,9 +361,6 @@ def main():
         w = synth.scaled(w, args.scale, align=8)
     job_params = w.total_params * (world if args.sharding == "replica" else 1)
     if args.sharding == "range" and world > 1:
-        if args.merge == "rda":
-            raise SystemExit("--merge rda needs whole-fragment norms between its passes: "
-                             "run it with --sharding replica")
         w.fragment_sizes = [hi - lo for lo, hi in
                             (ddist.shard_range(n, rank, world) for n in w.fragment_sizes)]
     frags = build_workload(w, device, rank, args.out_bf16, args.resident)
@@ -390,6 +387,10 @@ def main():
                                                  int4_scales[m], n=n0, learner_dtype=ldtype)
         torch.cuda.synchronize()
 
+    rda_scratch = None
+    if args.merge == "rda" and args.sharding == "range" and world > 1:
+        rda_scratch = torch.empty(sum((n + 7) // 8 * 8 for n in w.fragment_sizes), dtype=torch.float32,
+                                  device=device)
     # the same buffers are merged every step: marshal their addresses and counts once
     packed_ptrs = dd.pack_pointers(frags[0]["learners"]) if w.P == 1 else None
     packed_tokens = dd.pack_u64(frags[0]["tokens"]) if w.P == 1 else None
@@ -400,6 +401,10 @@ def main():
             ctx.merge_fragment_int4(f["global_"], f["momentum"], int4_codes, int4_scales, f["tokens"],
                                     f["quorum_mask"], f["K"], eta, mu, n=f["n"], flags=flags,
                                     out_bf16=f["out_bf16"], record=records, stream=stream)
+        elif args.merge == "rda" and rda_scratch is not None:
+            # range-sharded: the passes one by one, norms all-reduced over the ranks in between
+            ddist.rda_merge_range_sharded(ctx, frags, w.M, ldtype, eta, mu, records=records,
+                                          scratch=rda_scratch, flags=flags, stream=stream)
         elif args.merge == "rda":
             ctx.merge_fragments_batched_rda(frags, w.M, ldtype, eta, mu, flags=flags,
                                             records=records, stream=stream)

@@ -251,6 +251,34 @@ int dd_merge_fragments_batched_rda_push(dd_ctx *ctx, const dd_fragment_desc *des
                                         void *cuda_stream);
 
 /*
+ * One pass of the batched radial-directional merge, for a fragment that is sharded by
+ * element range over several GPUs.  The merge needs two whole-fragment quantities that a
+ * shard cannot know, so the caller runs the passes one by one on every shard and sums
+ * across the shards in between (the paper's RDA likewise all-reduces the norms first and
+ * the directions second, Appendix "Merging methods"):
+ *
+ *   DD_RDA_PASS_NORMS      writes records[p].delta_m_sq[j] = ||Theta - theta_j||^2 of the shard
+ *                          -> sum delta_m_sq[0 .. n_part) over the shards, in place
+ *   DD_RDA_PASS_DIRECTION  reads delta_m_sq; writes the shard's mean direction to scratch and
+ *                          its squared length to records[p].delta_sq
+ *                          -> sum delta_sq over the shards, in place
+ *   DD_RDA_PASS_APPLY      reads delta_m_sq and delta_sq; outer step (and push, if push_masks is
+ *                          given); writes the shard's ||Delta||^2, ||Theta'||^2, ||v'||^2
+ *                          -> sum those three for whole-fragment diagnostics
+ *
+ * records and scratch are required and must be the same memory in all three calls, as must
+ * every other argument.  Fragments of kind DD_MERGE_AVG are merged by the apply pass alone.
+ * With a single shard the three calls equal dd_merge_fragments_batched_rda[_push].
+ */
+enum { DD_RDA_PASS_NORMS = 0, DD_RDA_PASS_DIRECTION = 1, DD_RDA_PASS_APPLY = 2 };
+int dd_merge_fragments_batched_rda_pass(dd_ctx *ctx, const dd_fragment_desc *descs,
+                                        const uint64_t *push_masks /* may be NULL */, int P, int M,
+                                        dd_dtype learner_dtype, float outer_lr, float outer_mu,
+                                        uint32_t flags, const uint8_t *merge_kinds,
+                                        dd_merge_record *records, float *scratch, size_t scratch_elems,
+                                        int pass, void *cuda_stream);
+
+/*
  * int4 compression of outer gradients (Appendix "Outer gradients compression": 16 -> 4
  * bits per value before the merge, comparable quality; 2 and 1 bit are not).  The paper
  * prints no quantiser; this library's reading, fixed here so that both ends agree:

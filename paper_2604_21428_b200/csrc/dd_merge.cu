@@ -445,11 +445,14 @@ namespace ddm {
 
 template <bool BF16>
 static cudaError_t launch_rda_passes(const DevFrag *dev_frags, const Common &c, unsigned grid,
-                                     cudaStream_t stream)
+                                     cudaStream_t stream, int only_pass)
 {
-    rda_pass_kernel<BF16, kModeNorms><<<grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
-    rda_pass_kernel<BF16, kModeDir><<<grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
-    rda_pass_kernel<BF16, kModeApply><<<grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
+    if (only_pass < 0 || only_pass == DD_RDA_PASS_NORMS)
+        rda_pass_kernel<BF16, kModeNorms><<<grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
+    if (only_pass < 0 || only_pass == DD_RDA_PASS_DIRECTION)
+        rda_pass_kernel<BF16, kModeDir><<<grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
+    if (only_pass < 0 || only_pass == DD_RDA_PASS_APPLY)
+        rda_pass_kernel<BF16, kModeApply><<<grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
     return cudaGetLastError();
 }
 
@@ -460,7 +463,7 @@ static size_t round_up8(size_t n) { return (n + 7) / 8 * 8; }
 static int rda_batched_impl(dd_ctx *ctx, const dd_fragment_desc *descs, const uint64_t *push_masks,
                             int P, int M, dd_dtype learner_dtype, float outer_lr, float outer_mu,
                             uint32_t flags, const uint8_t *merge_kinds, dd_merge_record *records,
-                            float *scratch, size_t scratch_elems, void *cuda_stream)
+                            float *scratch, size_t scratch_elems, void *cuda_stream, int only_pass = -1)
 {
     int rc = check_common(ctx, M, learner_dtype, outer_lr, outer_mu, flags);
     if (rc != DD_OK) return rc;
@@ -551,8 +554,8 @@ static int rda_batched_impl(dd_ctx *ctx, const dd_fragment_desc *descs, const ui
 
     DD_CUDA(ctx, cudaMemcpyAsync(slot.dev, slot.host, (size_t)P * sizeof(DevFrag),
                                  cudaMemcpyHostToDevice, stream));
-    cudaError_t e = bf16 ? launch_rda_passes<true>(slot.dev, c, (unsigned)g, stream)
-                         : launch_rda_passes<false>(slot.dev, c, (unsigned)g, stream);
+    cudaError_t e = bf16 ? launch_rda_passes<true>(slot.dev, c, (unsigned)g, stream, only_pass)
+                         : launch_rda_passes<false>(slot.dev, c, (unsigned)g, stream, only_pass);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "rda_pass_kernel launch");
     DD_CUDA(ctx, cudaEventRecord(slot.done, stream));
     slot.used = true;
@@ -582,6 +585,22 @@ extern "C" int dd_merge_fragments_batched_rda_push(dd_ctx *ctx, const dd_fragmen
     if (P > 0 && !push_masks) return DD_ERR_INVALID_ARG;
     return rda_batched_impl(ctx, descs, push_masks, P, M, learner_dtype, outer_lr, outer_mu, flags,
                             merge_kinds, records, scratch, scratch_elems, cuda_stream);
+}
+
+extern "C" int dd_merge_fragments_batched_rda_pass(dd_ctx *ctx, const dd_fragment_desc *descs,
+                                                   const uint64_t *push_masks, int P, int M,
+                                                   dd_dtype learner_dtype, float outer_lr,
+                                                   float outer_mu, uint32_t flags,
+                                                   const uint8_t *merge_kinds, dd_merge_record *records,
+                                                   float *scratch, size_t scratch_elems, int pass,
+                                                   void *cuda_stream)
+{
+    if (pass != DD_RDA_PASS_NORMS && pass != DD_RDA_PASS_DIRECTION && pass != DD_RDA_PASS_APPLY)
+        return DD_ERR_INVALID_ARG;
+    // the passes hand their results over in memory the caller keeps between the calls
+    if (P > 0 && (!records || !scratch)) return DD_ERR_INVALID_ARG;
+    return rda_batched_impl(ctx, descs, push_masks, P, M, learner_dtype, outer_lr, outer_mu, flags,
+                            merge_kinds, records, scratch, scratch_elems, cuda_stream, pass);
 }
 
 extern "C" int dd_merge_fragment_rda(dd_ctx *ctx, float *global, float *momentum,

@@ -20,13 +20,14 @@ STATUS_OK, STATUS_QUORUM_NOT_MET, STATUS_ZERO_WEIGHT, STATUS_WAIT_LIMIT = 0, 1, 
 HEAVY_BALL, DIAG_PER_LEARNER, DIAG_STATE = 1, 2, 4
 DEBUG_EXPIRE_WAIT = 1 << 30
 MERGE_AVG, MERGE_RDA = 0, 1
+RDA_PASS_NORMS, RDA_PASS_DIRECTION, RDA_PASS_APPLY = 0, 1, 2
 FRAG_LAYER, FRAG_TENSOR, FRAG_BALANCED = 0, 1, 2
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libddmerge.so")
 
 EXPORTS = (
     "dd_create", "dd_destroy", "dd_merge_fragment", "dd_merge_fragments_batched",
-    "dd_merge_fragment_push", "dd_merge_fragments_batched_push", "dd_merge_fragments_batched_rda_push",
+    "dd_merge_fragment_push", "dd_merge_fragments_batched_push", "dd_merge_fragments_batched_rda_push", "dd_merge_fragments_batched_rda_pass",
     "dd_merge_fragment_host", "dd_merge_fragments_batched_noalloc",
     "dd_merge_fragment_rda", "dd_merge_fragments_batched_rda",
     "dd_quantize_outer_gradient_int4", "dd_merge_fragment_int4",
@@ -118,6 +119,11 @@ def _load() -> ctypes.CDLL:
         vp, ctypes.POINTER(CFragmentDesc), u64p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
         ctypes.c_float, ctypes.c_float, ctypes.c_uint32, ctypes.POINTER(ctypes.c_uint8), vp, vp,
         ctypes.c_size_t, vp]
+    lib.dd_merge_fragments_batched_rda_pass.restype = ctypes.c_int
+    lib.dd_merge_fragments_batched_rda_pass.argtypes = [
+        vp, ctypes.POINTER(CFragmentDesc), u64p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+        ctypes.c_float, ctypes.c_float, ctypes.c_uint32, ctypes.POINTER(ctypes.c_uint8), vp, vp,
+        ctypes.c_size_t, ctypes.c_int, vp]
     lib.dd_quantize_outer_gradient_int4.restype = ctypes.c_int
     lib.dd_quantize_outer_gradient_int4.argtypes = [vp, vp, vp, ctypes.c_int, ctypes.c_size_t, vp, vp, vp]
     lib.dd_merge_fragment_int4.restype = ctypes.c_int
@@ -222,6 +228,14 @@ def _stream_handle(stream) -> int | None:
     if isinstance(stream, int):
         return stream
     return int(stream.cuda_stream)
+
+
+def record_field_columns(name: str):
+    """(first, last + 1) float64 columns of ``dd_merge_record`` field ``name`` in a records buffer
+    viewed as float64 [count, RECORD_BYTES // 8] -- for summing fields across GPUs in place."""
+    f = getattr(CRecord, name)
+    assert f.offset % 8 == 0 and f.size % 8 == 0, name
+    return f.offset // 8, (f.offset + f.size) // 8
 
 
 def new_records(count: int, device=None):
@@ -366,6 +380,22 @@ class Context:
                 self._h, descs, _u64_array([int(x) & (2**64 - 1) for x in push_masks]), P, M,
                 learner_dtype, ctypes.c_float(outer_lr), ctypes.c_float(outer_mu), *tail))
 
+
+    def merge_fragments_batched_rda_pass(self, fragments, M: int, learner_dtype: int, outer_lr: float,
+                                         outer_mu: float, pass_index: int, *, records, scratch,
+                                         merge_kinds=None, flags: int = 0, push_masks=None,
+                                         stream=None) -> None:
+        """``dd_merge_fragments_batched_rda_pass``: one of the three passes (RDA_PASS_NORMS,
+        RDA_PASS_DIRECTION, RDA_PASS_APPLY) over this GPU's shard of every fragment; the caller
+        sums the hand-over fields of ``records`` across the shards between the passes."""
+        P = len(fragments)
+        descs, _keep = _pack_descs(fragments, M)
+        kinds = None if merge_kinds is None else (ctypes.c_uint8 * P)(*[int(k) for k in merge_kinds])
+        pm = None if push_masks is None else _u64_array([int(x) & (2**64 - 1) for x in push_masks])
+        self._check(lib.dd_merge_fragments_batched_rda_pass(
+            self._h, descs, pm, P, M, learner_dtype, ctypes.c_float(outer_lr), ctypes.c_float(outer_mu),
+            ctypes.c_uint32(flags), kinds, _ptr(records), _ptr(scratch),
+            ctypes.c_size_t(int(scratch.numel())), int(pass_index), _stream_handle(stream)))
     def broadcast_fragment(self, global_, learners, apply_mask: int, alpha: float = 0.0, *,
                            n: int | None = None, learner_dtype: int | None = None,
                            stream=None) -> None:

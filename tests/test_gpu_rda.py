@@ -156,3 +156,48 @@ def test_batched_mixed_avg_and_rda(dd, ctx):
             assert floor_rel_err(dev[p]["momentum"].cpu().numpy(), v) <= TOL_STATE, (k, p)
             dev[p]["global_"].copy_(torch.from_numpy(theta))
             dev[p]["momentum"].copy_(torch.from_numpy(v))
+
+
+@pytest.mark.parametrize("shards", [2, 3])
+def test_range_sharded_rda_equals_unsharded(dd, ctx, shards):
+    """A fragment cut into element ranges, as a multi-GPU job would hold it: the three passes run
+    shard by shard and the hand-over fields of the records are summed in between (here by the
+    test, on one GPU, where ranks would all-reduce).  Result: the oracle's merge of the whole
+    fragment; whole-fragment diagnostics in every shard's record."""
+    from paper_2604_21428_b200 import dist as ddist
+
+    n, M = 300_011, 5
+    tokens, mask, K = [100, 200, 0, 400, 500], 0b11101, 2
+    theta, v, learners = synth.fragment_cpu(n, M, "bf16", 4711)
+    o_theta, o_v = theta.copy(), v.copy()
+    ref = oracle.merge_fragment(o_theta, o_v, learners, tokens, mask, K, ETA, MU, merge=oracle.MERGE_RDA)
+    t_dev, v_dev = torch.from_numpy(theta).cuda(), torch.from_numpy(v).cuda()
+    l_dev = [to_torch_learner(a, "cuda") for a in learners]
+    ranges = [ddist.shard_range(n, r, shards) for r in range(shards)]
+    frags = [[dict(global_=t_dev[lo:hi], momentum=v_dev[lo:hi], learners=[t[lo:hi] for t in l_dev],
+                   tokens=tokens, quorum_mask=mask, K=K, n=hi - lo)] for lo, hi in ranges]
+    recs = [dd.new_records(1) for _ in range(shards)]
+    scratch = [torch.empty((hi - lo + 7) // 8 * 8, dtype=torch.float32, device="cuda") for lo, hi in ranges]
+
+    def all_shards_sum(parts):                     # what an all-reduce would leave on every rank
+        total = torch.stack(parts).sum(dim=0)
+        for p in parts:
+            p.copy_(total)
+
+    for p in (dd.RDA_PASS_NORMS, dd.RDA_PASS_DIRECTION, dd.RDA_PASS_APPLY):
+        for r in range(shards):
+            ctx.merge_fragments_batched_rda_pass(frags[r], M, dd.BF16, ETA, MU, p, records=recs[r],
+                                                 scratch=scratch[r], flags=dd.DIAG_STATE)
+        torch.cuda.synchronize()
+        for name in ddist.RDA_HANDOVER_FIELDS[p]:
+            a, b = dd.record_field_columns(name)
+            tables = [rec.view(torch.float64).view(-1, dd.RECORD_BYTES // 8) for rec in recs]
+            parts = [t[:, a:b].clone() for t in tables]
+            all_shards_sum(parts)
+            for t, part in zip(tables, parts):
+                t[:, a:b] = part
+    torch.cuda.synchronize()
+    assert floor_rel_err(t_dev.cpu().numpy(), o_theta) <= TOL_STATE
+    assert floor_rel_err(v_dev.cpu().numpy(), o_v) <= TOL_STATE
+    for rec in recs:
+        _check_record(dd.read_records(rec)[0], ref)

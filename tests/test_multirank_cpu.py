@@ -88,3 +88,65 @@ def test_range_sharded_merge_equals_unsharded(world, n):
 def test_whole_job_rate():
     assert ddist.whole_job_rate(500, 4, 2, 1000.0) == 4000.0
     assert ddist.max_over_ranks(3.5) == 3.5          # no process group: identity
+
+
+class _FakePassCtx:
+    """Stands in for the GPU passes of a range-sharded radial-directional merge: each pass writes
+    this rank's share of the fields it hands over and checks that the previous hand-over has been
+    summed over the ranks before it runs."""
+
+    def __init__(self, rank, world, dd):
+        self.rank, self.world, self.dd, self.calls = rank, world, dd, []
+
+    def _table(self, records):
+        return records.view(torch.float64).view(-1, self.dd.RECORD_BYTES // 8)
+
+    def merge_fragments_batched_rda_pass(self, fragments, M, learner_dtype, lr, mu, pass_index, *, records,
+                                         scratch, merge_kinds=None, flags=0, push_masks=None, stream=None):
+        dd, t, r = self.dd, self._table(records), self.rank
+        total = sum(range(1, self.world + 1))
+        a, b = dd.record_field_columns("delta_m_sq")
+        c, _ = dd.record_field_columns("delta_sq")
+        if pass_index == dd.RDA_PASS_NORMS:
+            t[:, a:a + M] = torch.arange(M, dtype=torch.float64) + (r + 1)
+        elif pass_index == dd.RDA_PASS_DIRECTION:
+            assert torch.equal(t[0, a:a + M], torch.arange(M, dtype=torch.float64) * self.world + total)
+            t[:, c] = 10.0 * (r + 1)
+        else:
+            assert float(t[0, c]) == 10.0 * total
+            assert torch.equal(t[0, a:a + M], torch.arange(M, dtype=torch.float64) * self.world + total)
+            for k, name in enumerate(("delta_sq", "theta_sq", "mom_sq")):
+                t[:, dd.record_field_columns(name)[0]] = (k + 1.0) * (r + 1)
+        self.calls.append(pass_index)
+
+
+def _rda_worker(rank, world, port, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        from paper_2604_21428_b200 import ddmerge as dd
+        P, M = 3, 4
+        records = torch.zeros(P * dd.RECORD_BYTES, dtype=torch.uint8)
+        ctx = _FakePassCtx(rank, world, dd)
+        ddist.rda_merge_range_sharded(ctx, [None] * P, M, dd.BF16, 0.7, 0.9, records=records,
+                                      scratch=torch.zeros(8))
+        t = records.view(torch.float64).view(P, dd.RECORD_BYTES // 8)
+        total = sum(range(1, world + 1))
+        ok = ctx.calls == [dd.RDA_PASS_NORMS, dd.RDA_PASS_DIRECTION, dd.RDA_PASS_APPLY]
+        for k, name in enumerate(("delta_sq", "theta_sq", "mom_sq")):
+            ok = ok and bool(torch.all(t[:, dd.record_field_columns(name)[0]] == (k + 1.0) * total))
+        a, _ = dd.record_field_columns("delta_m_sq")
+        # the norms were summed once, after the first pass, and not again at the end
+        ok = ok and torch.equal(t[1, a:a + M], torch.arange(M, dtype=torch.float64) * world + total)
+        out[rank] = bool(ok)
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_range_sharded_rda_hands_over_between_passes(world):
+    mgr = mp.Manager()
+    out = mgr.dict()
+    mp.spawn(_rda_worker, args=(world, _free_port(), out), nprocs=world, join=True)
+    assert all(out[r] for r in range(world)) and len(out) == world
