@@ -20,6 +20,15 @@ ETA, MU = synth.OUTER_LR, synth.OUTER_MU
 WINDOW = 1 << 16
 
 
+def _free_bytes():
+    """Free device memory once this process has returned what earlier tests left cached."""
+    import gc
+
+    gc.collect()
+    torch.cuda.empty_cache()
+    return torch.cuda.mem_get_info()[0]
+
+
 def _windows(n, count, rng):
     """First, last and `count` random windows (8-element aligned starts)."""
     if n <= 2 * WINDOW:
@@ -62,7 +71,7 @@ def _run(name, n_windows, merges):
     w = synth.workload(name)
     # resident: the participants' copies, Theta and v (the algorithmic bytes count Theta and v twice)
     need = w.algorithmic_bytes() - 8 * w.total_params
-    free, _ = torch.cuda.mem_get_info()
+    free = _free_bytes()
     if free < need + (4 << 30):
         pytest.skip(f"needs {need >> 30} GiB of device memory, {free >> 30} GiB free")
     dev = torch.device("cuda", 0)
@@ -148,7 +157,7 @@ def test_scale500m_full_size_int4_sampled():
 
     w = synth.workload("scale500m")
     n = w.fragment_sizes[0]
-    free, _ = torch.cuda.mem_get_info()
+    free = _free_bytes()
     if free < (24 << 30):
         pytest.skip("needs 24 GiB of device memory")
     dev = torch.device("cuda", 0)
@@ -204,7 +213,7 @@ def test_scale500m_full_size_rda_properties():
 
     w = synth.workload("scale500m")
     n = w.fragment_sizes[0]
-    free, _ = torch.cuda.mem_get_info()
+    free = _free_bytes()
     if free < (36 << 30):
         pytest.skip("needs 36 GiB of device memory")
     dev = torch.device("cuda", 0)
@@ -269,7 +278,7 @@ def test_fragment_beyond_32_bit_offsets():
     from paper_2604_21428_b200 import ddmerge as dd
 
     n = (1 << 32) + 3 * 8192 + 5
-    free, _ = torch.cuda.mem_get_info()
+    free = _free_bytes()
     if free < 10 * n + (6 << 30):
         pytest.skip("needs 46 GiB of device memory")
     dev = torch.device("cuda", 0)
@@ -311,7 +320,7 @@ def test_int4_fragment_beyond_32_bit_offsets():
     from paper_2604_21428_b200 import ddmerge as dd
 
     n = (1 << 32) + 97 * 128 + 5
-    free, _ = torch.cuda.mem_get_info()
+    free = _free_bytes()
     if free < 11 * n + (6 << 30):
         pytest.skip("needs 50 GiB of device memory")
     dev = torch.device("cuda", 0)
