@@ -361,8 +361,11 @@ def main():
         w = synth.scaled(w, args.scale, align=8)
     job_params = w.total_params * (world if args.sharding == "replica" else 1)
     if args.sharding == "range" and world > 1:
+        # int4 scales cover blocks of 128 elements: shard on block boundaries so that the sharded
+        # job quantises exactly the blocks the unsharded one would
+        align = 128 if args.merge == "int4" else 8
         w.fragment_sizes = [hi - lo for lo, hi in
-                            (ddist.shard_range(n, rank, world) for n in w.fragment_sizes)]
+                            (ddist.shard_range(n, rank, world, align) for n in w.fragment_sizes)]
     frags = build_workload(w, device, rank, args.out_bf16, args.resident)
     ctx = dd.Context(local_rank)
     grid, block, tile = ctx.launch_geometry(dd.BF16 if w.learner_dtype == "bf16" else dd.F32)
