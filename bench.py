@@ -36,6 +36,17 @@ NCU_TRAFFIC_BYTES_PER_PARAM = {
 }
 
 
+def host_cpu_model() -> str:
+    try:
+        with open("/proc/cpuinfo") as fh:
+            for ln in fh:
+                if ln.lower().startswith("model name"):
+                    return ln.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -662,7 +673,9 @@ def main():
             "value": ns / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
             "sample": f"first {ns} elements of fragment 0 of {w.name}, {len(part)} participating "
                       f"{w.learner_dtype} learners, one merge, {dt:.1f} s, single thread of "
-                      f"{os.cpu_count()} host cores"}
+                      f"{os.cpu_count()} host cores",
+            "host_cpu": host_cpu_model(), "host_cores": os.cpu_count(),
+            "affinity_cores": len(os.sched_getaffinity(0))}
         # Beside it, because the paper's own syncer is a CPU program: the same element loop
         # spread over all host cores (OpenMP; not the checked oracle, a timing baseline only).
         try:
