@@ -413,15 +413,17 @@ def test_host_buffers_entry_point(dd, ctx, n, chunk):
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
-@pytest.mark.parametrize("alpha", [0.0, 0.5, 0.25])
-def test_broadcast_to_learners(dd, ctx, dtype, alpha):
-    # learner side of an update: theta_m <- alpha theta_m + (1 - alpha) Theta'
+@pytest.mark.parametrize("alpha,shift", [(0.0, 0), (0.0, 8), (0.5, 0), (0.25, 8)])
+def test_broadcast_to_learners(dd, ctx, dtype, alpha, shift):
+    # learner side of an update: theta_m <- alpha theta_m + (1 - alpha) Theta'; copies that start
+    # on a 32-byte boundary (shift 0) take 32-byte stores, copies 16 bytes off it (shift 8) do not
     n, M = 50_003, 5
     theta, _, learners = synth.fragment_cpu(n, M, dtype, 91)
     mask = 0b10110
     t_dev = torch.from_numpy(theta).cuda()
     full = [_guarded(a.view(np.int16) if dtype == "bf16" else a,
-                     torch.int16 if dtype == "bf16" else torch.float32) for a in learners]
+                     torch.int16 if dtype == "bf16" else torch.float32,
+                     shift=shift if dtype == "bf16" else shift // 2) for a in learners]
     views = [v.view(torch.bfloat16) if dtype == "bf16" else v for _, v in full]
     ptrs = [views[m] if m != 0 else None for m in range(M)]          # learner 0: not selected, null
     ctx.broadcast_fragment(t_dev, ptrs, mask, alpha, n=n, learner_dtype=dd.BF16 if dtype == "bf16" else dd.F32)
@@ -441,6 +443,7 @@ def test_broadcast_to_learners(dd, ctx, dtype, alpha):
                 assert floor_rel_err(got, ref) <= 1e-6
         else:
             np.testing.assert_array_equal(got, ref)                # untouched
+        _check_guard(full[m][0].float(), n, shift if dtype == "bf16" else shift // 2)
 
 
 def test_bounded_wait_expires_and_context_survives(dd, ctx):
