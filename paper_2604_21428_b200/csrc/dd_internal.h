@@ -30,7 +30,7 @@ struct alignas(16) DevFrag {
     int has_steps;
     float *scratch;                      // radial-directional merge: n floats for the mean direction
     int kind;                            // DD_MERGE_AVG or DD_MERGE_RDA
-    int pad_;
+    int n_part_host;                     // |S| as the host counted it (sizes the per-lane norm area)
     unsigned long long push_mask;        // learners whose copy is overwritten with Theta' (fused push)
     unsigned long long pad2_;
     const void *ptrs[DD_MAX_LEARNERS];
@@ -49,6 +49,7 @@ struct Common {
     double *partials;                    // [P][nq][grid] per-CTA partial sums
     unsigned *tickets;                   // [P] completion counters, zero between calls
     int nq;                              // quantities per fragment in `partials`
+    int pl_cap = 0;                      // participants the per-lane norm area holds (0: none)
 };
 
 }  // namespace ddm

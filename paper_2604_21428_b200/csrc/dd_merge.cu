@@ -44,12 +44,25 @@ rda_pass_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ Commo
 
 namespace ddm {
 
+// Shared memory of the per-lane norm sums: 32 floats per warp and participant.
+static size_t pl_area_bytes(int participants) { return (size_t)participants * kWarps * 32 * sizeof(float); }
+
+// Participants the per-lane norm area must hold for a batch (0: some fragment has too many and
+// every piece is reduced at once instead).
+static int pl_capacity(const DevFrag *frags, int P, bool rda_only)
+{
+    int cap = 0;
+    for (int p = 0; p < P; ++p)
+        if (!rda_only || frags[p].kind == DD_MERGE_RDA) cap = frags[p].n_part_host > cap ? frags[p].n_part_host : cap;
+    return cap <= kPlMaxParticipants ? cap : 0;
+}
+
 // Opts a kernel in to its dynamic shared memory and reports how many CTAs fit on an SM.
 template <typename K>
 static cudaError_t prepare_kernel(K kernel, int *blocks)
 {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)kTmaRingBytes);
+                                         (int)(kTmaRingBytes + pl_area_bytes(kPlMaxParticipants)));
     int b = 0;
     if (e == cudaSuccess)
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kernel, kThreads, kTmaRingBytes);
@@ -111,6 +124,7 @@ int fill_fragment(DevFrag &d, float *global, float *momentum, void *out_bf16,
         const bool takes_part = ((d.mask >> m) & 1ull) && tokens[m] > 0;
         // the kernel sums the participants' token counts exactly, in 64 bits
         if (takes_part && __builtin_add_overflow(token_sum, tokens[m], &token_sum)) return DD_ERR_INVALID_ARG;
+        if (takes_part) ++d.n_part_host;
         if (takes_part && n > 0) {
             const void *p = learner_ptrs[m];
             if (!p) return DD_ERR_INVALID_ARG;
@@ -219,10 +233,11 @@ template <bool BF16, bool PL>
 static cudaError_t launch(bool single, const DevFrag *one, const DevFrag *dev_frags,
                           const Common &c, unsigned grid, cudaStream_t stream)
 {
+    const size_t smem = kTmaRingBytes + pl_area_bytes(c.pl_cap);
     if (single)
-        merge_single_tma_kernel<BF16, PL><<<grid, kThreads, kTmaRingBytes, stream>>>(*one, c);
+        merge_single_tma_kernel<BF16, PL><<<grid, kThreads, smem, stream>>>(*one, c);
     else
-        merge_batched_tma_kernel<BF16, PL><<<grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
+        merge_batched_tma_kernel<BF16, PL><<<grid, kThreads, smem, stream>>>(dev_frags, c);
     return cudaGetLastError();
 }
 
@@ -323,6 +338,7 @@ static int merge_fragment_impl(dd_ctx *ctx, float *global, float *momentum,
     c.total_tiles = frag.tile_end;
     c.records = record;
     c.nq = kNumScalarDiag + (pl ? M : 0);
+    if (pl && frag.n_part_host <= kPlMaxParticipants) c.pl_cap = frag.n_part_host;
     if (record) {
         rc = ensure_workspace(ctx, 1, (size_t)c.nq, (size_t)ctx->grid[bf16][pl]);
         if (rc != DD_OK) return rc;
@@ -404,6 +420,7 @@ static int merge_batched_impl(dd_ctx *ctx, const dd_fragment_desc *descs, const 
     c.total_tiles = tile;
     c.records = records;
     c.nq = kNumScalarDiag + (pl ? M : 0);
+    if (pl) c.pl_cap = pl_capacity(slot.host, P, false);
     if (records) {
         rc = ensure_workspace(ctx, (size_t)P, (size_t)c.nq, (size_t)ctx->grid[bf16][pl]);
         if (rc != DD_OK) return rc;
@@ -448,7 +465,7 @@ static cudaError_t launch_rda_passes(const DevFrag *dev_frags, const Common &c, 
                                      cudaStream_t stream, int only_pass)
 {
     if (only_pass < 0 || only_pass == DD_RDA_PASS_NORMS)
-        rda_pass_kernel<BF16, kModeNorms><<<grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
+        rda_pass_kernel<BF16, kModeNorms><<<grid, kThreads, kTmaRingBytes + pl_area_bytes(c.pl_cap), stream>>>(dev_frags, c);
     if (only_pass < 0 || only_pass == DD_RDA_PASS_DIRECTION)
         rda_pass_kernel<BF16, kModeDir><<<grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
     if (only_pass < 0 || only_pass == DD_RDA_PASS_APPLY)
@@ -547,6 +564,7 @@ static int rda_batched_impl(dd_ctx *ctx, const dd_fragment_desc *descs, const ui
     c.total_tiles = tile;
     c.records = records;
     c.nq = kNumScalarDiag + M;
+    c.pl_cap = pl_capacity(slot.host, P, true);
     rc = ensure_workspace(ctx, (size_t)P, (size_t)c.nq, (size_t)ctx->grid[bf16][1]);
     if (rc != DD_OK) return rc;
     c.partials = ctx->partials;

@@ -27,6 +27,8 @@ constexpr int kTmaStages = DD_TMA_STAGES;
 constexpr int kTmaChunk = 2048;                           // bytes per slot / per bulk copy
 constexpr int kSuperRow = 1024;                           // elements a warp merges per round (4 steps per lane)
 constexpr size_t kTmaRingBytes = (size_t)kWarps * kTmaStages * kTmaChunk;
+constexpr int kPlMaxParticipants = 48;                    // per-lane norm area: 1 KB per participant per CTA
+constexpr int kPlFlushRows = 128;                         // rounds a lane sums in fp32 before the fp64 hand-over
 constexpr int kWaitLimit = 1 << 18;                       // try_wait attempts before giving up
 constexpr unsigned kWaitHintNs = 4000;                    // each attempt may sleep this long (~1 s in all)
 static_assert(kTileElems == kWarps * kSuperRow, "one super-row per warp per tile");
@@ -107,6 +109,22 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
     const int s = sm.n_part;
     constexpr bool kHasV = MODE == kModeMerge || MODE == kModeApply;
     constexpr bool kNorms = PL || MODE == kModeNorms;
+    // Per-participant squared norms: every lane keeps its own fp32 sum per participant in shared
+    // memory (behind the rings) and the warp reduces them once per kPlFlushRows rounds, not once
+    // per piece; without the area (more than kPlMaxParticipants) each piece is reduced at once.
+    float *const pl = kNorms && c.pl_cap > 0 && sm.n_part <= c.pl_cap
+                          ? reinterpret_cast<float *>(ring_base + kTmaRingBytes) + (size_t)warp * c.pl_cap * 32
+                          : nullptr;
+    int pl_rows = 0;
+    auto pl_flush = [&]() {
+        for (int j = 0; j < sm.n_part; ++j) {
+            float t = pl[j * 32 + lane];
+            pl[j * 32 + lane] = 0.0f;
+            t = warp_sum(t);
+            if (lane == 0) sm.dm[warp][j] += (double)t;
+        }
+        pl_rows = 0;
+    };
     const int nmid = MODE == kModeApply ? 2 : s * LB;      // pieces between Theta and v
     const int npieces = 2 + nmid + (kHasV ? 2 : 0);
     const float *const theta = sm.theta;
@@ -218,23 +236,23 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
             for (int j = 0; j < s; ++j) {
                 const float w = sm.w[j];
                 const float2 w2 = make_float2(w, w);
-                float q = 0.0f;
+                float2 q2 = make_float2(0.0f, 0.0f);
                 if (BF16) {
                     const unsigned char *slot = acquire();
 #pragma unroll
                     for (int r = 0; r < 4; ++r) {
                         const uint4 x = *reinterpret_cast<const uint4 *>(slot + r * 512 + lane * 16);
                         const unsigned word[4] = {x.x, x.y, x.z, x.w};
-                        float qr = 0.0f;
+                        float2 qr = make_float2(0.0f, 0.0f);
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
                             const float2 th = make_float2(__uint_as_float(word[k] << 16),
                                                           __uint_as_float(word[k] & 0xffff0000u));
                             const float2 d = __fadd2_rn(th, nT[r][k]);
                             if (MODE != kModeNorms) acc[r][k] = __ffma2_rn(w2, d, acc[r][k]);
-                            if (kNorms) qr = fmaf(d.x, d.x, fmaf(d.y, d.y, qr));
+                            if (kNorms) qr = __ffma2_rn(d, d, qr);          // even / odd elements side by side
                         }
-                        if (kNorms && (unsigned)(r * 32 + lane) < cnt) q += qr;
+                        if (kNorms && (unsigned)(r * 32 + lane) < cnt) q2 = __fadd2_rn(q2, qr);
                     }
                     release();
                 } else {
@@ -250,24 +268,30 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
                                                   make_float2(__uint_as_float(a.z), __uint_as_float(a.w)),
                                                   make_float2(__uint_as_float(b.x), __uint_as_float(b.y)),
                                                   make_float2(__uint_as_float(b.z), __uint_as_float(b.w))};
-                            float qr = 0.0f;
+                            float2 qr = make_float2(0.0f, 0.0f);
 #pragma unroll
                             for (int k = 0; k < 4; ++k) {
                                 const float2 d = __fadd2_rn(th[k], nT[r][k]);
                                 if (MODE != kModeNorms) acc[r][k] = __ffma2_rn(w2, d, acc[r][k]);
-                                if (kNorms) qr = fmaf(d.x, d.x, fmaf(d.y, d.y, qr));
+                                if (kNorms) qr = __ffma2_rn(d, d, qr);
                             }
-                            if (kNorms && (unsigned)(r * 32 + lane) < cnt) q += qr;
+                            if (kNorms && (unsigned)(r * 32 + lane) < cnt) q2 = __fadd2_rn(q2, qr);
                         }
                         release();
                     }
                 }
                 if (kNorms && !rs.failed) {
-                    q = warp_sum(q);
-                    if (lane == 0) sm.dm[warp][j] += (double)q;
+                    float q = q2.x + q2.y;
+                    if (pl != nullptr) {
+                        pl[j * 32 + lane] += q;
+                    } else {
+                        q = warp_sum(q);
+                        if (lane == 0) sm.dm[warp][j] += (double)q;
+                    }
                 }
             }
         }
+        if (kNorms && pl != nullptr && ++pl_rows == kPlFlushRows) pl_flush();
         if (MODE == kModeNorms) continue;
 
         float dsq = 0.0f, tsq = 0.0f, msq = 0.0f;
@@ -348,6 +372,7 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
         }
     }
 
+    if (kNorms && pl != nullptr && pl_rows > 0) pl_flush();
     if (rs.failed) {
         // Give the copies still in flight a bounded chance to land before this
         // warp's slots can be reused or the CTA exits, and say what happened.
@@ -372,6 +397,9 @@ __device__ __forceinline__ void merge_body_tma(const DevFrag *frags, const Commo
     extern __shared__ __align__(128) unsigned char ring_base[];
     const unsigned G = gridDim.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if ((PL || MODE == kModeNorms) && c.pl_cap > 0)   // per-lane norm sums start at zero (and are left so)
+        for (int i = threadIdx.x; i < c.pl_cap * kWarps * 32; i += kThreads)
+            reinterpret_cast<float *>(ring_base + kTmaRingBytes)[i] = 0.0f;
     if (lane == 0)
         for (int d = 0; d < kTmaStages; ++d) mbar_init(bars + warp * kTmaStages + d, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");

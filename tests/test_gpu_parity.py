@@ -646,3 +646,13 @@ def test_bitwise_reproducible_run_to_run(dd, ctx):
             first = got
         else:
             assert all(torch.equal(a, b) for a, b in zip(first, got)), rep
+
+
+@pytest.mark.parametrize("s", [47, 48, 49])
+def test_per_learner_norms_around_the_shared_memory_limit(dd, ctx, s):
+    """Up to 48 participants the per-participant norms are summed per lane in shared memory and
+    reduced once per run of rows; beyond, every piece is reduced at once.  Same result."""
+    M = 52
+    tokens = [100 + 3 * m for m in range(M)]
+    run_case(dd, ctx, 3 * 8192 + 70_001, M, "bf16", tokens, (1 << s) - 1, s, seed=300 + s,
+             flags=dd.DIAG_STATE | dd.DIAG_PER_LEARNER, merges=1)
