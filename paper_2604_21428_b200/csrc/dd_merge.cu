@@ -155,8 +155,9 @@ static int set_push(DevFrag &d, const void *const *learner_ptrs, uint64_t push_m
         if (misaligned(p)) return DD_ERR_ALIGNMENT;
         if (overlaps(p, lb, d.theta, 4 * n) || overlaps(p, lb, d.mom, 4 * n) || overlaps(p, lb, d.out_bf16, 2 * n))
             return DD_ERR_ALIAS;
-        for (int k = 0; k < m; ++k)        // two pushed (or read) copies sharing memory would race
-            if (learner_ptrs[k] && (((pm >> k) & 1ull) || (((d.mask >> k) & 1ull) && d.tokens[k] > 0)) &&
+        for (int k = 0; k < M; ++k)        // a pushed copy sharing memory with another pushed or read copy would race
+            if (k != m && learner_ptrs[k] &&
+                (((pm >> k) & 1ull) || (((d.mask >> k) & 1ull) && d.tokens[k] > 0)) &&
                 overlaps(p, lb, learner_ptrs[k], lb))
                 return DD_ERR_ALIAS;
     }

@@ -146,6 +146,11 @@ def test_push_argument_validation(dd, ctx):
         ctx.merge_fragment_push(t_dev, v_dev, [l_dev[0], l_dev[1], l_dev[1]], tokens, 0b001, 1, ETA, MU, 0b110,
                                 n=n, learner_dtype=dd.BF16)
     assert e.value.rc == dd.ERR_ALIAS
+    # a pushed learner sharing its buffer with a later learner that is only read
+    with pytest.raises(dd.DDMergeError) as e:
+        ctx.merge_fragment_push(t_dev, v_dev, [l_dev[0], l_dev[1], l_dev[0]], tokens, 0b100, 1, ETA, MU, 0b001,
+                                n=n, learner_dtype=dd.BF16)
+    assert e.value.rc == dd.ERR_ALIAS
     # bits at or above M are ignored
     ctx.merge_fragment_push(t_dev, v_dev, l_dev, tokens, 0b111, 1, ETA, MU, 0b1000, n=n, learner_dtype=dd.BF16)
     torch.cuda.synchronize()
