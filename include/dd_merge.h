@@ -71,11 +71,13 @@ enum {
     DD_HEAVY_BALL = 1u << 0,        /* Theta' = Theta - lr v' instead of the Nesterov form */
     DD_DIAG_PER_LEARNER = 1u << 1,  /* also ||Theta - theta_m||^2 for every participant */
     DD_DIAG_STATE = 1u << 2,        /* also ||Theta'||^2 and ||v'||^2 */
-    /* Test hook for the error path, not for production: every warp's first bulk copy
-     * is made to wait for bytes that never come, so its bounded wait expires (about a
-     * second), the fragment's record reports DD_STATUS_WAIT_LIMIT and the kernel
-     * returns normally with the context still usable.  Needs a record; the
-     * fragment's state is unspecified afterwards. */
+    /* Test hook for the error path.  Production callers must never set it: every warp's
+     * first bulk copy is made to wait for bytes that never come, so its bounded wait
+     * expires (about a second, up to three for the launch), every fragment the launch
+     * could not finish reports DD_STATUS_WAIT_LIMIT in its record and the kernel returns
+     * normally with the context still usable.  Needs records; the state of those
+     * fragments is unspecified afterwards.  Rejected by the int4 and allocation-free
+     * entry points. */
     DD_DEBUG_EXPIRE_WAIT = 1u << 30
 };
 
@@ -131,10 +133,13 @@ int dd_destroy(dd_ctx *ctx);
  *                     Theta' (the payload broadcast back to the learners)
  *   record            [device] optional; without it no diagnostics are computed
  *
- * The call enqueues one kernel on cuda_stream and returns.  The first call that
- * passes a record allocates the context's workspace; from then on the call
- * neither allocates nor synchronises, so it may be recorded into a CUDA graph by
- * stream capture (host arrays are consumed before it returns).
+ * The call enqueues one kernel on cuda_stream and returns.  The first call on a
+ * context that passes a record allocates the context's diagnostics workspace, sized
+ * once for any single-fragment call (every M, every flag); from then on
+ * dd_merge_fragment neither allocates nor synchronises, so it may be recorded into
+ * a CUDA graph by stream capture (host arrays are consumed before it returns).
+ * Only a batched call with many fragments can make the workspace grow later, which
+ * synchronises the device.
  */
 int dd_merge_fragment(dd_ctx *ctx, float *global, float *momentum,
                       const void *const *learner_ptrs, int M, dd_dtype learner_dtype,
@@ -286,6 +291,10 @@ int dd_merge_fragments_batched_rda_pass(dd_ctx *ctx, const dd_fragment_desc *des
  *   - D = Theta - theta_m in float32; scale = max|D| / 7 (float32), one per block;
  *   - code = D / scale rounded to nearest (ties to even), clamped to [-7, 7]; a block of
  *     zeros has scale 0 and codes 0;
+ *   - a non-finite D poisons its block, as it would poison an uncompressed merge: a NaN
+ *     makes the block's scale NaN (all codes 0), an infinity makes it infinite (finite
+ *     elements get code 0, infinite ones -7), so every element of the block decodes to a
+ *     non-finite value; other blocks are unaffected;
  *   - element i's code + 8 sits in nibble (i & 1) of byte i / 2 (even element low).
  *
  * dd_quantize_outer_gradient_int4 is the learner side:
@@ -353,9 +362,13 @@ int dd_merge_fragment_host(dd_ctx *ctx, float *global, float *momentum,
  *   - P <= DD_NOALLOC_MAX_FRAGMENTS, else DD_ERR_TOO_LARGE (nothing is launched);
  *   - DD_DIAG_PER_LEARNER is not offered (DD_ERR_INVALID_ARG);
  *   - the grid is capped at 592 CTAs.
- * The first call on a device resolves the array's device address (one
- * cudaGetSymbolAddress) and sizes the grid; make that first call before any
- * stream capture begins.  All calls on a device share the one array, and it
+ * The first call on a device does the set-up: it resolves the array's device
+ * address (one cudaGetSymbolAddress) and sizes the grid; with lazy module
+ * loading it is also the moment the CUDA runtime loads this library's device
+ * image, array included, onto that GPU, which can fail on a GPU that is already
+ * full.  Make that first call at start-up, and before any stream capture
+ * begins.  (Nothing is said here, either way, about recording later calls by
+ * stream capture.)  All calls on a device share the one array, and it
  * keeps the previous call's contents: the call itself clears what has to start
  * at zero, but two calls that overlap on the GPU (different streams, or
  * different host threads without ordering) race on it and give wrong results.

@@ -279,6 +279,10 @@ void ddo_apply_to_learner(void *learner, int learner_is_bf16, const float *Theta
  * scale = max|D| / 7 per block, code = round-half-even(D / scale) clamped to
  * [-7, 7], stored as code + 8 in a nibble (even element in the low nibble).
  * Every decision is taken in float32, the precision the kernel uses.
+ * Non-finite differences poison their block, as IEEE arithmetic would poison the
+ * uncompressed merge: a NaN difference makes the block's scale NaN (codes 0), an
+ * infinite one makes it infinite (a NaN quotient is coded -7), and either way every
+ * element of the block decodes to a non-finite value.
  */
 #define DDO_INT4_BLOCK 128
 
@@ -295,7 +299,7 @@ void ddo_quantize_int4(const float *Theta, const void *learner, int learner_is_b
                                        : ((const float *)learner)[i];
             float d = Theta[i] - th;
             float a = fabsf(d);
-            if (a > amax) amax = a;
+            if (isnan(a) || a > amax) amax = a;      /* a NaN in the block makes its scale NaN */
         }
         scale = amax / 7.0f;
         scales[b] = scale;
@@ -306,7 +310,7 @@ void ddo_quantize_int4(const float *Theta, const void *learner, int learner_is_b
             float q = scale > 0.0f ? rintf(d / scale) : 0.0f;
             int code;
             if (q > 7.0f) q = 7.0f;
-            if (q < -7.0f) q = -7.0f;
+            if (!(q >= -7.0f)) q = -7.0f;            /* also a NaN quotient (infinite D over infinite scale) */
             code = (int)q + 8;
             codes[i / 2] |= (uint8_t)(code << (4 * (i & 1)));
         }

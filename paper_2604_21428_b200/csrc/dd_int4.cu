@@ -55,9 +55,11 @@ quantize_int4_kernel(const float *__restrict__ theta, const void *__restrict__ l
             for (int u = 0; u < kQuantUnroll; ++u) {
                 const float d[4] = {__fsub_rn(t4[u].x, l4[u].x), __fsub_rn(t4[u].y, l4[u].y),
                                     __fsub_rn(t4[u].z, l4[u].z), __fsub_rn(t4[u].w, l4[u].w)};
-                // |d| is never NaN here (fmaxf drops it), so the maximum of the bit patterns is the maximum
-                float amax = fmaxf(fmaxf(fabsf(d[0]), fabsf(d[1])), fmaxf(fabsf(d[2]), fabsf(d[3])));
-                amax = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(amax)));
+                // The block maximum is taken on the bit patterns of |d|: they order like the values, and
+                // a NaN (pattern above infinity's) wins, so a block that holds a NaN gets a NaN scale.
+                const unsigned amax_bits = max(max(__float_as_uint(fabsf(d[0])), __float_as_uint(fabsf(d[1]))),
+                                               max(__float_as_uint(fabsf(d[2])), __float_as_uint(fabsf(d[3]))));
+                const float amax = __uint_as_float(__reduce_max_sync(0xffffffffu, amax_bits));
                 const float scale = __fdiv_rn(amax, 7.0f);
                 if (lane == 0) scales[b + u * warps] = scale;
                 // round(d / scale) without a division per element: q0 = d * (1 / scale) is within
@@ -92,7 +94,7 @@ quantize_int4_kernel(const float *__restrict__ theta, const void *__restrict__ l
     for (; b < nblocks; b += warps) {
         const unsigned long long e0 = b * kInt4Block + 4ull * lane;
         float d[4], T[4], th[4];
-        float amax = 0.0f;
+        unsigned amax_bits = 0u;
         if (vec_ok && e0 + 3 < n) {
             // 16 bytes of Theta and 8 (bf16) or 16 (fp32) bytes of the learner copy per lane
             const float4 t4 = __ldcs(reinterpret_cast<const float4 *>(theta + e0));
@@ -122,10 +124,9 @@ quantize_int4_kernel(const float *__restrict__ theta, const void *__restrict__ l
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             d[k] = __fsub_rn(T[k], th[k]);
-            amax = fmaxf(amax, fabsf(d[k]));
+            amax_bits = max(amax_bits, __float_as_uint(fabsf(d[k])));     // NaN wins, as above
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+        const float amax = __uint_as_float(__reduce_max_sync(0xffffffffu, amax_bits));
         const float scale = __fdiv_rn(amax, 7.0f);
         if (lane == 0) scales[b] = scale;
         unsigned packed = 0;

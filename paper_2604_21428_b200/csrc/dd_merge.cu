@@ -184,10 +184,14 @@ int check_common(const dd_ctx *ctx, int M, dd_dtype dtype, float lr, float mu, u
 }
 
 // Grows the diagnostics workspace; growth waits for the device to drain because
-// kernels in flight may still use the old one.
+// kernels in flight may still use the old one.  The first allocation already covers
+// every single-fragment call (any M, any flags, any of the library's grids), so only
+// a batch of many fragments can make it grow again.
 int ensure_workspace(dd_ctx *ctx, size_t P, size_t nq, size_t grid)
 {
-    const size_t need = P * nq * grid;
+    size_t need = P * nq * grid;
+    const size_t single_max = (size_t)(kNumScalarDiag + DD_MAX_LEARNERS) * (size_t)ctx->sm_count * 4;
+    if (need < single_max) need = single_max;
     if (need > ctx->partials_cap) {
         DD_CUDA(ctx, cudaDeviceSynchronize());
         if (ctx->partials) cudaFree(ctx->partials);

@@ -42,6 +42,7 @@ struct Smem {
     float cscale;                        // RDA apply: Delta = cscale * u
     void *push[DD_MAX_LEARNERS];         // copies that receive Theta' (compacted)
     int n_push;
+    int any_failed;                      // a warp of this CTA gave up a bounded wait in (or before) this fragment
     double red[kWarps][kNumScalarDiag];  // per-warp ||Delta||^2, ||Theta'||^2, ||v'||^2 of this fragment
     double dm[kWarps][DD_MAX_LEARNERS];  // per-warp per-participant ||Theta-theta_m||^2
 };
@@ -189,6 +190,7 @@ __device__ __forceinline__ void load_header(const DevFrag *f, int p, unsigned lo
         sm.kind = f->kind;
         sm.scratch = f->scratch;
         sm.cscale = 0.0f;
+        sm.any_failed = 0;
     }
     for (int j = lane; j < kWarps * DD_MAX_LEARNERS; j += 32) (&sm.dm[0][0])[j] = 0.0;
     if (lane < kWarps * kNumScalarDiag) (&sm.red[0][0])[lane] = 0.0;
@@ -300,7 +302,12 @@ __device__ __forceinline__ void process_tail(Smem &sm, const Common &c, unsigned
 // Wait-free: every CTA that worked on the fragment stores its partial sums,
 // fences, and draws a ticket; the CTA that draws the last ticket adds the
 // partials in a fixed order (so the result does not depend on CTA timing) and
-// re-arms the ticket for the next call.
+// re-arms the ticket for the next call.  The ticket word's top bit carries "some
+// CTA gave up a bounded wait in this fragment": a CTA sets it before it draws its
+// ticket, so the last CTA sees it from every CTA and reports DD_STATUS_WAIT_LIMIT
+// after the header (written by the CTA of the fragment's first tile) is in place.
+constexpr unsigned kTicketFailedBit = 0x80000000u;
+
 template <bool PL>
 __device__ __forceinline__ void flush_fragment(Smem &sm, const Common &c)
 {
@@ -328,8 +335,10 @@ __device__ __forceinline__ void flush_fragment(Smem &sm, const Common &c)
     const unsigned long long ntiles = sm.tile_end - sm.tile_begin;
     if (threadIdx.x == 0) {
         const unsigned expected = ntiles < G ? (unsigned)ntiles : G;
+        if (sm.any_failed) atomicOr(c.tickets + p, kTicketFailedBit);
         const unsigned ticket = atomicAdd(c.tickets + p, 1u);
-        sm.is_last = ticket == expected - 1u;
+        sm.is_last = (ticket & ~kTicketFailedBit) == expected - 1u;
+        if (ticket & kTicketFailedBit) sm.any_failed = 1;
     }
     __syncthreads();
     if (!sm.is_last) return;
@@ -351,7 +360,10 @@ __device__ __forceinline__ void flush_fragment(Smem &sm, const Common &c)
             else rec->delta_m_sq[q - kNumScalarDiag] = t;
         }
     }
-    if (threadIdx.x == 0) c.tickets[p] = 0u;
+    if (threadIdx.x == 0) {
+        if (sm.any_failed) rec->status = DD_STATUS_WAIT_LIMIT;
+        c.tickets[p] = 0u;
+    }
 }
 
 }  // namespace ddm

@@ -381,7 +381,7 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
             if (++rs.cslot == kTmaStages) { rs.cslot = 0; rs.cphase ^= 1u; }
         }
         rs.islot = rs.cslot;
-        if (lane == 0 && c.records != nullptr) atomicMax(&c.records[sm.frag].status, (int)DD_STATUS_WAIT_LIMIT);
+        if (lane == 0) sm.any_failed = 1;       // reported through the fragment's ticket (flush_fragment)
     }
 }
 
@@ -424,6 +424,11 @@ __device__ __forceinline__ void merge_body_tma(const DevFrag *frags, const Commo
         const bool plain = MODE == kModeMerge || (MODE == kModeApply && sm.kind == DD_MERGE_AVG);
         const bool worked_on = sm.status == DD_STATUS_OK && (plain || sm.kind == DD_MERGE_RDA);
         if (worked_on) {
+            // A warp whose ring failed in an earlier fragment skips its rows of this one too: the
+            // fragment is incomplete and must say so.
+            if (rs.failed && lane == 0 &&
+                ((tile - sm.tile_begin) * kWarps + (unsigned)warp) * (unsigned long long)(kSuperRow / kVec) < sm.n / kVec)
+                sm.any_failed = 1;
             const int rem = (int)(sm.n % kVec);
             const bool owns_tail = rem != 0 && warp == 0 && tile + (mine - 1) * G == tile_end - 1;
             float dsq = 0.0f, tsq = 0.0f, msq = 0.0f;

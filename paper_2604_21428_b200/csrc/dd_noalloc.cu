@@ -15,6 +15,7 @@
 #include <cuda_runtime.h>
 
 #include "dd_merge_tma.cuh"
+#include "dd_ctx.h"
 
 namespace ddm {
 namespace noalloc {
@@ -102,55 +103,6 @@ static int setup_current_device(DeviceState **out)
     return DD_OK;
 }
 
-static bool overlaps(const void *a, size_t abytes, const void *b, size_t bbytes)
-{
-    if (!a || !b || abytes == 0 || bbytes == 0) return false;
-    const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
-    return a0 < b0 + bbytes && b0 < a0 + abytes;
-}
-
-static bool misaligned(const void *p) { return ((uintptr_t)p & 15u) != 0; }
-
-// Same argument rules as the other entry points.
-static int fill(DevFrag &d, const dd_fragment_desc &f, int M, dd_dtype dtype)
-{
-    if (!f.learner_ptrs || !f.tokens || f.K < 0 || f.K > M) return DD_ERR_INVALID_ARG;
-    if (f.n > 0 && (!f.global || !f.momentum)) return DD_ERR_INVALID_ARG;
-    if (f.n > kMaxFragmentElems) return DD_ERR_TOO_LARGE;
-    if (misaligned(f.global) || misaligned(f.momentum) || misaligned(f.out_bf16)) return DD_ERR_ALIGNMENT;
-    const size_t n = (size_t)f.n, lb = (dtype == DD_BF16 ? 2u : 4u) * n;
-    if (overlaps(f.global, 4 * n, f.momentum, 4 * n) || overlaps(f.global, 4 * n, f.out_bf16, 2 * n) ||
-        overlaps(f.momentum, 4 * n, f.out_bf16, 2 * n))
-        return DD_ERR_ALIAS;
-    std::memset(&d, 0, sizeof d);
-    d.theta = f.global;
-    d.mom = f.momentum;
-    d.out_bf16 = static_cast<uint16_t *>(f.out_bf16);
-    d.n = f.n;
-    d.mask = M >= 64 ? f.quorum_mask : (f.quorum_mask & ((1ull << M) - 1ull));
-    d.K = f.K;
-    d.has_steps = f.steps != nullptr;
-    uint64_t token_sum = 0;
-    for (int m = 0; m < M; ++m) {
-        d.tokens[m] = f.tokens[m];
-        d.steps[m] = f.steps ? f.steps[m] : 0;
-        d.ptrs[m] = f.learner_ptrs[m];
-        if (f.steps && f.tokens[m] > 0 && f.steps[m] == 0) return DD_ERR_INVALID_ARG;
-        if (((d.mask >> m) & 1ull) && f.tokens[m] > 0 &&
-            __builtin_add_overflow(token_sum, f.tokens[m], &token_sum))
-            return DD_ERR_INVALID_ARG;
-        if (((d.mask >> m) & 1ull) && f.tokens[m] > 0 && n > 0) {
-            const void *p = f.learner_ptrs[m];
-            if (!p) return DD_ERR_INVALID_ARG;
-            if (misaligned(p)) return DD_ERR_ALIGNMENT;
-            if (overlaps(p, lb, f.global, 4 * n) || overlaps(p, lb, f.momentum, 4 * n) ||
-                overlaps(p, lb, f.out_bf16, 2 * n))
-                return DD_ERR_ALIAS;
-        }
-    }
-    return DD_OK;
-}
-
 }  // namespace noalloc
 }  // namespace ddm
 
@@ -180,7 +132,9 @@ extern "C" int dd_merge_fragments_batched_noalloc(const dd_fragment_desc *descs,
     static thread_local DevFrag host_frags[kMaxFragments];
     unsigned long long tile = 0;
     for (int p = 0; p < P; ++p) {
-        rc = fill(host_frags[p], descs[p], M, learner_dtype);
+        const dd_fragment_desc &d = descs[p];
+        rc = fill_fragment(host_frags[p], d.global, d.momentum, d.out_bf16, d.learner_ptrs, d.tokens, d.steps,
+                           d.quorum_mask, d.K, d.n, M, (learner_dtype == DD_BF16 ? 2u : 4u) * (size_t)d.n);
         if (rc != DD_OK) return rc;
         host_frags[p].tile_begin = tile;
         const unsigned long long t = (descs[p].n + kTileElems - 1) / kTileElems;

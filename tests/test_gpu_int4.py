@@ -55,6 +55,47 @@ def test_quantiser_bit_exact(dd, ctx, n, dtype):
     np.testing.assert_array_equal(codes.cpu().numpy(), ref_codes)
 
 
+@pytest.mark.parametrize("shift", [0, 1])
+def test_quantiser_non_finite_blocks(dd, ctx, shift):
+    """Blocks holding NaN or infinite differences: a NaN makes the block's scale NaN, an
+    infinity makes it infinite, whichever loop of the kernel handles the block (the unrolled
+    one, the one-block one, the unaligned one reached through ``shift``).  NaN scales are
+    compared as NaN, everything else bit for bit."""
+    nblocks = 4 * 8 * 148 * 8 + 37                      # several rounds of the unrolled loop + a rest
+    n = nblocks * 128 - 5
+    rng = np.random.default_rng(77)
+    theta = np.zeros(n, dtype=np.float32)
+    learner = rng.normal(0.0, 1e-3, size=n).astype(np.float32)
+    for b in range(0, nblocks, 3):
+        lo = b * 128
+        kind = (b // 3) % 4
+        if kind == 0:
+            learner[lo + 5] = np.nan                    # one NaN
+        elif kind == 1:
+            learner[lo + 4:lo + 8] = np.nan             # a lane's four elements all NaN
+        elif kind == 2:
+            learner[lo + 9] = np.inf                    # infinity (and finite neighbours)
+        else:
+            learner[lo + 17] = -np.inf
+            learner[lo + 18] = np.nan
+    ref_codes, ref_scales = oracle.quantize_int4(theta, learner)
+    # device buffers moved off 16-byte alignment by ``shift`` elements
+    t_full = torch.zeros(n + 8, dtype=torch.float32, device="cuda")
+    l_full = torch.zeros(n + 8, dtype=torch.float32, device="cuda")
+    t_dev, l_dev = t_full[shift:shift + n], l_full[shift:shift + n]
+    l_dev.copy_(torch.from_numpy(learner))
+    codes = torch.zeros((n + 1) // 2, dtype=torch.uint8, device="cuda")
+    scales = torch.zeros(nblocks, dtype=torch.float32, device="cuda")
+    ctx.quantize_outer_gradient_int4(t_dev, l_dev, codes, scales, n=n, learner_dtype=dd.F32)
+    torch.cuda.synchronize()
+    got_s = scales.cpu().numpy()
+    assert np.array_equal(np.isnan(got_s), np.isnan(ref_scales)) and np.isnan(ref_scales).sum() > 100
+    fin = ~np.isnan(ref_scales)
+    np.testing.assert_array_equal(got_s[fin].view(np.uint32), ref_scales[fin].view(np.uint32))
+    assert np.isinf(ref_scales).sum() > 100
+    np.testing.assert_array_equal(codes.cpu().numpy(), ref_codes)
+
+
 def test_quantiser_near_ties_and_extreme_scales(dd, ctx):
     """Outer gradients placed on, and one to three ulps beside, the half-integer multiples of
     the block scale -- where rint(d / scale) decides between two codes -- and blocks whose

@@ -472,6 +472,40 @@ def test_bounded_wait_expires_and_context_survives(dd, ctx):
     assert floor_rel_err(v_dev.cpu().numpy(), v) <= TOL_STATE
 
 
+def test_bounded_wait_expiry_marks_every_incomplete_fragment_of_a_batch(dd, ctx):
+    # Five fragments of 100 tiles on a grid of at most 296 CTAs: most CTAs own tiles of two
+    # fragments.  With the hook every warp gives up in the first fragment it works on and skips
+    # its rows of the later ones, so every fragment is incomplete and must say so (a fragment
+    # left at status 0 would present partial norms as valid).
+    grid, _, tile = ctx.launch_geometry(dd.BF16)
+    P, M, n = 5, 3, 100 * tile
+    assert P * 100 > grid
+    frags, hosts = [], []
+    for p in range(P):
+        theta, v, learners = synth.fragment_cpu(n, M, "bf16", 70 + p)
+        hosts.append((theta, v, learners))
+        frags.append(dict(global_=torch.from_numpy(theta).cuda(), momentum=torch.from_numpy(v).cuda(),
+                          learners=[to_torch_learner(a, "cuda") for a in learners],
+                          tokens=[1 + p, 2, 3], quorum_mask=0b111, K=1, n=n))
+    rec_buf = dd.new_records(P)
+    ctx.merge_fragments_batched(frags, M, dd.BF16, ETA, MU, flags=dd.DEBUG_EXPIRE_WAIT, records=rec_buf)
+    torch.cuda.synchronize()
+    recs = dd.read_records(rec_buf)
+    assert [r.status for r in recs] == [dd.STATUS_WAIT_LIMIT] * P
+    assert all(r.idx == [0, 1, 2] for r in recs)
+    # the next call on the same context and records is a normal merge again
+    for f, (theta, v, _) in zip(frags, hosts):
+        f["global_"].copy_(torch.from_numpy(theta))
+        f["momentum"].copy_(torch.from_numpy(v))
+    ctx.merge_fragments_batched(frags, M, dd.BF16, ETA, MU, flags=dd.DIAG_STATE, records=rec_buf)
+    torch.cuda.synchronize()
+    for p, (rec, f, (theta, v, learners)) in enumerate(zip(dd.read_records(rec_buf), frags, hosts)):
+        ref = oracle.merge_fragment(theta, v, learners, [1 + p, 2, 3], 0b111, 1, ETA, MU)
+        assert_record_matches(rec, ref, per_learner=False)
+        assert floor_rel_err(f["global_"].cpu().numpy(), theta) <= TOL_STATE
+        assert floor_rel_err(f["momentum"].cpu().numpy(), v) <= TOL_STATE
+
+
 def test_hand_worked_example_on_gpu(dd, ctx):
     # the two-learner merge worked on paper in tests/golden/merge_hand_worked.txt; every
     # intermediate is exact in binary32, so the GPU must reproduce it bit for bit

@@ -546,6 +546,24 @@ def test_int4_quantiser_properties():
     assert s_[0] == 1.0 and (c[0] & 15) == 15 and (c[0] >> 4) == 10 and (c[1] & 15) == 12
 
 
+def test_int4_quantiser_non_finite_differences_poison_their_block():
+    # three blocks: a NaN, an infinity, and an ordinary one that must be untouched by its neighbours
+    t = np.zeros(384, dtype=np.float32)
+    l = np.full(384, -1.0, dtype=np.float32)
+    l[3] = np.nan
+    l[128 + 7] = -np.inf                                # d = +inf
+    l[128 + 8] = np.inf                                 # d = -inf
+    c, s_ = oracle.quantize_int4(t, l)
+    assert np.isnan(s_[0]) and np.isposinf(s_[1]) and s_[2] == np.float32(1.0) / np.float32(7.0)
+    nib = np.stack([c & 15, c >> 4], axis=1).reshape(-1)
+    assert np.all(nib[:128] == 8)                       # NaN scale: every code 0
+    assert nib[128 + 7] == 1 and nib[128 + 8] == 1      # inf / inf is NaN, coded -7
+    assert np.all(np.delete(nib[128:256], [7, 8]) == 8) # finite / inf = 0
+    assert np.all(nib[256:] == 15)                      # the ordinary block: d = 1 = 7 * scale
+    dq = oracle.dequantize_int4(c, s_, 384)
+    assert not np.isfinite(dq[:256]).any() and np.all(dq[256:] == np.float32(7.0) * s_[2])
+
+
 def test_int4_merge_equals_plain_merge_of_dequantised_gradients():
     n, M = 3000, 4
     theta, v, learners = _frag(n=n, M=M, dtype="bf16", seed=72)
