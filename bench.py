@@ -5,17 +5,26 @@ One "step" is one pass of the whole hot path -- participation, weights, outer
 gradients, weighted reduce, outer optimizer step, norm diagnostics -- over one
 synthetic workload (default: one 500M-parameter fragment, 32 bf16 learner
 copies of which 24 are in quorum, fp32 global + momentum).  Prints ONE JSON
-line on rank 0.
+line on rank 0.  At N = 1 the line also carries, under "configs", one row for
+every other workload and merge kind (tiny, dense150m, dense1b3, moe4b, the
+radial-directional and int4 merges of the headline workload, the syncer loop),
+and, under roofline.same_run_ceilings, what this GPU gives probe kernels that
+move data like the merge does but compute nothing.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME]
-    python bench.py --impl reference      # the CPU oracle on a bounded sample
+    python bench.py --gpus 8               # starts 8 ranks itself, one per GPU
+    python bench.py --gpus 8 --dry-launch  # prints the ranks' environments, runs nothing
+    python bench.py --impl reference       # the CPU oracle on a bounded sample
 """
 from __future__ import annotations
 
 import argparse
+import ctypes
 import json
 import os
+import socket
 import statistics
+import subprocess
 import sys
 import threading
 import time
@@ -27,13 +36,11 @@ if ROOT not in sys.path:
 METRIC = "merged_params_per_sec"
 UNIT = "params/s"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per merged parameter and merge, from the ncu
-# captures summarised under profiles/ (absent: not captured for that merge kind and workload).
-# The radial-directional figure is the sum of its three passes.
-NCU_TRAFFIC_BYTES_PER_PARAM = {
-    ("avg", "scale500m"): 63.04, ("avg", "dense150m"): 27.73, ("avg", "dense1b3"): 41.61,
-    ("avg", "moe4b"): 41.50, ("rda", "scale500m"): 124.8, ("int4", "scale500m"): 26.24,
-}
+NOMINAL_HBM_GBS = 8000.0
+L2_BYTES = 126e6
+PROBE_SRC = os.path.join(ROOT, "bench_probes.cu")
+PROBE_LIB = os.path.join(ROOT, "bench_probes.so")
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_traffic_bytes_per_param.txt")
 
 
 def host_cpu_model() -> str:
@@ -47,7 +54,7 @@ def host_cpu_model() -> str:
     return "unknown"
 
 
-def parse_args():
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
@@ -55,11 +62,16 @@ def parse_args():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="scale500m")
     ap.add_argument("--scale", type=float, default=1.0, help="shrink every fragment (profiling)")
-    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-ceilings", action="store_true",
-                    help="skip the same-run copy / read bandwidth ceilings (torch kernels)")
+                    help="skip the same-run bandwidth ceilings (probe kernels)")
+    ap.add_argument("--configs", default="all",
+                    help="N = 1: which other workloads get a row in the line's 'configs' array: "
+                         "'all', 'none', or a comma-separated list of "
+                         "tiny,dense150m,dense1b3,moe4b,rda,int4,tape24")
+    ap.add_argument("--config-steps", type=int, default=20, help="timed launches per 'configs' row")
     ap.add_argument("--cpu-sample", type=int, default=1 << 27,
                     help="elements of the workload the CPU oracle is timed on")
     ap.add_argument("--out-bf16", action="store_true", help="also write the bf16 broadcast copy")
@@ -73,7 +85,65 @@ def parse_args():
     ap.add_argument("--sharding", choices=["replica", "range"], default="replica",
                     help="N>1: every rank merges its own copy of the workload (weak scaling), or "
                          "each rank owns a contiguous element range of every fragment (strong)")
-    return ap.parse_args()
+    ap.add_argument("--dry-launch", action="store_true",
+                    help="print the environment and command of every rank --gpus N would start, then exit")
+    return ap.parse_args(argv)
+
+
+# ---- workload accounting (reporting only) ----------------------------------------------
+
+def participants(w, p: int) -> int:
+    """Learners of fragment p whose mask bit is set and whose token count is positive."""
+    return sum(1 for m in range(w.M) if (w.masks[p] >> m) & 1 and int(w.tokens[p, m]) > 0)
+
+
+def bytes_per_param(merge: str, s: int, b_theta: int, out_bf16: bool = False) -> float:
+    """Algorithmic bytes per merged parameter: every participant's payload once, the global
+    fragment and the momentum read once and written once.
+      avg   s b + 16 (+ 2 with the bf16 copy)
+      int4  s (1/2 + 4/128) + 16
+      rda   the copies and Theta twice, Theta and v read and written, and the Gram products or the
+            stored direction: see rda_bytes_per_param."""
+    if merge == "int4":
+        return s * (0.5 + 4.0 / 128.0) + 16 + (2 if out_bf16 else 0)
+    if merge == "rda":
+        return rda_bytes_per_param(s, b_theta) + (2 if out_bf16 else 0)
+    return s * b_theta + 16 + (2 if out_bf16 else 0)
+
+
+def rda_bytes_per_param(s: int, b_theta: int) -> float:
+    """Three passes: norms (copies + Theta), direction (copies + Theta, write u), apply (Theta, v,
+    u read; Theta, v written) = 2 (s b + 4) + 24."""
+    return 2 * (s * b_theta + 4) + 24
+
+
+def algorithmic_bytes(w, merge: str = "avg", out_bf16: bool = False) -> int:
+    b_theta = 2 if w.learner_dtype == "bf16" else 4
+    return int(sum(n * bytes_per_param(merge, participants(w, p), b_theta, out_bf16)
+                   for p, n in enumerate(w.fragment_sizes)))
+
+
+def write_share(w, merge: str = "avg", out_bf16: bool = False) -> float:
+    """Fraction of the algorithmic bytes that are writes."""
+    total = algorithmic_bytes(w, merge, out_bf16)
+    writes = sum(n * (8 + (2 if out_bf16 else 0) + (4 if merge == "rda" else 0)) for n in w.fragment_sizes)
+    return writes / total if total else 0.0
+
+
+def ncu_traffic_table():
+    """(merge kind, workload) -> DRAM bytes per merged parameter measured by ncu
+    (dram__bytes_read.sum + dram__bytes_write.sum); the file is written with the summaries
+    under profiles/."""
+    table = {}
+    try:
+        with open(TRAFFIC_FILE) as fh:
+            for ln in fh:
+                ln = ln.split("#", 1)[0].split()
+                if len(ln) >= 3:
+                    table[(ln[0], ln[1])] = float(ln[2])
+    except OSError:
+        pass
+    return table
 
 
 # ---- clocks ------------------------------------------------------------------------
@@ -142,7 +212,7 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(self.samples)}
 
 
-# ---- measured peaks -----------------------------------------------------------------
+# ---- measured peaks and same-run ceilings ---------------------------------------------
 
 def hbm_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -153,31 +223,79 @@ def hbm_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def measure_ceilings(device, reps=10):
-    """What this machine gives plain streaming kernels in the same run (torch library
-    kernels, not the product): a device-to-device copy and a read-only reduction."""
-    import torch
+def build_probes(force: bool = False) -> str:
+    """Compiles bench_probes.cu (sm_100a) into bench_probes.so when missing or stale."""
+    if not force and os.path.exists(PROBE_LIB) and os.path.getmtime(PROBE_LIB) >= os.path.getmtime(PROBE_SRC):
+        return PROBE_LIB
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    tmp = PROBE_LIB + f".tmp{os.getpid()}"
+    cmd = [nvcc, "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
+           "--shared", "-Xcompiler", "-fPIC", "-cudart", "static", "-o", tmp, PROBE_SRC]
+    proc = subprocess.run(cmd, capture_output=True, text=True)
+    if proc.returncode != 0:
+        sys.stderr.write(proc.stdout + proc.stderr)
+        raise RuntimeError("nvcc failed building bench_probes.so")
+    os.replace(tmp, PROBE_LIB)
+    return PROBE_LIB
 
-    n = 1 << 29                                        # 2 GiB of float32 per array
-    a = torch.ones(n, dtype=torch.float32, device=device)
-    b = torch.empty_like(a)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    out = {}
-    for name, fn, nbytes in (("copy_ceiling_gbs", lambda: b.copy_(a), 8 * n),
-                             ("read_ceiling_gbs", lambda: a.sum(), 4 * n)):
-        for _ in range(3):
-            fn()
-        best = None
-        for _ in range(reps):
-            ev0.record()
-            fn()
-            ev1.record()
-            ev1.synchronize()
-            ms = ev0.elapsed_time(ev1)
-            best = ms if best is None or ms < best else best
-        out[name] = nbytes / (best * 1e-3) / 1e9
-    del a, b
-    return out
+
+class Probes:
+    """The probe kernels of bench_probes.cu on one scratch buffer."""
+
+    def __init__(self, device, scratch_bytes: int = 9 << 30):
+        import torch
+        self.lib = ctypes.CDLL(build_probes())
+        self.lib.ddp_stream_probe.restype = ctypes.c_double
+        self.lib.ddp_stream_probe.argtypes = [
+            ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+            ctypes.c_size_t, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
+            ctypes.POINTER(ctypes.c_double)]
+        free = torch.cuda.mem_get_info(device)[0]
+        self.bytes = int(min(scratch_bytes, max(1 << 30, free // 2)))
+        self.buf = torch.empty(self.bytes, dtype=torch.uint8, device=device)
+        self.buf.fill_(0x3c)
+        self.stream = int(torch.cuda.current_stream().cuda_stream)
+
+    def run(self, rd2=0, rd4=0, wr4=0, wr2=0, push_in_place=False, ctas_per_sm=2, reps=10):
+        """GB/s of the shape (best of ``reps``), streams sized to fill the scratch buffer."""
+        row_bytes = 2048 * (rd2 + (0 if push_in_place else wr2)) + 4096 * max(rd4, wr4)
+        if push_in_place:
+            row_bytes += 2048 * max(0, wr2 - rd2)
+        rows = (self.bytes - (1 << 20)) // row_bytes
+        ms = ctypes.c_double(0.0)
+        gbs = self.lib.ddp_stream_probe(self.buf.data_ptr(), self.bytes, rd2, rd4, wr4, wr2,
+                                        rows * 1024, int(push_in_place), ctas_per_sm, reps, self.stream,
+                                        ctypes.byref(ms))
+        if gbs < 0:
+            raise RuntimeError(f"bandwidth probe failed (code {gbs})")
+        return gbs
+
+    def close(self):
+        import torch
+        del self.buf
+        torch.cuda.empty_cache()
+
+
+def measure_ceilings(device):
+    """What this GPU gives, in this run, to kernels that move data the way the merge does but
+    compute nothing (bench_probes.cu): a read-only stream set, a write-only one, and the
+    headline mix; each over the whole scratch buffer (about 9 GB), best of 10."""
+    pr = Probes(device)
+    out = {
+        "read_gbs": pr.run(rd2=24),
+        "write_gbs": pr.run(wr4=2),
+        "mix_gbs": pr.run(rd2=24, rd4=2, wr4=2),
+        "how": "bench_probes.cu: 2 KB cp.async.bulk warp rings over 24 two-byte streams (read); "
+               "st.global.cs.v8 into two four-byte streams (write); the merge's own pattern at "
+               "24 participants, 87.5 % reads (mix); about 9 GB each, best of 10, CUDA events",
+    }
+    return out, pr
+
+
+def blend_ceiling(read_gbs: float, write_gbs: float, wshare: float) -> float:
+    """Bandwidth of a stream with the given share of writes if reads and writes each ran at
+    their own ceiling and did not disturb one another (an upper bound, not a measurement)."""
+    return 1.0 / ((1.0 - wshare) / read_gbs + wshare / write_gbs)
 
 
 # ---- the reference arm: the CPU oracle ------------------------------------------------
@@ -188,8 +306,6 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    import numpy as np
-
     import oracle
     from paper_2604_21428_b200 import synth
 
@@ -226,6 +342,54 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ---- starting the ranks -----------------------------------------------------------------
+
+def _free_port() -> int:
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as s:
+        s.bind(("127.0.0.1", 0))
+        return int(s.getsockname()[1])
+
+
+def launch_plan(n_ranks: int, argv, port: int | None = None):
+    """Environment and command of every rank of a one-node job: one process per GPU."""
+    port = port or _free_port()
+    plan = []
+    for r in range(n_ranks):
+        env = {"RANK": str(r), "LOCAL_RANK": str(r), "WORLD_SIZE": str(n_ranks),
+               "LOCAL_WORLD_SIZE": str(n_ranks), "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(port)}
+        plan.append({"rank": r, "env": env, "argv": [sys.executable, os.path.abspath(__file__)] + list(argv)})
+    return plan
+
+
+def spawn_ranks(args, argv) -> int:
+    """``python bench.py --gpus N`` outside a launcher: starts the N ranks itself (what
+    ``python -m torch.distributed.run --nproc-per-node N`` would do) and waits for them.  Rank 0
+    prints the JSON line; the exit code is the first non-zero one."""
+    plan = launch_plan(args.gpus, argv)
+    procs = []
+    for item in plan:
+        procs.append(subprocess.Popen(item["argv"], env=dict(os.environ, **item["env"])))
+    rc = 0
+    try:
+        pending = list(procs)
+        while pending:
+            for pr in list(pending):
+                code = pr.poll()
+                if code is None:
+                    continue
+                pending.remove(pr)
+                if code != 0 and rc == 0:
+                    rc = code
+                    for other in pending:           # a rank failed: the others would wait for it forever
+                        other.terminate()
+            time.sleep(0.05)
+    finally:
+        for pr in procs:
+            if pr.poll() is None:
+                pr.kill()
+    return rc
+
+
 # ---- our arm ---------------------------------------------------------------------------
 
 def build_workload(w, device, rank_seed, out_bf16, resident="all"):
@@ -250,7 +414,320 @@ def build_workload(w, device, rank_seed, out_bf16, resident="all"):
     return frags
 
 
-def run_replay(args):
+def resident_bytes(w, resident: str) -> int:
+    b_theta = 2 if w.learner_dtype == "bf16" else 4
+    copies = [w.M if resident == "all" else participants(w, p) for p in range(w.P)]
+    return int(sum(n * (8 + c * b_theta) for n, c in zip(w.fragment_sizes, copies)))
+
+
+class Merger:
+    """One workload resident on the GPU and the library call that merges it."""
+
+    def __init__(self, dd, ctx, w, device, *, merge="avg", out_bf16=False, resident="all", rank_seed=0,
+                 frags=None, range_sharded_rda=False):
+        import torch
+        from paper_2604_21428_b200 import synth
+        self.dd, self.ctx, self.w, self.merge, self.device = dd, ctx, w, merge, device
+        self.frags = frags if frags is not None else build_workload(w, device, rank_seed, out_bf16, resident)
+        self.ldtype = dd.BF16 if w.learner_dtype == "bf16" else dd.F32
+        self.records = dd.new_records(w.P, device=device)
+        self.flags = dd.DIAG_STATE
+        self.eta, self.mu = synth.OUTER_LR, synth.OUTER_MU
+        self.launches_per_step = 1
+        self.int4_codes = self.int4_scales = None
+        self.rda_scratch = None
+        if merge == "int4":
+            # the learners' side, outside every timed region: compress each participant's outer gradient
+            assert w.P == 1, "the int4 merge takes a single-fragment workload"
+            self.quantise()
+        if merge == "rda":
+            self.launches_per_step = 3
+            if range_sharded_rda:
+                self.rda_scratch = torch.empty(sum((n + 7) // 8 * 8 for n in w.fragment_sizes),
+                                               dtype=torch.float32, device=device)
+        # the same buffers are merged every step: marshal their addresses and counts once
+        self.packed_ptrs = dd.pack_pointers(self.frags[0]["learners"]) if w.P == 1 else None
+        self.packed_tokens = dd.pack_u64(self.frags[0]["tokens"]) if w.P == 1 else None
+
+    def quantise(self):
+        import torch
+        f, w = self.frags[0], self.w
+        n0 = f["n"]
+        self.int4_codes, self.int4_scales = [None] * w.M, [None] * w.M
+        for m in range(w.M):
+            if (f["quorum_mask"] >> m) & 1 and f["tokens"][m] > 0:
+                self.int4_codes[m] = torch.empty((n0 + 1) // 2, dtype=torch.uint8, device=self.device)
+                self.int4_scales[m] = torch.empty((n0 + 127) // 128, dtype=torch.float32, device=self.device)
+                self.ctx.quantize_outer_gradient_int4(f["global_"], f["learners"][m], self.int4_codes[m],
+                                                      self.int4_scales[m], n=n0, learner_dtype=self.ldtype)
+        torch.cuda.synchronize()
+
+    def step(self, stream=None):
+        import torch
+        from paper_2604_21428_b200 import dist as ddist
+        ctx, w, f0 = self.ctx, self.w, self.frags[0]
+        stream = stream if stream is not None else torch.cuda.current_stream()
+        if self.merge == "int4":
+            ctx.merge_fragment_int4(f0["global_"], f0["momentum"], self.int4_codes, self.int4_scales,
+                                    f0["tokens"], f0["quorum_mask"], f0["K"], self.eta, self.mu, n=f0["n"],
+                                    flags=self.flags, out_bf16=f0["out_bf16"], record=self.records,
+                                    stream=stream)
+        elif self.merge == "rda" and self.rda_scratch is not None:
+            # range-sharded: the passes one by one, norms all-reduced over the ranks in between
+            ddist.rda_merge_range_sharded(ctx, self.frags, w.M, self.ldtype, self.eta, self.mu,
+                                          records=self.records, scratch=self.rda_scratch,
+                                          flags=self.flags, stream=stream)
+        elif self.merge == "rda":
+            ctx.merge_fragments_batched_rda(self.frags, w.M, self.ldtype, self.eta, self.mu,
+                                            flags=self.flags, records=self.records, stream=stream)
+        elif w.P == 1:
+            ctx.merge_fragment(f0["global_"], f0["momentum"], self.packed_ptrs, self.packed_tokens,
+                               f0["quorum_mask"], f0["K"], self.eta, self.mu, n=f0["n"],
+                               learner_dtype=self.ldtype, flags=self.flags, out_bf16=f0["out_bf16"],
+                               record=self.records, stream=stream)
+        else:
+            ctx.merge_fragments_batched(self.frags, w.M, self.ldtype, self.eta, self.mu, flags=self.flags,
+                                        records=self.records, stream=stream)
+
+    # ---- parity evidence on the buffers that are about to be timed --------------------
+    def first_merge_parity(self, max_fragments: int = 4):
+        """Runs the FIRST merge (fresh state) and compares sampled 65,536-element windows of it
+        with the oracle: inputs are copied out before the merge; nothing flows from the GPU into
+        the oracle.  The int4 merge is checked end to end (the oracle quantises the window itself;
+        windows start on block boundaries).  A radial-directional merge depends on whole-fragment
+        norms, so a window cannot be given to the oracle: no windows, said so."""
+        import numpy as np
+        import torch
+
+        import oracle
+        w = self.w
+        if self.merge == "rda":
+            self.step()
+            torch.cuda.synchronize()
+            return {"windows": 0, "note": "radial-directional merge: whole-fragment norms, no window "
+                                           "parity here; element-by-element parity is in tests/test_gpu_rda.py"}
+
+        def host_learner(t):
+            t = t.cpu()
+            return t.view(torch.int16).numpy().view(np.uint16).copy() if t.dtype == torch.bfloat16 \
+                else t.numpy().copy()
+
+        picks = sorted(set([0, w.P - 1] + list(range(0, w.P, max(1, w.P // max_fragments)))))[:max_fragments + 1]
+        saved = {}
+        for p in picks:
+            f = self.frags[p]
+            n = f["n"]
+            win = min(1 << 16, n)
+            starts = sorted({0, max(0, (n - win) // 128 * 128), (n // 3) // 128 * 128, (2 * n // 3) // 128 * 128})
+            starts = [s0 for s0 in starts if s0 + win <= n]
+            part = [m for m in range(w.M) if (f["quorum_mask"] >> m) & 1 and f["tokens"][m] > 0]
+            saved[p] = (win, starts, [(f["global_"][s0:s0 + win].cpu().numpy().copy(),
+                                       f["momentum"][s0:s0 + win].cpu().numpy().copy(),
+                                       [host_learner(f["learners"][m][s0:s0 + win]) if m in part else None
+                                        for m in range(w.M)]) for s0 in starts])
+        self.step()
+        torch.cuda.synchronize()
+        recs = self.dd.read_records(self.records)
+        worst = {"t": 0.0, "v": 0.0}
+        exact, nwin = True, 0
+        for p in picks:
+            f, rec = self.frags[p], recs[p]
+            win, starts, per = saved[p]
+            for s0, (t0, v0, ls) in zip(starts, per):
+                if self.merge == "int4":
+                    q = [None if a is None else oracle.quantize_int4(t0, a) for a in ls]
+                    ref = oracle.merge_fragment_int4(t0, v0, [None if x is None else x[0] for x in q],
+                                                     [None if x is None else x[1] for x in q], f["tokens"],
+                                                     f["quorum_mask"], f["K"], self.eta, self.mu)
+                else:
+                    ref = oracle.merge_fragment(t0, v0, ls, f["tokens"], f["quorum_mask"], f["K"],
+                                                self.eta, self.mu)
+                exact &= (rec.status, rec.n_part, rec.idx) == (ref.status, ref.n_part, ref.idx)
+                exact &= rec.w_hat == [float(np.float32(x)) for x in ref.w_hat]
+                for got, want, which in ((f["global_"], t0, "t"), (f["momentum"], v0, "v")):
+                    g = got[s0:s0 + win].cpu().numpy().astype(np.float64)
+                    o = want.astype(np.float64)
+                    rms = float(np.sqrt(np.mean(o * o))) or 1.0
+                    worst[which] = max(worst[which], float(np.max(np.abs(g - o) / np.maximum(np.abs(o), rms))))
+                nwin += 1
+        return {"windows": nwin, "window_elems": saved[picks[0]][0], "fragments_sampled": len(picks),
+                "max_err_theta": worst["t"], "max_err_momentum": worst["v"], "tolerance": 1e-5,
+                "participation_and_weights_bit_exact": bool(exact),
+                "metric": "first merge: max |gpu - oracle| / max(|oracle|, rms(oracle))"}
+
+    def timed(self, steps: int, warmup: int, world: int = 1):
+        """``warmup`` untimed steps, then ``steps`` timed ones bracketed by a barrier and a
+        synchronize on both sides; one CUDA event after every step gives the per-launch times."""
+        import torch
+        import torch.distributed as dist
+        stream = torch.cuda.current_stream()
+        for _ in range(max(warmup, 3)):
+            self.step()
+        torch.cuda.synchronize()
+        recs = self.dd.read_records(self.records)
+        assert all(r.status == 0 for r in recs), [r.status for r in recs]
+        sampler = ClockSampler(self.device.index or 0)
+        events = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        sampler.start()
+        events[0].record(stream)
+        for k in range(steps):
+            self.step()
+            events[k + 1].record(stream)
+        torch.cuda.synchronize()
+        sampler.stop()
+        if world > 1:
+            dist.barrier()
+        total_ms = events[0].elapsed_time(events[-1])
+        per_launch_ms = [events[k].elapsed_time(events[k + 1]) for k in range(steps)]
+        return total_ms, per_launch_ms, sampler.summary()
+
+    def timed_cold(self, steps: int):
+        """A workload that fits in L2 is also timed cold: a 512 MB buffer is rewritten between
+        launches and only the merge is bracketed by events."""
+        import torch
+        stream = torch.cuda.current_stream()
+        flush = torch.empty(512 << 20, dtype=torch.uint8, device=self.device)
+        cold = []
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for k in range(steps):
+            flush.fill_(k & 0xff)
+            e0.record(stream)
+            self.step()
+            e1.record(stream)
+            e1.synchronize()
+            cold.append(e0.elapsed_time(e1))
+        del flush
+        return {"median": statistics.median(cold), "min": min(cold), "max": max(cold)}
+
+    def timed_graph(self, reps: int = 50):
+        """A single small fragment is launch-bound from Python (the host needs longer to issue a
+        merge than the GPU to run it): the same calls captured once into a CUDA graph and
+        replayed give the device-bound time per merge.  The single-fragment call is capture-safe
+        (one kernel launch, no allocation or synchronisation once the workspace exists)."""
+        import torch
+        side = torch.cuda.Stream(device=self.device)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                for _ in range(reps):
+                    self.step(side)
+        torch.cuda.synchronize()
+        times = []
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(8):
+            e0.record()
+            graph.replay()
+            e1.record()
+            e1.synchronize()
+            times.append(e0.elapsed_time(e1) / reps)
+        del graph
+        return {"median": statistics.median(times[3:]), "min": min(times[3:]), "merges_per_graph": reps}
+
+    def free(self):
+        import torch
+        self.frags = self.int4_codes = self.int4_scales = self.rda_scratch = self.records = None
+        self.packed_ptrs = None
+        torch.cuda.empty_cache()
+
+
+def roofline_of(w, merge, out_bf16, per_launch_ms, ceilings, traffic_table, workload_name):
+    """The roofline object of one timed workload (HBM-bound; no tensor cores on this path)."""
+    alg = algorithmic_bytes(w, merge, out_bf16)
+    avg = sum(per_launch_ms) / len(per_launch_ms)
+    achieved = alg / (avg * 1e-3) / 1e9
+    peak, peak_kind = hbm_peak()
+    tpp = None if out_bf16 else traffic_table.get((merge, workload_name))
+    r = {
+        "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+        "peak_source": f"of {peak_kind}",
+        "traffic": None if tpp is None else tpp * w.total_params,
+        "algorithmic_bytes_per_launch": alg, "bytes_per_param": alg / w.total_params,
+        "write_share": write_share(w, merge, out_bf16),
+        "kernel_ms": {"avg": avg, "median": statistics.median(per_launch_ms), "min": min(per_launch_ms),
+                      "max": max(per_launch_ms)},
+        "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+    }
+    if ceilings:
+        blend = blend_ceiling(ceilings["read_gbs"], ceilings["write_gbs"], r["write_share"])
+        r["frac_of_read_ceiling"] = achieved / ceilings["read_gbs"]
+        r["blend_ceiling_gbs"] = blend
+        r["frac_of_blend_ceiling"] = achieved / blend
+    return r
+
+
+def config_row(dd, ctx, device, name, merge, args, ceilings, probes, traffic_table, merger=None,
+               resident="all"):
+    """One row of the line's 'configs' array: a workload merged ``--config-steps`` times."""
+    import torch
+
+    from paper_2604_21428_b200 import synth
+    w = merger.w if merger is not None else synth.workload(name)
+    own = merger is None
+    note = None
+    if own:
+        free = torch.cuda.mem_get_info(device)[0]
+        if resident_bytes(w, resident) + (3 << 30) > free:
+            resident = "participants"
+        if resident_bytes(w, resident) + (3 << 30) > free:
+            return {"workload": name, "merge": merge, "skipped":
+                    f"needs {resident_bytes(w, resident) >> 30} GiB resident, {free >> 30} GiB free"}
+        if resident == "participants":
+            note = "only the participating learner copies are resident (the others are never read)"
+        merger = Merger(dd, ctx, w, device, merge=merge, resident=resident)
+    else:
+        # another merge kind on buffers that are already resident: back to the seeded state first, so
+        # that the parity windows below are again those of a FIRST merge
+        merger.merge = merge
+        merger.launches_per_step = 3 if merge == "rda" else 1
+        for p, f in enumerate(merger.frags):
+            synth.fill_fragment_gpu(f["global_"], f["momentum"], f["learners"], seed=w.seed * 1000 + p)
+        if merge == "int4":
+            merger.quantise()
+    row = {"workload": name, "merge": merge, "fragments": w.P, "params": w.total_params, "M": w.M,
+           "participants": [participants(w, p) for p in range(w.P)], "learner_dtype": w.learner_dtype}
+    if note:
+        row["note"] = note
+    try:
+        if not args.no_cpu_baseline:
+            row["parity"] = merger.first_merge_parity()
+        _, per_launch, clocks = merger.timed(args.config_steps, 3)
+        r = roofline_of(w, merge, False, per_launch, ceilings, traffic_table, name)
+        row.update({
+            "ms": r["kernel_ms"], "params_per_s": w.total_params / (r["kernel_ms"]["avg"] * 1e-3),
+            "bytes_per_param": r["bytes_per_param"], "write_share": r["write_share"],
+            "achieved_gbs": r["achieved"], "frac": r["frac"], "frac_of_nominal_8TBs": r["frac_of_nominal_8TBs"],
+            "launches_per_merge": merger.launches_per_step, "steps": args.config_steps,
+            "sm_mhz": clocks["sm_mhz"], "clock_reasons": clocks["reasons"],
+            "traffic_bytes_per_param_ncu": traffic_table.get((merge, name)),
+        })
+        for k in ("frac_of_read_ceiling", "blend_ceiling_gbs", "frac_of_blend_ceiling"):
+            if k in r:
+                row[k] = r[k]
+        alg = r["algorithmic_bytes_per_launch"]
+        if alg < 4 * L2_BYTES:
+            row["l2"] = "fits L2: 'ms' is warm (back to back); cold = 512 MB flush between launches"
+            row["ms_l2_flushed"] = merger.timed_cold(min(args.config_steps, 20))
+            row["achieved_gbs_l2_flushed"] = alg / (row["ms_l2_flushed"]["median"] * 1e-3) / 1e9
+            if w.P == 1 and merge == "avg":
+                row["ms_cuda_graph_replay"] = merger.timed_graph()
+        else:
+            row["l2"] = "inputs larger than L2 (no flush)"
+        if probes is not None and merge == "avg":
+            # the same access pattern with the arithmetic left out, at this workload's mean participant count
+            s_mean = max(1, round(sum(row["participants"]) / w.P))
+            if w.learner_dtype == "bf16":
+                row["pattern_probe_gbs"] = probes.run(rd2=s_mean, rd4=2, wr4=2, reps=5)
+                row["frac_of_pattern_probe"] = row["achieved_gbs"] / row["pattern_probe_gbs"]
+    finally:
+        if own:
+            merger.free()
+    return row
+
+
+def run_replay(args, ceilings=None):
     """Second workload: the syncer loop itself.  A 1.34B-parameter dense decoder (24 layers,
     d 2048, d_ff 8192) is cut into P = H = 24 balanced fragments by the library's planner;
     8 bf16 learners, K = 1, grace window of a quarter step; every syncer step merges the
@@ -295,7 +772,7 @@ def run_replay(args):
     torch.cuda.synchronize()
     sampler = ClockSampler(0)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    merged_params = merged_bytes = launches = 0
+    merged_params = merged_bytes = written_bytes = launches = 0
     sampler.start()
     ev0.record(stream)
     for t in range(args.warmup, total_steps):
@@ -308,6 +785,7 @@ def run_replay(args):
                 # merge (read s copies, Theta, v; write Theta', v') + push (write the alive copies);
                 # the unfused form reads Theta' once more in its broadcast launch
                 merged_bytes += sizes[p] * (2 * s_p + 16) + sizes[p] * (2 * alive)
+                written_bytes += sizes[p] * (8 + 2 * alive)
                 if not syncer.fused_push:
                     merged_bytes += sizes[p] * 4
                     launches += 1
@@ -318,6 +796,16 @@ def run_replay(args):
     ms = ev0.elapsed_time(ev1)
     peak, peak_kind = hbm_peak()
     achieved = merged_bytes / (ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_source": f"of {peak_kind}", "traffic": None,
+                "algorithmic_bytes": merged_bytes, "write_share": written_bytes / max(merged_bytes, 1),
+                "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "note": ("merge and push fused in one launch per syncer step" if syncer.fused_push else
+                         "merge + broadcast launches of the syncer loop") + ", host work included"}
+    if ceilings:
+        blend = blend_ceiling(ceilings["read_gbs"], ceilings["write_gbs"], roofline["write_share"])
+        roofline["blend_ceiling_gbs"] = blend
+        roofline["frac_of_blend_ceiling"] = achieved / blend
     line = {
         "metric": METRIC, "value": merged_params / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
@@ -329,27 +817,127 @@ def run_replay(args):
                    "planner": "balanced", "learner_dtype": "bf16",
                    "l2": "inputs larger than L2 (no flush)"},
         "clocks": sampler.summary(), "gpu_launches": launches,
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_source": f"of {peak_kind}", "traffic": None,
-                     "algorithmic_bytes": merged_bytes,
-                     "note": ("merge and push fused in one launch per syncer step" if syncer.fused_push else
-                              "merge + broadcast launches of the syncer loop") + ", host work included"},
+        "roofline": roofline,
         "e2e": None, "cpu_baseline": None,
     }
-    print(json.dumps(line), flush=True)
     ctx.close()
+    del syncer, theta, mom, learners
+    torch.cuda.empty_cache()
+    return line
 
 
-def main():
-    args = parse_args()
-    if args.impl == "reference":
-        run_reference(args)
-        return
-    if args.workload == "tape24":
-        run_replay(args)
-        return
+def e2e_leg(dd, ctx, merger, args, world):
+    """End to end through the public host-buffer call: pinned host buffers in, results in host
+    memory, host<->device copies inside the timed region."""
+    import torch
+    import torch.distributed as dist
 
+    from paper_2604_21428_b200 import dist as ddist
+    w, f = merger.w, merger.frags[0]
+    n = f["n"]
+    part = [m for m in range(w.M) if (f["quorum_mask"] >> m) & 1 and f["tokens"][m] > 0]
+    # Page-locked host memory is bounded: every rank of the node pins its own buffers, so
+    # with several ranks (or little free host memory) the end-to-end leg streams a leading
+    # slice of the fragment instead of all of it.
+    esz = 2 if w.learner_dtype == "bf16" else 4
+    per_elem = len(part) * esz + 8
+    try:
+        avail = next(int(l.split()[1]) * 1024 for l in open("/proc/meminfo") if l.startswith("MemAvailable"))
+    except Exception:
+        avail = 64 << 30
+    local_world = int(os.environ.get("LOCAL_WORLD_SIZE", str(world)))
+    budget = int(0.4 * avail / max(local_world, 1))
+    n = max(8, min(n, budget // per_elem) // 8 * 8)
+    h_theta = torch.empty(n, dtype=torch.float32, pin_memory=True)
+    h_mom = torch.empty(n, dtype=torch.float32, pin_memory=True)
+    h_theta.copy_(f["global_"][:n])
+    h_mom.copy_(f["momentum"][:n])
+    h_learners = [None] * w.M
+    for m in part:
+        h_learners[m] = torch.empty(n, dtype=f["learners"][m].dtype, pin_memory=True)
+        h_learners[m].copy_(f["learners"][m][:n])
+    h2d = n * (len(part) * esz + 8)
+    d2h = n * 8 + dd.RECORD_BYTES
+    ctx.merge_fragment_host(h_theta, h_mom, h_learners, f["tokens"], f["quorum_mask"], f["K"],
+                            merger.eta, merger.mu, n=n, learner_dtype=merger.ldtype, flags=merger.flags)  # warm-up
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(args.e2e_steps):
+        rec = ctx.merge_fragment_host(h_theta, h_mom, h_learners, f["tokens"], f["quorum_mask"], f["K"],
+                                      merger.eta, merger.mu, n=n, learner_dtype=merger.ldtype,
+                                      flags=merger.flags)
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    assert rec.status == 0
+    dt_max = ddist.max_over_ranks(dt, device=merger.device)
+    # every rank streams its own copy (or its own range) of n elements per step
+    out = {"value": n * world * args.e2e_steps / dt_max, "unit": UNIT,
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+           "steps": args.e2e_steps, "elements_per_rank_step": n,
+           "h2d_gbs": h2d * args.e2e_steps / dt_max / 1e9,
+           "path": "dd_merge_fragment_host: pinned host buffers, chunked H2D -> kernel -> D2H "
+                   "pipeline, blocking"}
+    del h_learners, h_theta, h_mom
+    return out
+
+
+def cpu_baseline_leg(merger, args):
+    """The oracle as it stands on the host cores, on a bounded sample of the same workload."""
     import numpy as np
+    import torch
+
+    import oracle
+    w, f = merger.w, merger.frags[0]
+    ns = min(args.cpu_sample, f["n"])
+    part = [m for m in range(w.M) if (f["quorum_mask"] >> m) & 1 and f["tokens"][m] > 0]
+    theta = f["global_"][:ns].cpu().numpy()
+    mom = f["momentum"][:ns].cpu().numpy()
+    learners = [None] * w.M
+    for m in part:
+        t_m = f["learners"][m][:ns].cpu()
+        learners[m] = (t_m.view(torch.int16).numpy().view(np.uint16)
+                       if w.learner_dtype == "bf16" else t_m.numpy())
+    oracle.build()
+    t0 = time.perf_counter()
+    oracle.merge_fragment(theta, mom, learners, f["tokens"], f["quorum_mask"], f["K"], merger.eta, merger.mu)
+    dt = time.perf_counter() - t0
+    out = {"value": ns / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+           "sample": f"first {ns} elements of fragment 0 of {w.name}, {len(part)} participating "
+                     f"{w.learner_dtype} learners, one merge, {dt:.1f} s, single thread of "
+                     f"{os.cpu_count()} host cores",
+           "host_cpu": host_cpu_model(), "host_cores": os.cpu_count(),
+           "affinity_cores": len(os.sched_getaffinity(0))}
+    # Beside it, because the paper's own syncer is a CPU program: the same element loop
+    # spread over all host cores (OpenMP; not the checked oracle, a timing baseline only).
+    try:
+        cores = len(os.sched_getaffinity(0))
+        t0 = time.perf_counter()
+        oracle.merge_fragment_all_cores(theta, mom, learners, f["tokens"], f["quorum_mask"], f["K"],
+                                        merger.eta, merger.mu)
+        dt_all = time.perf_counter() - t0
+        out["all_cores"] = {"value": ns / dt_all, "unit": UNIT, "cores": cores,
+                            "kind": "oracle element loop under OpenMP", "seconds": dt_all}
+    except Exception as exc:      # no OpenMP runtime on the box: the oracle figure stands alone
+        out["all_cores"] = {"unavailable": str(exc)[:120]}
+    return out
+
+
+def wanted_configs(args, headline, headline_merge):
+    names = ["tiny", "dense150m", "dense1b3", "moe4b", "rda", "int4", "tape24"]
+    if args.configs == "none":
+        return []
+    if args.configs != "all":
+        asked = [x.strip() for x in args.configs.split(",") if x.strip()]
+        bad = [x for x in asked if x not in names]
+        if bad:
+            raise SystemExit(f"--configs: unknown {bad}; choose from {names}")
+        names = [x for x in names if x in asked]
+    return [x for x in names if not (x == headline and headline_merge == "avg")]
+
+
+def run_ours(args):
     import torch
     import torch.distributed as dist
 
@@ -366,6 +954,25 @@ def main():
     device = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
+        world = dist.get_world_size()            # the world that really initialised
+
+    traffic_table = ncu_traffic_table()
+    ceilings = probes = None
+    if not args.no_ceilings:
+        if rank == 0:
+            build_probes()
+        if world > 1:
+            dist.barrier()
+        ceilings, probes = measure_ceilings(device)
+
+    if args.workload == "tape24":
+        line = run_replay(args, ceilings)
+        if ceilings:
+            line["roofline"]["same_run_ceilings"] = ceilings
+        if probes is not None:
+            probes.close()
+        print(json.dumps(line), flush=True)
+        return
 
     w = synth.workload(args.workload)
     if args.scale != 1.0:
@@ -377,203 +984,33 @@ def main():
         align = 128 if args.merge == "int4" else 8
         w.fragment_sizes = [hi - lo for lo, hi in
                             (ddist.shard_range(n, rank, world, align) for n in w.fragment_sizes)]
-    frags = build_workload(w, device, rank, args.out_bf16, args.resident)
+    if probes is not None and resident_bytes(w, args.resident) + (4 << 30) > torch.cuda.mem_get_info(device)[0]:
+        probes.close()                           # the workload needs the room of the probes' scratch buffer
+        probes = None
     ctx = dd.Context(local_rank)
-    grid, block, tile = ctx.launch_geometry(dd.BF16 if w.learner_dtype == "bf16" else dd.F32)
-    ldtype = dd.BF16 if w.learner_dtype == "bf16" else dd.F32
-    records = dd.new_records(w.P, device=device)
-    flags = dd.DIAG_STATE
-    eta, mu = synth.OUTER_LR, synth.OUTER_MU
-    stream = torch.cuda.current_stream()
+    merger = Merger(dd, ctx, w, device, merge=args.merge, out_bf16=args.out_bf16, resident=args.resident,
+                    rank_seed=rank, range_sharded_rda=args.merge == "rda" and args.sharding == "range" and world > 1)
+    grid, block, tile = ctx.launch_geometry(merger.ldtype)
 
-    int4_codes = int4_scales = None
-    if args.merge == "int4":
-        # the learners' side, outside the timed region: compress every participant's outer gradient
-        assert w.P == 1, "--merge int4 takes a single-fragment workload"
-        f = frags[0]
-        n0 = f["n"]
-        int4_codes, int4_scales = [None] * w.M, [None] * w.M
-        for m in range(w.M):
-            if (f["quorum_mask"] >> m) & 1 and f["tokens"][m] > 0:
-                int4_codes[m] = torch.empty((n0 + 1) // 2, dtype=torch.uint8, device=device)
-                int4_scales[m] = torch.empty((n0 + 127) // 128, dtype=torch.float32, device=device)
-                ctx.quantize_outer_gradient_int4(f["global_"], f["learners"][m], int4_codes[m],
-                                                 int4_scales[m], n=n0, learner_dtype=ldtype)
-        torch.cuda.synchronize()
-
-    rda_scratch = None
-    if args.merge == "rda" and args.sharding == "range" and world > 1:
-        rda_scratch = torch.empty(sum((n + 7) // 8 * 8 for n in w.fragment_sizes), dtype=torch.float32,
-                                  device=device)
-    # the same buffers are merged every step: marshal their addresses and counts once
-    packed_ptrs = dd.pack_pointers(frags[0]["learners"]) if w.P == 1 else None
-    packed_tokens = dd.pack_u64(frags[0]["tokens"]) if w.P == 1 else None
-
-    def step(stream=stream):
-        if args.merge == "int4":
-            f = frags[0]
-            ctx.merge_fragment_int4(f["global_"], f["momentum"], int4_codes, int4_scales, f["tokens"],
-                                    f["quorum_mask"], f["K"], eta, mu, n=f["n"], flags=flags,
-                                    out_bf16=f["out_bf16"], record=records, stream=stream)
-        elif args.merge == "rda" and rda_scratch is not None:
-            # range-sharded: the passes one by one, norms all-reduced over the ranks in between
-            ddist.rda_merge_range_sharded(ctx, frags, w.M, ldtype, eta, mu, records=records,
-                                          scratch=rda_scratch, flags=flags, stream=stream)
-        elif args.merge == "rda":
-            ctx.merge_fragments_batched_rda(frags, w.M, ldtype, eta, mu, flags=flags,
-                                            records=records, stream=stream)
-        elif w.P == 1:
-            f = frags[0]
-            ctx.merge_fragment(f["global_"], f["momentum"], packed_ptrs, packed_tokens,
-                               f["quorum_mask"], f["K"], eta, mu, n=f["n"], learner_dtype=ldtype,
-                               flags=flags, out_bf16=f["out_bf16"], record=records, stream=stream)
-        else:
-            ctx.merge_fragments_batched(frags, w.M, ldtype, eta, mu, flags=flags, records=records,
-                                        stream=stream)
-
-    # ---- parity evidence on the buffers that are about to be timed: sampled windows of
-    # the very first merge (fresh state) against the oracle -----------------------------
     parity = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and args.merge == "avg":
-        import oracle
-        f = frags[0]
-        n = f["n"]
-        win = min(1 << 16, n)
-        starts = sorted({0, max(0, (n - win) // 8 * 8), (n // 3) // 8 * 8, (2 * n // 3) // 8 * 8})
-        starts = [s0 for s0 in starts if s0 + win <= n]
-        part = [m for m in range(w.M) if (f["quorum_mask"] >> m) & 1 and f["tokens"][m] > 0]
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        parity = merger.first_merge_parity()
 
-        def host_learner(t):
-            t = t.cpu()
-            return t.view(torch.int16).numpy().view(np.uint16).copy() if t.dtype == torch.bfloat16 \
-                else t.numpy().copy()
-
-        saved = [(f["global_"][s0:s0 + win].cpu().numpy().copy(),
-                  f["momentum"][s0:s0 + win].cpu().numpy().copy(),
-                  [host_learner(f["learners"][m][s0:s0 + win]) if m in part else None
-                   for m in range(w.M)]) for s0 in starts]
-        step()
-        torch.cuda.synchronize()
-        rec = dd.read_records(records)[0]
-        worst = {"t": 0.0, "v": 0.0}
-        exact = True
-        for s0, (t0, v0, ls) in zip(starts, saved):
-            ref = oracle.merge_fragment(t0, v0, ls, f["tokens"], f["quorum_mask"], f["K"], eta, mu)
-            exact &= (rec.status, rec.n_part, rec.idx) == (ref.status, ref.n_part, ref.idx)
-            exact &= rec.w_hat == [float(np.float32(x)) for x in ref.w_hat]
-            for got, want, which in ((f["global_"], t0, "t"), (f["momentum"], v0, "v")):
-                g = got[s0:s0 + win].cpu().numpy().astype(np.float64)
-                o = want.astype(np.float64)
-                rms = float(np.sqrt(np.mean(o * o))) or 1.0
-                worst[which] = max(worst[which], float(np.max(np.abs(g - o) / np.maximum(np.abs(o), rms))))
-        parity = {"windows": len(starts), "window_elems": win, "max_err_theta": worst["t"],
-                  "max_err_momentum": worst["v"], "tolerance": 1e-5,
-                  "participation_and_weights_bit_exact": bool(exact),
-                  "metric": "first merge: max |gpu - oracle| / max(|oracle|, rms(oracle))"}
-
-    for _ in range(max(args.warmup, 3)):
-        step()
-    torch.cuda.synchronize()
-    recs = dd.read_records(records)
-    assert all(r.status == 0 for r in recs), [r.status for r in recs]
-
-    sampler = ClockSampler(local_rank)
-    events = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
-    sampler.start()
-    events[0].record(stream)
-    for k in range(args.steps):
-        step()
-        events[k + 1].record(stream)
-    torch.cuda.synchronize()
-    sampler.stop()
-    if world > 1:
-        dist.barrier()
-    total_ms = events[0].elapsed_time(events[-1])
-    per_launch_ms = [events[k].elapsed_time(events[k + 1]) for k in range(args.steps)]
+    total_ms, per_launch_ms, clocks = merger.timed(args.steps, args.warmup, world)
     max_ms = ddist.max_over_ranks(total_ms, device=device)
-
-    # A workload that fits in L2 (126 MB) is also timed cold: a 512 MB buffer is
-    # rewritten between launches and only the merge is bracketed by events.
-    cold_ms = None
-    if w.algorithmic_bytes(out_bf16=args.out_bf16) < 4 * 126e6:
-        flush = torch.empty(512 << 20, dtype=torch.uint8, device=device)
-        cold = []
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        for k in range(min(args.steps, 20)):
-            flush.fill_(k & 0xff)
-            e0.record(stream)
-            step()
-            e1.record(stream)
-            e1.synchronize()
-            cold.append(e0.elapsed_time(e1))
-        cold_ms = {"median": statistics.median(cold), "min": min(cold), "max": max(cold)}
-        del flush
-
-    # A single small fragment is launch-bound from Python (the host needs longer to issue a
-    # merge than the GPU to run it): the same calls captured once into a CUDA graph and
-    # replayed give the device-bound time per merge.  The library call is capture-safe
-    # (one kernel launch, no allocation or synchronisation once the workspace exists).
-    graph_ms = None
-    if cold_ms is not None and w.P == 1 and args.merge == "avg":
-        side = torch.cuda.Stream(device=device)
-        graph = torch.cuda.CUDAGraph()
-        reps = 50
-        with torch.cuda.stream(side):
-            with torch.cuda.graph(graph, stream=side):
-                for _ in range(reps):
-                    step(side)
-        torch.cuda.synchronize()
-        times = []
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        for _ in range(8):
-            e0.record()
-            graph.replay()
-            e1.record()
-            e1.synchronize()
-            times.append(e0.elapsed_time(e1) / reps)
-        graph_ms = {"median": statistics.median(times[3:]), "min": min(times[3:]), "merges_per_graph": reps}
-        del graph
-
-    params_per_step = w.total_params
     value = ddist.whole_job_rate(job_params, args.steps, 1, max_ms)
-    alg_bytes = w.algorithmic_bytes(out_bf16=args.out_bf16)
-    launches_per_step = 1
-    if args.merge == "int4":
-        alg_bytes = sum(int(n * (w.participants(p) * (0.5 + 4.0 / 128.0) + 16))
-                        for p, n in enumerate(w.fragment_sizes))
-    if args.merge == "rda":
-        # learner copies and Theta are read twice (norms, direction), the direction is
-        # written and read back once: 2 (s b + 4) + 24 bytes per parameter
-        esz = 2 if w.learner_dtype == "bf16" else 4
-        alg_bytes = sum(n * (2 * (w.participants(p) * esz + 4) + 24)
-                        for p, n in enumerate(w.fragment_sizes))
-        launches_per_step = 3
-    avg_launch_ms = sum(per_launch_ms) / len(per_launch_ms)
-    slowest = sorted(range(len(per_launch_ms)), key=lambda k: -per_launch_ms[k])[:3]
-    achieved = alg_bytes / (avg_launch_ms * 1e-3) / 1e9
-    peak, peak_kind = hbm_peak()
-    traffic_pp = None if args.out_bf16 else NCU_TRAFFIC_BYTES_PER_PARAM.get((args.merge, args.workload))
-    roofline = {
-        "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-        "frac": achieved / peak, "peak_source": f"of {peak_kind}",
-        "traffic": None if traffic_pp is None else traffic_pp * params_per_step,
-        "algorithmic_bytes_per_launch": alg_bytes,
-        "bytes_per_param": alg_bytes / params_per_step,
-        "kernel_ms": {"avg": avg_launch_ms, "median": statistics.median(per_launch_ms),
-                      "min": min(per_launch_ms), "max": max(per_launch_ms),
-                      "slowest_steps": slowest},
-        "frac_of_nominal_8TBs": achieved / 8000.0,
-    }
-    if graph_ms is not None:
-        roofline["ms_per_merge_cuda_graph_replay"] = graph_ms
-    if cold_ms is not None:
-        roofline["kernel_ms_l2_flushed"] = cold_ms
-        roofline["achieved_l2_flushed"] = alg_bytes / (cold_ms["median"] * 1e-3) / 1e9
-    if not args.no_ceilings:
-        roofline["same_run_ceilings"] = measure_ceilings(device)
+    roofline = roofline_of(w, args.merge, args.out_bf16, per_launch_ms, ceilings, traffic_table, args.workload)
+    roofline["kernel_ms"]["slowest_steps"] = sorted(range(len(per_launch_ms)), key=lambda k: -per_launch_ms[k])[:3]
+    alg_bytes = roofline["algorithmic_bytes_per_launch"]
+    fits_l2 = alg_bytes < 4 * L2_BYTES
+    if fits_l2:
+        roofline["kernel_ms_l2_flushed"] = merger.timed_cold(min(args.steps, 20))
+        roofline["achieved_l2_flushed"] = alg_bytes / (roofline["kernel_ms_l2_flushed"]["median"] * 1e-3) / 1e9
+        if w.P == 1 and args.merge == "avg":
+            roofline["ms_per_merge_cuda_graph_replay"] = merger.timed_graph()
+    if ceilings:
+        roofline["same_run_ceilings"] = ceilings
+        roofline["frac_of_mix_ceiling"] = roofline["achieved"] / ceilings["mix_gbs"]
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -581,116 +1018,70 @@ def main():
         "scaling": "weak" if args.sharding == "replica" else "strong", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {
-            "workload": w.name, "fragments": w.P, "params_per_step": params_per_step, "M": w.M,
-            "participants": [w.participants(p) for p in range(w.P)],
-            "learner_dtype": w.learner_dtype, "state_dtype": "f32", "outer_lr": eta,
-            "outer_mu": mu, "flags": "nesterov+diag_state", "out_bf16": bool(args.out_bf16),
+            "workload": w.name, "fragments": w.P, "params_per_step": w.total_params, "M": w.M,
+            "participants": [participants(w, p) for p in range(w.P)],
+            "learner_dtype": w.learner_dtype, "state_dtype": "f32", "outer_lr": merger.eta,
+            "outer_mu": merger.mu, "flags": "nesterov+diag_state", "out_bf16": bool(args.out_bf16),
             "merge": args.merge,
             "grid": grid, "block": block, "tile_elems": tile,
-            "l2": "inputs larger than L2 (no flush)" if alg_bytes > 4 * 126e6
-                  else "fits L2: timed warm (back to back) and cold (512 MB flush between launches)",
+            "l2": "fits L2: timed warm (back to back) and cold (512 MB flush between launches)" if fits_l2
+                  else "inputs larger than L2 (no flush)",
             "parallelism": f"{args.sharding} x{world}" if world > 1 else "single",
         },
-        "clocks": sampler.summary(),
-        "gpu_launches": args.steps * launches_per_step,
+        "clocks": clocks,
+        "gpu_launches": args.steps * merger.launches_per_step,
         "roofline": roofline,
     }
 
-    # ---- end to end: host buffers through dd_merge_fragment_host -------------------
     if not args.no_e2e and w.P == 1 and args.merge == "avg":
-        f = frags[0]
-        n = f["n"]
-        part = [m for m in range(w.M) if (f["quorum_mask"] >> m) & 1 and f["tokens"][m] > 0]
-        # Page-locked host memory is bounded: every rank of the node pins its own buffers, so
-        # with several ranks (or little free host memory) the end-to-end leg streams a leading
-        # slice of the fragment instead of all of it.
-        esz0 = 2 if w.learner_dtype == "bf16" else 4
-        per_elem = len(part) * esz0 + 8
-        try:
-            avail = next(int(l.split()[1]) * 1024 for l in open("/proc/meminfo") if l.startswith("MemAvailable"))
-        except Exception:
-            avail = 64 << 30
-        local_world = int(os.environ.get("LOCAL_WORLD_SIZE", str(world)))
-        budget = int(0.4 * avail / max(local_world, 1))
-        n = max(8, min(n, budget // per_elem) // 8 * 8)
-        h_theta = torch.empty(n, dtype=torch.float32, pin_memory=True)
-        h_mom = torch.empty(n, dtype=torch.float32, pin_memory=True)
-        h_theta.copy_(f["global_"][:n])
-        h_mom.copy_(f["momentum"][:n])
-        h_learners = [None] * w.M
-        for m in part:
-            h_learners[m] = torch.empty(n, dtype=f["learners"][m].dtype, pin_memory=True)
-            h_learners[m].copy_(f["learners"][m][:n])
-        esz = 2 if w.learner_dtype == "bf16" else 4
-        h2d = n * (len(part) * esz + 8)
-        d2h = n * 8 + dd.RECORD_BYTES
-        ctx.merge_fragment_host(h_theta, h_mom, h_learners, f["tokens"], f["quorum_mask"], f["K"],
-                                eta, mu, n=n, learner_dtype=ldtype, flags=flags)      # warm-up
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        for _ in range(args.e2e_steps):
-            rec = ctx.merge_fragment_host(h_theta, h_mom, h_learners, f["tokens"],
-                                          f["quorum_mask"], f["K"], eta, mu, n=n,
-                                          learner_dtype=ldtype, flags=flags)
-        torch.cuda.synchronize()
-        dt = time.perf_counter() - t0
-        assert rec.status == 0
-        dt_max = ddist.max_over_ranks(dt, device=device)
-        # every rank streams its own copy (or its own range) of n elements per step
-        e2e_params = n * world
-        line["e2e"] = {"value": e2e_params * args.e2e_steps / dt_max, "unit": UNIT,
-                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                       "steps": args.e2e_steps, "elements_per_rank_step": n,
-                       "path": "dd_merge_fragment_host: pinned host buffers, chunked H2D -> "
-                               "kernel -> D2H pipeline, blocking"}
-        del h_learners, h_theta, h_mom
+        line["e2e"] = e2e_leg(dd, ctx, merger, args, world)
     else:
         line["e2e"] = None
-
     if parity is not None:
         line["parity"] = parity
-
-    # ---- the oracle on the host cores, bounded sample of the same workload -----------
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        import oracle
-        f = frags[0]
-        ns = min(args.cpu_sample, f["n"])
-        part = [m for m in range(w.M) if (f["quorum_mask"] >> m) & 1 and f["tokens"][m] > 0]
-        theta = f["global_"][:ns].cpu().numpy()
-        mom = f["momentum"][:ns].cpu().numpy()
-        learners = [None] * w.M
-        for m in part:
-            t_m = f["learners"][m][:ns].cpu()
-            learners[m] = (t_m.view(torch.int16).numpy().view(np.uint16)
-                           if w.learner_dtype == "bf16" else t_m.numpy())
-        oracle.build()
-        t0 = time.perf_counter()
-        oracle.merge_fragment(theta, mom, learners, f["tokens"], f["quorum_mask"], f["K"], eta, mu)
-        dt = time.perf_counter() - t0
-        line["cpu_baseline"] = {
-            "value": ns / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"first {ns} elements of fragment 0 of {w.name}, {len(part)} participating "
-                      f"{w.learner_dtype} learners, one merge, {dt:.1f} s, single thread of "
-                      f"{os.cpu_count()} host cores",
-            "host_cpu": host_cpu_model(), "host_cores": os.cpu_count(),
-            "affinity_cores": len(os.sched_getaffinity(0))}
-        # Beside it, because the paper's own syncer is a CPU program: the same element loop
-        # spread over all host cores (OpenMP; not the checked oracle, a timing baseline only).
-        try:
-            cores = len(os.sched_getaffinity(0))
-            t0 = time.perf_counter()
-            oracle.merge_fragment_all_cores(theta, mom, learners, f["tokens"], f["quorum_mask"], f["K"],
-                                            eta, mu)
-            dt_all = time.perf_counter() - t0
-            line["cpu_baseline"]["all_cores"] = {"value": ns / dt_all, "unit": UNIT, "cores": cores,
-                                                 "kind": "oracle element loop under OpenMP",
-                                                 "seconds": dt_all}
-        except Exception as exc:      # no OpenMP runtime on the box: the oracle figure stands alone
-            line["cpu_baseline"]["all_cores"] = {"unavailable": str(exc)[:120]}
+        line["cpu_baseline"] = cpu_baseline_leg(merger, args)
     elif rank == 0:
         line["cpu_baseline"] = None
+
+    # ---- one row per other workload and merge kind (N = 1 only) ------------------------------
+    if rank == 0 and world == 1 and args.scale == 1.0:
+        rows = []
+        todo = wanted_configs(args, args.workload, args.merge)
+        for name in [x for x in todo if x in ("rda", "int4")]:
+            # the other merge kinds of the headline workload, on the buffers that are already resident
+            if w.P == 1 and args.merge == "avg" and w.learner_dtype == "bf16":
+                rows.append(config_row(dd, ctx, device, args.workload, name, args, ceilings, probes,
+                                       traffic_table, merger=merger))
+        merger.free()
+        merger = None
+        for name in [x for x in todo if x not in ("rda", "int4", "tape24")]:
+            rows.append(config_row(dd, ctx, device, name, "avg", args, ceilings, probes, traffic_table,
+                                   resident="participants" if name == "moe4b" else "all"))
+        if probes is not None:
+            probes.close()
+            probes = None
+        if "tape24" in todo:
+            sub = parse_args(["--workload", "tape24", "--steps", "48", "--warmup", "24"])
+            tl = run_replay(sub, ceilings)
+            rows.append({"workload": "tape24", "merge": "avg + fused push", "fragments": 24,
+                         "params": tl["config"]["model_params"], "M": 8,
+                         "ms": {"avg": tl["ms_per_step"]}, "params_per_s": tl["value"],
+                         "achieved_gbs": tl["roofline"]["achieved"], "frac": tl["roofline"]["frac"],
+                         "frac_of_nominal_8TBs": tl["roofline"]["frac_of_nominal_8TBs"],
+                         "write_share": tl["roofline"]["write_share"],
+                         "blend_ceiling_gbs": tl["roofline"].get("blend_ceiling_gbs"),
+                         "frac_of_blend_ceiling": tl["roofline"].get("frac_of_blend_ceiling"),
+                         "steps": 48, "launches_per_merge": 1, "sm_mhz": tl["clocks"]["sm_mhz"],
+                         "clock_reasons": tl["clocks"]["reasons"],
+                         "note": "one syncer step per bench step: dd_select_quorum + one launch that "
+                                 "merges the due fragment and pushes it to the learners that are up; "
+                                 "host work included"})
+        line["configs"] = rows
+    if merger is not None:
+        merger.free()
+    if probes is not None:
+        probes.close()
 
     if rank == 0:
         print(json.dumps(line), flush=True)
@@ -699,5 +1090,20 @@ def main():
         dist.destroy_process_group()
 
 
+def main(argv=None):
+    argv = list(sys.argv[1:] if argv is None else argv)
+    args = parse_args(argv)
+    if args.dry_launch:
+        print(json.dumps(launch_plan(max(args.gpus, 1), [a for a in argv if a != "--dry-launch"])), flush=True)
+        return 0
+    if args.impl == "reference":
+        run_reference(args)
+        return 0
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return spawn_ranks(args, argv)
+    run_ours(args)
+    return 0
+
+
 if __name__ == "__main__":
-    main()
+    sys.exit(main())

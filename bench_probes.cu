@@ -1,0 +1,217 @@
+// Bandwidth probes for bench.py (measurement code; not part of libddmerge).
+//
+// One kernel reproduces the data movement of the fused merge with the arithmetic left
+// out: every warp owns a ring of three 2 KB shared-memory slots that its lane 0 fills
+// with bulk asynchronous copies (cp.async.bulk, no tensor map, addressed to this CTA
+// only), two pieces ahead of the one being consumed; a row is 1024 elements of every
+// stream; results leave through 32-byte-per-lane streaming stores (st.global.cs.v8).
+// The number of streams of each kind is a launch argument, so the same kernel gives
+//   - a read-only ceiling          (24 two-byte streams, nothing written),
+//   - a write-only ceiling         (two four-byte streams, nothing read),
+//   - the merge's own mix          (s two-byte + two four-byte streams read, the two
+//                                   four-byte streams rewritten in place),
+//   - the push / broadcast shapes  (additional two-byte streams written).
+// What is written depends on what was read, so the stores carry computed data.
+//
+// C ABI: ddp_stream_probe() below.  The caller owns the device buffer; nothing here
+// allocates device memory.  Every wait is bounded; a wait that runs out sets an error
+// word at the start of the buffer and the call returns a negative number.
+#include <cstdint>
+#include <cstring>
+
+#include <cuda_runtime.h>
+
+namespace {
+
+constexpr int kWarps = 8, kThreads = 256, kStages = 3;
+constexpr int kWaitLimit = 1 << 16;          // attempts of up to 4 us each
+constexpr int kMaxStreams = 64;
+
+__device__ __forceinline__ unsigned smem_addr(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ bool wait_bounded(unsigned bar, unsigned parity)
+{
+    for (int i = 0; i < kWaitLimit; ++i) {
+        unsigned ok;
+        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+                     " selp.u32 %0, 1, 0, p;\n}"
+                     : "=r"(ok) : "r"(bar), "r"(parity), "r"(4000u) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+
+struct Args {
+    const char *rd2[kMaxStreams];
+    char *wr2[kMaxStreams];
+    const char *rd4[2];
+    char *wr4[2];
+    int n_rd2, n_rd4, n_wr4, n_wr2;
+    unsigned long long rows;            // rows of 1024 elements per stream
+    int *err;
+};
+
+__device__ __forceinline__ void st_v8(void *p, uint4 a, uint4 b)
+{
+    asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 :: "l"(p), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w)
+                 : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 2) stream_probe_kernel(const __grid_constant__ Args a)
+{
+    extern __shared__ __align__(128) unsigned char ring_base[];
+    __shared__ unsigned long long bars[kWarps * kStages];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned char *ring = ring_base + (size_t)warp * kStages * 2048;
+    const unsigned ring_s = smem_addr(ring), bar_s = smem_addr(bars + warp * kStages);
+    if (lane == 0)
+        for (int d = 0; d < kStages; ++d)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar_s + 8u * d), "r"(1u) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+
+    const unsigned long long stride = (unsigned long long)gridDim.x * kWarps;
+    const unsigned long long first = (unsigned long long)blockIdx.x * kWarps + warp;
+    const int npieces = 2 * a.n_rd4 + a.n_rd2;      // order: rd4[0] halves, rd2 pieces, rd4[1] halves
+    unsigned long long irow = first;
+    int ipiece = 0, islot = 0, cslot = 0;
+    unsigned cphase = 0;
+    bool failed = false;
+    auto issue = [&]() {
+        if (failed || npieces == 0 || irow >= a.rows) return;
+        if (lane == 0) {
+            const char *src;
+            const int lead = a.n_rd4 > 0 ? 2 : 0;
+            if (ipiece < lead) src = a.rd4[0] + irow * 4096 + ipiece * 2048;
+            else if (ipiece - lead < a.n_rd2) src = a.rd2[ipiece - lead] + irow * 2048;
+            else src = a.rd4[1] + irow * 4096 + (ipiece - lead - a.n_rd2) * 2048;
+            const unsigned bar = bar_s + 8u * islot;
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(2048u) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         :: "r"(ring_s + 2048u * islot), "l"(src), "r"(2048u), "r"(bar) : "memory");
+        }
+        if (++ipiece == npieces) { ipiece = 0; irow += stride; }
+        if (++islot == kStages) islot = 0;
+    };
+    for (int p = 0; p < kStages - 1; ++p) issue();
+
+    unsigned keep = 0;
+    for (unsigned long long row = first; row < a.rows && !failed; row += stride) {
+        uint4 acc[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) acc[r] = make_uint4(lane, r, (unsigned)row, 7u);
+        for (int p = 0; p < npieces; ++p) {
+            __syncwarp();                               // the slot consumed last is free again
+            issue();
+            const bool ok = wait_bounded(bar_s + 8u * cslot, cphase);
+            if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+            const unsigned char *slot = ring + cslot * 2048;
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const uint4 x = *reinterpret_cast<const uint4 *>(slot + r * 512 + lane * 16);
+                acc[r].x ^= x.x; acc[r].y += x.y; acc[r].z ^= x.z; acc[r].w += x.w;
+            }
+            if (++cslot == kStages) { cslot = 0; cphase ^= 1u; }
+        }
+        if (failed) break;
+        for (int q = 0; q < a.n_wr4; ++q)
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+                st_v8(a.wr4[q] + row * 4096 + (r * 32 + lane) * 32, acc[r], acc[(r + 1) & 3]);
+        for (int q = 0; q < a.n_wr2; ++q)
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+                __stcs(reinterpret_cast<uint4 *>(a.wr2[q] + row * 2048 + (r * 32 + lane) * 16), acc[r]);
+        keep ^= acc[0].x ^ acc[1].y ^ acc[2].z ^ acc[3].w;
+    }
+    if (failed) {
+        // one bounded look at every slot still owed a copy, then report
+        for (int d = 0; d < kStages; ++d) (void)wait_bounded(bar_s + 8u * d, 0u);
+        if (lane == 0) atomicExch(a.err, 1);
+    } else if (keep == 0x9e3779b9u && a.n_wr4 + a.n_wr2 == 0) {
+        a.err[1] = 1;                                   // keeps the reads of a read-only run alive
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+// Runs the probe `reps` times (after two warm-up launches) on `cuda_stream` and returns the
+// best rate in GB/s of (bytes read + bytes written) over the CUDA-event time of one launch;
+// *best_ms receives that time.  Streams are carved from `buffer` (device memory, 256-byte
+// aligned, `buffer_bytes` long): n_rd2 / n_wr2 streams of 2 bytes per element, n_rd4 / n_wr4
+// of 4 bytes per element, `elems` elements each (rounded down to a multiple of 1024).  As in
+// the merge, the four-byte outputs are the four-byte inputs (in place) when both exist;
+// two-byte outputs overwrite the two-byte inputs when `push_in_place` is set, else they are
+// streams of their own.  ctas_per_sm sizes the persistent grid (2 is the merge's shape).
+// Returns -1 for bad arguments or a buffer that is too small, -2 for a CUDA error, -3 when a
+// bounded wait ran out on the device.
+double ddp_stream_probe(void *buffer, size_t buffer_bytes, int n_rd2, int n_rd4, int n_wr4, int n_wr2,
+                        size_t elems, int push_in_place, int ctas_per_sm, int reps, void *cuda_stream,
+                        double *best_ms)
+{
+    if (!buffer || n_rd2 < 0 || n_rd2 > kMaxStreams || n_wr2 < 0 || n_wr2 > kMaxStreams || n_rd4 < 0 ||
+        n_rd4 > 2 || n_wr4 < 0 || n_wr4 > 2 || ctas_per_sm < 1 || reps < 1 || ((uintptr_t)buffer & 255u))
+        return -1.0;
+    const unsigned long long rows = elems / 1024;
+    if (rows == 0) return -1.0;
+    Args a;
+    std::memset(&a, 0, sizeof a);
+    a.n_rd2 = n_rd2; a.n_rd4 = n_rd4; a.n_wr4 = n_wr4; a.n_wr2 = n_wr2; a.rows = rows;
+    char *base = static_cast<char *>(buffer);
+    size_t used = 256;                                   // the error words live in the first 256 bytes
+    a.err = reinterpret_cast<int *>(base);
+    auto take = [&](size_t bytes) -> char * {
+        char *p = base + used;
+        used += (bytes + 255) / 256 * 256;
+        return p;
+    };
+    for (int i = 0; i < n_rd2; ++i) a.rd2[i] = take(rows * 2048);
+    for (int i = 0; i < n_rd4; ++i) a.rd4[i] = take(rows * 4096);
+    for (int i = 0; i < n_wr4; ++i) a.wr4[i] = i < n_rd4 ? const_cast<char *>(a.rd4[i]) : take(rows * 4096);
+    for (int i = 0; i < n_wr2; ++i)
+        a.wr2[i] = push_in_place && i < n_rd2 ? const_cast<char *>(a.rd2[i]) : take(rows * 2048);
+    if (used > buffer_bytes) return -1.0;
+
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int dev = 0, sms = 0, fit = 0;
+    const size_t smem = (size_t)kWarps * kStages * 2048;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaFuncSetAttribute(stream_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&fit, stream_probe_kernel, kThreads, smem) != cudaSuccess ||
+        cudaMemsetAsync(a.err, 0, 256, stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return -2.0;
+    }
+    if (ctas_per_sm > fit) ctas_per_sm = fit;
+    unsigned long long grid = (unsigned long long)sms * ctas_per_sm;
+    if (grid > (rows + kWarps - 1) / kWarps) grid = (rows + kWarps - 1) / kWarps;
+    cudaEvent_t e0, e1;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return -2.0;
+    float best = 0.0f;
+    bool bad = false;
+    for (int r = -2; r < reps && !bad; ++r) {
+        cudaEventRecord(e0, stream);
+        stream_probe_kernel<<<(unsigned)grid, kThreads, smem, stream>>>(a);
+        cudaEventRecord(e1, stream);
+        float ms = 0.0f;
+        if (cudaEventSynchronize(e1) != cudaSuccess || cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) bad = true;
+        if (r >= 0 && (best == 0.0f || ms < best)) best = ms;
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    int err = 0;
+    if (bad || cudaMemcpy(&err, a.err, sizeof err, cudaMemcpyDeviceToHost) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return -2.0;
+    }
+    if (err) return -3.0;
+    if (best_ms) *best_ms = best;
+    const double bytes = (double)rows * (2048.0 * (n_rd2 + n_wr2) + 4096.0 * (n_rd4 + n_wr4));
+    return bytes / (best * 1e-3) / 1e9;
+}
+
+}  // extern "C"

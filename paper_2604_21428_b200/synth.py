@@ -50,20 +50,6 @@ class Workload:
     def total_params(self) -> int:
         return int(sum(self.fragment_sizes))
 
-    def participants(self, p: int) -> int:
-        """Number of learners with mask bit set and a positive token count."""
-        return sum(1 for m in range(self.M)
-                   if (self.masks[p] >> m) & 1 and int(self.tokens[p, m]) > 0)
-
-    def algorithmic_bytes(self, out_bf16: bool = False) -> int:
-        """Bytes the merge must move: every participant's copy once, the global
-        fragment and the momentum read once and written once."""
-        b_theta = 2 if self.learner_dtype == "bf16" else 4
-        total = 0
-        for p, n in enumerate(self.fragment_sizes):
-            total += n * (self.participants(p) * b_theta + 16 + (2 if out_bf16 else 0))
-        return total
-
 
 def dense_layer_params(d: int, d_ff: int) -> int:
     return 4 * d * d + 2 * d * d_ff + 2 * d

@@ -1,4 +1,5 @@
-"""bench.py's reference arm (the oracle on the host cores) prints the agreed JSON line."""
+"""bench.py without a GPU: the reference arm (the oracle on the host cores) prints the agreed JSON
+line, --gpus N plans one rank per GPU, and the byte accounting matches the stated formulas."""
 import json
 import os
 import subprocess
@@ -30,3 +31,55 @@ def test_reference_arm_other_ranks_do_nothing():
                           "--gpus", "2", "--steps", "1"], capture_output=True, text=True,
                          timeout=120, cwd=ROOT, env=env)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_dry_launch_plans_one_rank_per_gpu():
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4", "--steps", "7",
+                          "--dry-launch"], capture_output=True, text=True, timeout=120, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    plan = json.loads(out.stdout)
+    assert [item["rank"] for item in plan] == [0, 1, 2, 3]
+    ports = {item["env"]["MASTER_PORT"] for item in plan}
+    assert len(ports) == 1 and 1024 < int(ports.pop()) < 65536
+    for r, item in enumerate(plan):
+        env = item["env"]
+        assert env["RANK"] == env["LOCAL_RANK"] == str(r)
+        assert env["WORLD_SIZE"] == env["LOCAL_WORLD_SIZE"] == "4" and env["MASTER_ADDR"] == "127.0.0.1"
+        assert item["argv"][1].endswith("bench.py") and item["argv"][2:] == ["--gpus", "4", "--steps", "7"]
+
+
+def test_spawned_ranks_run_with_their_environment(tmp_path):
+    # the launcher itself, with a stand-in for the ranks' work: every rank of the reference arm but
+    # rank 0 exits silently, rank 0 prints the line -- so one line comes back from N processes
+    sys.path.insert(0, ROOT)
+    import bench
+    args = bench.parse_args(["--gpus", "3", "--impl", "reference", "--steps", "1", "--warmup", "0",
+                             "--workload", "tiny"])
+    script = tmp_path / "run.py"
+    script.write_text("import sys\nsys.path.insert(0, %r)\nimport bench\n"
+                      "sys.exit(bench.spawn_ranks(bench.parse_args(%r), %r))\n"
+                      % (ROOT, ["--gpus", "3"], ["--gpus", "3", "--impl", "reference", "--steps", "1",
+                                                 "--warmup", "0", "--workload", "tiny"]))
+    out = subprocess.run([sys.executable, str(script)], capture_output=True, text=True, timeout=600, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1 and json.loads(lines[0])["n_gpus"] == 3 and args.gpus == 3
+
+
+def test_byte_accounting_follows_the_stated_formulas():
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2604_21428_b200 import synth
+    w = synth.workload("scale500m")
+    assert bench.participants(w, 0) == 24
+    assert bench.algorithmic_bytes(w) == 500_000_000 * (24 * 2 + 16)
+    assert bench.algorithmic_bytes(w, out_bf16=True) == 500_000_000 * (24 * 2 + 18)
+    assert bench.algorithmic_bytes(w, "int4") == int(500_000_000 * (24 * (0.5 + 4 / 128) + 16))
+    assert abs(bench.write_share(w) - 8 / 64) < 1e-12
+    t = synth.workload("tiny")
+    assert bench.algorithmic_bytes(t) == (1 << 20) * (2 * 4 + 16)
+    d = synth.workload("dense150m")
+    assert [bench.participants(d, p) for p in range(d.P)] == [6] * 4
+    # no interference: all reads at the read ceiling, all writes at the write ceiling
+    assert abs(bench.blend_ceiling(7000.0, 7000.0, 0.3) - 7000.0) < 1e-9
+    assert abs(bench.blend_ceiling(8000.0, 4000.0, 0.5) - 1 / (0.5 / 8000 + 0.5 / 4000)) < 1e-9

@@ -70,7 +70,9 @@ def _run(name, n_windows, merges):
 
     w = synth.workload(name)
     # resident: the participants' copies, Theta and v (the algorithmic bytes count Theta and v twice)
-    need = w.algorithmic_bytes() - 8 * w.total_params
+    b_theta = 2 if w.learner_dtype == "bf16" else 4
+    need = sum(n * (8 + b_theta * sum(1 for m in range(w.M) if (w.masks[p] >> m) & 1 and int(w.tokens[p, m]) > 0))
+               for p, n in enumerate(w.fragment_sizes))
     free = _free_bytes()
     if free < need + (4 << 30):
         pytest.skip(f"needs {need >> 30} GiB of device memory, {free >> 30} GiB free")
