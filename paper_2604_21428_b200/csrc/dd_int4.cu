@@ -159,21 +159,12 @@ struct ScalePtrs {
     const float *p[DD_MAX_LEARNERS];
 };
 
-__global__ void __launch_bounds__(256, 3)
-merge_int4_kernel(const __grid_constant__ DevFrag frag, const __grid_constant__ ScalePtrs sp,
-                  const __grid_constant__ Common c)
+// The element loop of the int4 merge.  WIDE: Theta and v start on 32-byte boundaries and are
+// read and written with 256-bit accesses (two 128-bit ones otherwise).
+template <bool WIDE>
+__device__ __forceinline__ void int4_elements(Smem &sm, const float *const *sptr, const Common &c)
 {
-    __shared__ Smem sm;
-    __shared__ const float *sptr[DD_MAX_LEARNERS];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x < 32) {
-        load_header<kModeMerge>(&frag, 0, blockIdx.x, c, sm);
-        __syncwarp();
-        for (int j = lane; j < sm.n_part; j += 32) sptr[j] = sp.p[sm.idx[j]];
-    }
-    __syncthreads();
-    if (sm.status != DD_STATUS_OK) return;
-
     const unsigned long long n = sm.n;
     const unsigned long long nfull = n / 16;                      // whole 16-element steps
     const int s = sm.n_part;
@@ -226,8 +217,8 @@ merge_int4_kernel(const __grid_constant__ DevFrag frag, const __grid_constant__ 
         for (int h = 0; h < 2; ++h) {
             const unsigned v8 = (unsigned)(2 * vi + h);            // index of the 8-element half
             float T[8], V[8];
-            load_f32x8<false>(sm.theta, v8, T);
-            load_f32x8<false>(sm.mom, v8, V);
+            load_f32x8<WIDE>(sm.theta, v8, T);
+            load_f32x8<WIDE>(sm.mom, v8, V);
             float dsq = 0.0f, tsq = 0.0f, msq = 0.0f;
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
@@ -241,8 +232,8 @@ merge_int4_kernel(const __grid_constant__ DevFrag frag, const __grid_constant__ 
                 tsq = fmaf(tn, tn, tsq);
                 msq = fmaf(vn, vn, msq);
             }
-            store_f32x8<false>(sm.mom, v8, V);
-            store_f32x8<false>(sm.theta, v8, T);
+            store_f32x8<WIDE>(sm.mom, v8, V);
+            store_f32x8<WIDE>(sm.theta, v8, T);
             if (sm.out_bf16 != nullptr)
                 st_stream16(reinterpret_cast<uint4 *>(sm.out_bf16) + v8,
                             make_uint4(pack_bf16x2(T[0], T[1]), pack_bf16x2(T[2], T[3]),
@@ -278,6 +269,28 @@ merge_int4_kernel(const __grid_constant__ DevFrag frag, const __grid_constant__ 
         if (lane == 0) { sm.red[warp][0] = a_d; sm.red[warp][1] = a_t; sm.red[warp][2] = a_m; }
         flush_fragment<false>(sm, c);
     }
+}
+
+#ifndef DD_INT4_MINB
+#define DD_INT4_MINB 3
+#endif
+__global__ void __launch_bounds__(256, DD_INT4_MINB)
+merge_int4_kernel(const __grid_constant__ DevFrag frag, const __grid_constant__ ScalePtrs sp,
+                  const __grid_constant__ Common c)
+{
+    __shared__ Smem sm;
+    __shared__ const float *sptr[DD_MAX_LEARNERS];
+    const int lane = threadIdx.x & 31;
+    if (threadIdx.x < 32) {
+        load_header<kModeMerge>(&frag, 0, blockIdx.x, c, sm);
+        __syncwarp();
+        for (int j = lane; j < sm.n_part; j += 32) sptr[j] = sp.p[sm.idx[j]];
+    }
+    __syncthreads();
+    if (sm.status != DD_STATUS_OK) return;
+
+    if (sm.wide) int4_elements<true>(sm, sptr, c);
+    else int4_elements<false>(sm, sptr, c);
 }
 
 }  // namespace ddm
@@ -339,7 +352,7 @@ extern "C" int dd_merge_fragment_int4(dd_ctx *ctx, float *global, float *momentu
     if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
     const unsigned long long nvec = (n + 15) / 16;
     unsigned long long grid = (nvec + 255) / 256;
-    const unsigned long long cap = (unsigned long long)ctx->sm_count * 3;   // 3 CTAs of 256 threads per SM
+    const unsigned long long cap = (unsigned long long)ctx->sm_count * DD_INT4_MINB;   // resident CTAs of 256 threads per SM
     if (grid > cap) grid = cap;
     if (grid == 0) grid = 1;
     frag.tile_begin = 0;
