@@ -70,7 +70,7 @@ def parse_args(argv=None):
     ap.add_argument("--configs", default="all",
                     help="N = 1: which other workloads get a row in the line's 'configs' array: "
                          "'all', 'none', or a comma-separated list of "
-                         "tiny,dense150m,dense1b3,moe4b,rda,int4,tape24")
+                         "tiny,dense150m,dense1b3,moe4b,rda,int4,push,broadcast,tape24")
     ap.add_argument("--config-steps", type=int, default=20, help="timed launches per 'configs' row")
     ap.add_argument("--cpu-sample", type=int, default=1 << 27,
                     help="elements of the workload the CPU oracle is timed on")
@@ -106,6 +106,8 @@ def bytes_per_param(merge: str, s: int, b_theta: int, out_bf16: bool = False) ->
             stored direction: see rda_bytes_per_param."""
     if merge == "int4":
         return s * (0.5 + 4.0 / 128.0) + 16 + (2 if out_bf16 else 0)
+    if merge == "push":           # the merge, and Theta' written over every participant's copy
+        return 2 * s * b_theta + 16
     if merge == "rda":
         return rda_bytes_per_param(s, b_theta) + (2 if out_bf16 else 0)
     return s * b_theta + 16 + (2 if out_bf16 else 0)
@@ -126,7 +128,10 @@ def algorithmic_bytes(w, merge: str = "avg", out_bf16: bool = False) -> int:
 def write_share(w, merge: str = "avg", out_bf16: bool = False) -> float:
     """Fraction of the algorithmic bytes that are writes."""
     total = algorithmic_bytes(w, merge, out_bf16)
-    writes = sum(n * (8 + (2 if out_bf16 else 0) + (4 if merge == "rda" else 0)) for n in w.fragment_sizes)
+    b_theta = 2 if w.learner_dtype == "bf16" else 4
+    writes = sum(n * (8 + (2 if out_bf16 else 0) + (4 if merge == "rda" else 0) +
+                      (participants(w, p) * b_theta if merge == "push" else 0))
+                 for p, n in enumerate(w.fragment_sizes))
     return writes / total if total else 0.0
 
 
@@ -434,6 +439,7 @@ class Merger:
         self.flags = dd.DIAG_STATE
         self.eta, self.mu = synth.OUTER_LR, synth.OUTER_MU
         self.launches_per_step = 1
+        self.push_mask = 0              # learners whose copy the merge overwrites with Theta' (fused push)
         self.int4_codes = self.int4_scales = None
         self.rda_scratch = None
         if merge == "int4":
@@ -480,6 +486,11 @@ class Merger:
         elif self.merge == "rda":
             ctx.merge_fragments_batched_rda(self.frags, w.M, self.ldtype, self.eta, self.mu,
                                             flags=self.flags, records=self.records, stream=stream)
+        elif w.P == 1 and self.push_mask:
+            ctx.merge_fragment_push(f0["global_"], f0["momentum"], self.packed_ptrs, self.packed_tokens,
+                                    f0["quorum_mask"], f0["K"], self.eta, self.mu, self.push_mask, n=f0["n"],
+                                    learner_dtype=self.ldtype, flags=self.flags, record=self.records,
+                                    stream=stream)
         elif w.P == 1:
             ctx.merge_fragment(f0["global_"], f0["momentum"], self.packed_ptrs, self.packed_tokens,
                                f0["quorum_mask"], f0["K"], self.eta, self.mu, n=f0["n"],
@@ -530,6 +541,7 @@ class Merger:
         recs = self.dd.read_records(self.records)
         worst = {"t": 0.0, "v": 0.0}
         exact, nwin = True, 0
+        pushed_ok, pushed_same = True, 1.0
         for p in picks:
             f, rec = self.frags[p], recs[p]
             win, starts, per = saved[p]
@@ -544,16 +556,29 @@ class Merger:
                                                 self.eta, self.mu)
                 exact &= (rec.status, rec.n_part, rec.idx) == (ref.status, ref.n_part, ref.idx)
                 exact &= rec.w_hat == [float(np.float32(x)) for x in ref.w_hat]
+                if self.push_mask:
+                    # every pushed copy now holds Theta' rounded to the learner dtype
+                    want_bits = oracle.bf16_rne(t0)
+                    for m in range(w.M):
+                        if (self.push_mask >> m) & 1:
+                            pushed_ok &= bool(np.array_equal(host_learner(f["learners"][m][s0:s0 + win]),
+                                                             oracle.bf16_rne(f["global_"][s0:s0 + win].cpu().numpy())))
+                            same = np.mean(host_learner(f["learners"][m][s0:s0 + win]) == want_bits)
+                            pushed_same = min(pushed_same, float(same))
                 for got, want, which in ((f["global_"], t0, "t"), (f["momentum"], v0, "v")):
                     g = got[s0:s0 + win].cpu().numpy().astype(np.float64)
                     o = want.astype(np.float64)
                     rms = float(np.sqrt(np.mean(o * o))) or 1.0
                     worst[which] = max(worst[which], float(np.max(np.abs(g - o) / np.maximum(np.abs(o), rms))))
                 nwin += 1
-        return {"windows": nwin, "window_elems": saved[picks[0]][0], "fragments_sampled": len(picks),
-                "max_err_theta": worst["t"], "max_err_momentum": worst["v"], "tolerance": 1e-5,
-                "participation_and_weights_bit_exact": bool(exact),
-                "metric": "first merge: max |gpu - oracle| / max(|oracle|, rms(oracle))"}
+        out = {"windows": nwin, "window_elems": saved[picks[0]][0], "fragments_sampled": len(picks),
+               "max_err_theta": worst["t"], "max_err_momentum": worst["v"], "tolerance": 1e-5,
+               "participation_and_weights_bit_exact": bool(exact),
+               "metric": "first merge: max |gpu - oracle| / max(|oracle|, rms(oracle))"}
+        if self.push_mask:
+            out["pushed_copies_equal_rounded_theta"] = bool(pushed_ok)
+            out["pushed_bits_equal_to_oracle_fraction_min"] = pushed_same
+        return out
 
     def timed(self, steps: int, warmup: int, world: int = 1):
         """``warmup`` untimed steps, then ``steps`` timed ones bracketed by a barrier and a
@@ -680,7 +705,8 @@ def config_row(dd, ctx, device, name, merge, args, ceilings, probes, traffic_tab
     else:
         # another merge kind on buffers that are already resident: back to the seeded state first, so
         # that the parity windows below are again those of a FIRST merge
-        merger.merge = merge
+        merger.merge = "avg" if merge == "push" else merge
+        merger.push_mask = merger.frags[0]["quorum_mask"] if merge == "push" else 0
         merger.launches_per_step = 3 if merge == "rda" else 1
         for p, f in enumerate(merger.frags):
             synth.fill_fragment_gpu(f["global_"], f["momentum"], f["learners"], seed=w.seed * 1000 + p)
@@ -695,6 +721,8 @@ def config_row(dd, ctx, device, name, merge, args, ceilings, probes, traffic_tab
             row["parity"] = merger.first_merge_parity()
         _, per_launch, clocks = merger.timed(args.config_steps, 3)
         r = roofline_of(w, merge, False, per_launch, ceilings, traffic_table, name)
+        if merge == "push":
+            row["note"] = "the merge also overwrites every participant's copy with Theta' (fused push, in place)" 
         row.update({
             "ms": r["kernel_ms"], "params_per_s": w.total_params / (r["kernel_ms"]["avg"] * 1e-3),
             "bytes_per_param": r["bytes_per_param"], "write_share": r["write_share"],
@@ -715,6 +743,10 @@ def config_row(dd, ctx, device, name, merge, args, ceilings, probes, traffic_tab
                 row["ms_cuda_graph_replay"] = merger.timed_graph()
         else:
             row["l2"] = "inputs larger than L2 (no flush)"
+        if probes is not None and merge == "push" and w.learner_dtype == "bf16":
+            s_all = row["participants"][0]
+            row["pattern_probe_gbs"] = probes.run(rd2=s_all, rd4=2, wr4=2, wr2=s_all, push_in_place=True, reps=5)
+            row["frac_of_pattern_probe"] = row["achieved_gbs"] / row["pattern_probe_gbs"]
         if probes is not None and merge == "avg":
             # the same access pattern with the arithmetic left out, at this workload's mean participant count
             s_mean = max(1, round(sum(row["participants"]) / w.P))
@@ -724,6 +756,65 @@ def config_row(dd, ctx, device, name, merge, args, ceilings, probes, traffic_tab
     finally:
         if own:
             merger.free()
+    return row
+
+
+def broadcast_row(dd, ctx, merger, args, ceilings, probes):
+    """The learner side alone: Theta' read once and written (alpha = 0) over every participant's copy."""
+    import numpy as np
+    import torch
+
+    import oracle
+    w, f = merger.w, merger.frags[0]
+    n = f["n"]
+    mask = f["quorum_mask"]
+    k = participants(w, 0)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        ctx.broadcast_fragment(f["global_"], merger.packed_ptrs, mask, 0.0, n=n, learner_dtype=merger.ldtype,
+                               stream=stream)
+    for _ in range(3):
+        step()
+    events = [torch.cuda.Event(enable_timing=True) for _ in range(args.config_steps + 1)]
+    torch.cuda.synchronize()
+    events[0].record(stream)
+    for i in range(args.config_steps):
+        step()
+        events[i + 1].record(stream)
+    torch.cuda.synchronize()
+    ms = [events[i].elapsed_time(events[i + 1]) for i in range(args.config_steps)]
+    esz = 2 if w.learner_dtype == "bf16" else 4
+    alg = n * (4 + k * esz)
+    avg = sum(ms) / len(ms)
+    peak, _ = hbm_peak()
+    row = {"workload": w.name, "merge": "broadcast", "fragments": 1, "params": n, "M": w.M, "copies_written": k,
+           "learner_dtype": w.learner_dtype,
+           "ms": {"avg": avg, "median": statistics.median(ms), "min": min(ms), "max": max(ms)},
+           "params_per_s": n / (avg * 1e-3), "bytes_per_param": alg / n, "write_share": k * esz / (4 + k * esz),
+           "achieved_gbs": alg / (avg * 1e-3) / 1e9, "frac": alg / (avg * 1e-3) / 1e9 / peak,
+           "frac_of_nominal_8TBs": alg / (avg * 1e-3) / 1e9 / NOMINAL_HBM_GBS, "launches_per_merge": 1,
+           "steps": args.config_steps, "l2": "inputs larger than L2 (no flush)",
+           "note": "dd_broadcast_fragment, alpha = 0: the learner side of a syncer update on its own"}
+    if ceilings:
+        blend = blend_ceiling(ceilings["read_gbs"], ceilings["write_gbs"], row["write_share"])
+        row["blend_ceiling_gbs"] = blend
+        row["frac_of_blend_ceiling"] = row["achieved_gbs"] / blend
+        row["frac_of_write_ceiling"] = row["achieved_gbs"] / ceilings["write_gbs"]
+    if probes is not None and w.learner_dtype == "bf16":
+        row["pattern_probe_gbs"] = probes.run(rd4=1, wr2=k, reps=5)
+        row["frac_of_pattern_probe"] = row["achieved_gbs"] / row["pattern_probe_gbs"]
+    if not args.no_cpu_baseline:
+        # a window of every written copy against the oracle's rounding of the same Theta'
+        win = min(1 << 16, n)
+        want = oracle.bf16_rne(f["global_"][:win].cpu().numpy()) if esz == 2 else f["global_"][:win].cpu().numpy()
+        ok = True
+        for m in range(w.M):
+            if (mask >> m) & 1:
+                got = f["learners"][m][:win].cpu()
+                got = got.view(torch.int16).numpy().view(np.uint16) if esz == 2 else got.numpy()
+                ok &= bool(np.array_equal(got, want))
+        row["parity"] = {"windows": k, "window_elems": win, "copies_bit_equal_to_oracle_rounding": ok}
     return row
 
 
@@ -925,7 +1016,7 @@ def cpu_baseline_leg(merger, args):
 
 
 def wanted_configs(args, headline, headline_merge):
-    names = ["tiny", "dense150m", "dense1b3", "moe4b", "rda", "int4", "tape24"]
+    names = ["tiny", "dense150m", "dense1b3", "moe4b", "rda", "int4", "push", "broadcast", "tape24"]
     if args.configs == "none":
         return []
     if args.configs != "all":
@@ -1048,14 +1139,17 @@ def run_ours(args):
     if rank == 0 and world == 1 and args.scale == 1.0:
         rows = []
         todo = wanted_configs(args, args.workload, args.merge)
-        for name in [x for x in todo if x in ("rda", "int4")]:
+        for name in [x for x in todo if x in ("rda", "int4", "push", "broadcast")]:
             # the other merge kinds of the headline workload, on the buffers that are already resident
             if w.P == 1 and args.merge == "avg" and w.learner_dtype == "bf16":
-                rows.append(config_row(dd, ctx, device, args.workload, name, args, ceilings, probes,
-                                       traffic_table, merger=merger))
+                if name == "broadcast":
+                    rows.append(broadcast_row(dd, ctx, merger, args, ceilings, probes))
+                else:
+                    rows.append(config_row(dd, ctx, device, args.workload, name, args, ceilings, probes,
+                                           traffic_table, merger=merger))
         merger.free()
         merger = None
-        for name in [x for x in todo if x not in ("rda", "int4", "tape24")]:
+        for name in [x for x in todo if x not in ("rda", "int4", "push", "broadcast", "tape24")]:
             rows.append(config_row(dd, ctx, device, name, "avg", args, ceilings, probes, traffic_table,
                                    resident="participants" if name == "moe4b" else "all"))
         if probes is not None:

@@ -15,6 +15,10 @@ constexpr int kStepsPerLane = 4;         // 8-element steps a lane handles per w
 constexpr int kTileElems = kThreads * kVec * kStepsPerLane;   // 8192 elements per tile: 1024 per warp
 constexpr int kNumScalarDiag = 3;        // delta_sq, theta_sq, mom_sq
 constexpr unsigned long long kMaxFragmentElems = 1ull << 34;   // 8-element steps are indexed in 32 bits
+// Radial-directional merges of at most this many participants take the two-launch form through
+// the participants' Gram matrix (its s (s + 1) / 2 products run on the CUDA cores).
+#define DD_RDA_GRAM_MAX_PARTICIPANTS 8
+constexpr int kGramPairsMax = DD_RDA_GRAM_MAX_PARTICIPANTS * (DD_RDA_GRAM_MAX_PARTICIPANTS + 1) / 2;
 
 // One fragment as the kernel sees it.  Raw counters, mask and pointers travel to
 // the device; participation and weights are derived there.
@@ -49,6 +53,7 @@ struct Common {
     double *partials;                    // [P][nq][grid] per-CTA partial sums
     unsigned *tickets;                   // [P] completion counters, zero between calls
     int nq;                              // quantities per fragment in `partials`
+    double *gram = nullptr;              // [P][kGramPairsMax] Gram matrices (lower triangle) of the two-launch RDA
     int pl_cap = 0;                      // participants the per-lane norm area holds (0: none)
 };
 

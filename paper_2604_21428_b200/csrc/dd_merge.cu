@@ -390,6 +390,14 @@ static int merge_batched_impl(dd_ctx *ctx, const dd_fragment_desc *descs, const 
     if (P == 0) return DD_OK;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
 
+    if (P == 1) {
+        // one fragment travels in the kernel parameters: no staging slot, no descriptor copy
+        const dd_fragment_desc &d = descs[0];
+        return merge_fragment_impl(ctx, d.global, d.momentum, d.learner_ptrs, M, learner_dtype, d.tokens, d.steps,
+                                   d.quorum_mask, d.K, outer_lr, outer_mu, flags, (size_t)d.n,
+                                   push_masks ? push_masks[0] : 0, d.out_bf16, records, cuda_stream);
+    }
+
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
 

@@ -19,7 +19,9 @@ namespace ddm {
 // needs three: per-participant norms, the mean direction u = sum_j (w_j/||D_j||) D_j
 // written to a scratch array together with ||u||^2, and the outer step with
 // Delta = (sum_j w_j ||D_j||) u / ||u||.
-enum : int { kModeMerge = 0, kModeNorms = 1, kModeDir = 2, kModeApply = 3 };
+// With few participants two launches are enough: the Gram matrix of the outer gradients
+// (dd_rda_gram.cuh), then the ordinary merge with weights derived from it (kModeMergeGram).
+enum : int { kModeMerge = 0, kModeNorms = 1, kModeDir = 2, kModeApply = 3, kModeMergeGram = 4 };
 
 struct Smem {
     const void *ptr[DD_MAX_LEARNERS];    // participant j's buffer (compacted)
@@ -214,10 +216,36 @@ __device__ __forceinline__ void load_header(const DevFrag *f, int p, unsigned lo
         }
         __syncwarp();
     }
+    if (MODE == kModeMergeGram && f->kind == DD_MERGE_RDA && status == DD_STATUS_OK) {
+        // Second launch of the two-launch radial-directional merge: with G the Gram matrix of the
+        // outer gradients, ||D_j|| = sqrt(G_jj), a_j = w_hat_j / ||D_j|| (0 for a zero gradient),
+        // ||u||^2 = a^T G a, and Delta = sum_j (c a_j) D_j with c = (sum_j w_hat_j ||D_j||) / ||u||:
+        // the ordinary merge with other weights.  At most 8 participants: lane j owns participant j.
+        const double *g = c.gram + (size_t)p * kGramPairsMax;
+        const bool on = lane < n_part;
+        const double wj = on ? (double)sm.w[lane] : 0.0;
+        const double nj = on ? sqrt(__ldcg(g + lane * (lane + 1) / 2 + lane)) : 0.0;
+        const double aj = nj > 0.0 ? wj / nj : 0.0;
+        const double radial = warp_sum(wj * nj);
+        double row = 0.0;
+#pragma unroll
+        for (int k = 0; k < DD_RDA_GRAM_MAX_PARTICIPANTS; ++k) {
+            const double ak = __shfl_sync(0xffffffffu, aj, k);
+            if (on && k < n_part) {
+                const int hi = lane > k ? lane : k, lo = lane > k ? k : lane;
+                row += ak * __ldcg(g + hi * (hi + 1) / 2 + lo);
+            }
+        }
+        const double usq = warp_sum(on ? aj * row : 0.0);
+        const double cs = usq > 0.0 ? radial / sqrt(usq) : 0.0;
+        if (on) sm.w[lane] = (float)(cs * aj);
+        __syncwarp();
+    }
     // The CTA that owns the fragment's first tile publishes the header (once per
     // call: the later passes of a radial-directional merge leave it alone).
-    const bool publish = MODE == kModeMerge ? f->kind == DD_MERGE_AVG
-                                            : (MODE == kModeNorms && f->kind == DD_MERGE_RDA);
+    const bool publish = (MODE == kModeMerge || MODE == kModeMergeGram)
+                             ? f->kind == DD_MERGE_AVG
+                             : (MODE == kModeNorms && f->kind == DD_MERGE_RDA);
     if (publish && c.records != nullptr && tile == f->tile_begin) {
         dd_merge_record *rec = c.records + p;
         for (int j = lane; j < DD_MAX_LEARNERS; j += 32) {
@@ -299,14 +327,24 @@ __device__ __forceinline__ void process_tail(Smem &sm, const Common &c, unsigned
 
 // ---- step 6: per-CTA partials, ticket, fixed-order final reduce ----------------
 //
-// Wait-free: every CTA that worked on the fragment stores its partial sums,
-// fences, and draws a ticket; the CTA that draws the last ticket adds the
+// Wait-free: every CTA that worked on the fragment stores its partial sums and
+// draws a ticket (a release-acquire atomic); the CTA that draws the last ticket adds the
 // partials in a fixed order (so the result does not depend on CTA timing) and
 // re-arms the ticket for the next call.  The ticket word's top bit carries "some
 // CTA gave up a bounded wait in this fragment": a CTA sets it before it draws its
 // ticket, so the last CTA sees it from every CTA and reports DD_STATUS_WAIT_LIMIT
 // after the header (written by the CTA of the fragment's first tile) is in place.
 constexpr unsigned kTicketFailedBit = 0x80000000u;
+
+// Ticket draw with release and acquire semantics at GPU scope: everything this CTA wrote before
+// the barrier that precedes the call is visible to whoever draws a later ticket and then
+// synchronises its own CTA.  One such atomic replaces a fence per writer plus a fence per reader.
+__device__ __forceinline__ unsigned ticket_add_acq_rel(unsigned *addr, unsigned val)
+{
+    unsigned old;
+    asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], %2;" : "=r"(old) : "l"(addr), "r"(val) : "memory");
+    return old;
+}
 
 template <bool PL>
 __device__ __forceinline__ void flush_fragment(Smem &sm, const Common &c)
@@ -322,27 +360,24 @@ __device__ __forceinline__ void flush_fragment(Smem &sm, const Common &c)
 #pragma unroll
         for (int w = 0; w < kWarps; ++w) t += sm.red[w][threadIdx.x];
         part[(size_t)threadIdx.x * G + blockIdx.x] = t;
-        __threadfence();
     } else if (PL && threadIdx.x >= 32 && threadIdx.x < 32 + s) {
         const int j = threadIdx.x - 32;
         double t = 0.0;
 #pragma unroll
         for (int w = 0; w < kWarps; ++w) t += sm.dm[w][j];
         part[(size_t)(kNumScalarDiag + j) * G + blockIdx.x] = t;
-        __threadfence();
     }
     __syncthreads();
     const unsigned long long ntiles = sm.tile_end - sm.tile_begin;
     if (threadIdx.x == 0) {
         const unsigned expected = ntiles < G ? (unsigned)ntiles : G;
         if (sm.any_failed) atomicOr(c.tickets + p, kTicketFailedBit);
-        const unsigned ticket = atomicAdd(c.tickets + p, 1u);
+        const unsigned ticket = ticket_add_acq_rel(c.tickets + p, 1u);
         sm.is_last = (ticket & ~kTicketFailedBit) == expected - 1u;
         if (ticket & kTicketFailedBit) sm.any_failed = 1;
     }
     __syncthreads();
     if (!sm.is_last) return;
-    __threadfence();
     dd_merge_record *rec = c.records + p;
     const unsigned first = (unsigned)(sm.tile_begin % G);
     const int nq_used = kNumScalarDiag + (PL ? s : 0);

@@ -421,7 +421,8 @@ __device__ __forceinline__ void merge_body_tma(const DevFrag *frags, const Commo
         cur = sm.frag;
         const unsigned long long tile_end = sm.tile_end;
         const unsigned long long mine = (tile_end - tile + G - 1) / G;      // this CTA's tiles in the fragment
-        const bool plain = MODE == kModeMerge || (MODE == kModeApply && sm.kind == DD_MERGE_AVG);
+        const bool plain = MODE == kModeMerge || MODE == kModeMergeGram ||
+                           (MODE == kModeApply && sm.kind == DD_MERGE_AVG);
         const bool worked_on = sm.status == DD_STATUS_OK && (plain || sm.kind == DD_MERGE_RDA);
         if (worked_on) {
             // A warp whose ring failed in an earlier fragment skips its rows of this one too: the
