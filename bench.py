@@ -70,7 +70,7 @@ def parse_args(argv=None):
     ap.add_argument("--configs", default="all",
                     help="N = 1: which other workloads get a row in the line's 'configs' array: "
                          "'all', 'none', or a comma-separated list of "
-                         "tiny,dense150m,dense1b3,moe4b,rda,int4,push,broadcast,tape24")
+                         "tiny,dense150m,dense1b3,moe4b,rda,rda_dense150m,int4,push,broadcast,tape24")
     ap.add_argument("--config-steps", type=int, default=20, help="timed launches per 'configs' row")
     ap.add_argument("--cpu-sample", type=int, default=1 << 27,
                     help="elements of the workload the CPU oracle is timed on")
@@ -80,6 +80,9 @@ def parse_args(argv=None):
     ap.add_argument("--merge", choices=["avg", "rda", "int4"], default="avg",
                     help="weighted direct averaging (the headline path), radial-directional, or "
                          "direct averaging of int4-compressed outer gradients")
+    ap.add_argument("--rda-three-pass", action="store_true",
+                    help="--merge rda: force the three-launch form (norms, direction, apply) where the "
+                         "two-launch form through the Gram matrix would be taken")
     ap.add_argument("--resident", choices=["all", "participants"], default="all",
                     help="allocate every learner copy, or only those that take part")
     ap.add_argument("--sharding", choices=["replica", "range"], default="replica",
@@ -97,7 +100,7 @@ def participants(w, p: int) -> int:
     return sum(1 for m in range(w.M) if (w.masks[p] >> m) & 1 and int(w.tokens[p, m]) > 0)
 
 
-def bytes_per_param(merge: str, s: int, b_theta: int, out_bf16: bool = False) -> float:
+def bytes_per_param(merge: str, s: int, b_theta: int, out_bf16: bool = False, rda_three_pass: bool = False) -> float:
     """Algorithmic bytes per merged parameter: every participant's payload once, the global
     fragment and the momentum read once and written once.
       avg   s b + 16 (+ 2 with the bf16 copy)
@@ -109,27 +112,41 @@ def bytes_per_param(merge: str, s: int, b_theta: int, out_bf16: bool = False) ->
     if merge == "push":           # the merge, and Theta' written over every participant's copy
         return 2 * s * b_theta + 16
     if merge == "rda":
-        return rda_bytes_per_param(s, b_theta) + (2 if out_bf16 else 0)
+        return rda_bytes_per_param(s, b_theta, rda_three_pass) + (2 if out_bf16 else 0)
     return s * b_theta + 16 + (2 if out_bf16 else 0)
 
 
-def rda_bytes_per_param(s: int, b_theta: int) -> float:
-    """Three passes: norms (copies + Theta), direction (copies + Theta, write u), apply (Theta, v,
-    u read; Theta, v written) = 2 (s b + 4) + 24."""
+RDA_GRAM_MAX_PARTICIPANTS = 8
+
+
+def rda_bytes_per_param(s: int, b_theta: int, three_pass: bool = False) -> float:
+    """Up to 8 participants, two launches: the Gram matrix of the outer gradients (copies + Theta)
+    and the ordinary merge (copies, Theta, v read; Theta, v written) = 2 s b + 20.  Otherwise three:
+    norms (copies + Theta), direction (copies + Theta, write u), apply (Theta, v, u read; Theta, v
+    written) = 2 (s b + 4) + 24."""
+    if s <= RDA_GRAM_MAX_PARTICIPANTS and not three_pass:
+        return 2 * s * b_theta + 20
     return 2 * (s * b_theta + 4) + 24
 
 
-def algorithmic_bytes(w, merge: str = "avg", out_bf16: bool = False) -> int:
+def rda_launches(w, three_pass: bool = False) -> int:
+    gram = not three_pass and all(participants(w, p) <= RDA_GRAM_MAX_PARTICIPANTS for p in range(w.P))
+    return 2 if gram else 3
+
+
+def algorithmic_bytes(w, merge: str = "avg", out_bf16: bool = False, rda_three_pass: bool = False) -> int:
     b_theta = 2 if w.learner_dtype == "bf16" else 4
-    return int(sum(n * bytes_per_param(merge, participants(w, p), b_theta, out_bf16)
+    three = merge == "rda" and rda_launches(w, rda_three_pass) == 3      # one form for the whole batch
+    return int(sum(n * bytes_per_param(merge, participants(w, p), b_theta, out_bf16, three)
                    for p, n in enumerate(w.fragment_sizes)))
 
 
-def write_share(w, merge: str = "avg", out_bf16: bool = False) -> float:
+def write_share(w, merge: str = "avg", out_bf16: bool = False, rda_three_pass: bool = False) -> float:
     """Fraction of the algorithmic bytes that are writes."""
-    total = algorithmic_bytes(w, merge, out_bf16)
+    total = algorithmic_bytes(w, merge, out_bf16, rda_three_pass)
     b_theta = 2 if w.learner_dtype == "bf16" else 4
-    writes = sum(n * (8 + (2 if out_bf16 else 0) + (4 if merge == "rda" else 0) +
+    stored_direction = merge == "rda" and rda_launches(w, rda_three_pass) == 3
+    writes = sum(n * (8 + (2 if out_bf16 else 0) + (4 if stored_direction else 0) +
                       (participants(w, p) * b_theta if merge == "push" else 0))
                  for p, n in enumerate(w.fragment_sizes))
     return writes / total if total else 0.0
@@ -447,7 +464,7 @@ class Merger:
             assert w.P == 1, "the int4 merge takes a single-fragment workload"
             self.quantise()
         if merge == "rda":
-            self.launches_per_step = 3
+            self.launches_per_step = 3 if range_sharded_rda else rda_launches(w)
             if range_sharded_rda:
                 self.rda_scratch = torch.empty(sum((n + 7) // 8 * 8 for n in w.fragment_sizes),
                                                dtype=torch.float32, device=device)
@@ -658,9 +675,9 @@ class Merger:
         torch.cuda.empty_cache()
 
 
-def roofline_of(w, merge, out_bf16, per_launch_ms, ceilings, traffic_table, workload_name):
+def roofline_of(w, merge, out_bf16, per_launch_ms, ceilings, traffic_table, workload_name, rda_three_pass=False):
     """The roofline object of one timed workload (HBM-bound; no tensor cores on this path)."""
-    alg = algorithmic_bytes(w, merge, out_bf16)
+    alg = algorithmic_bytes(w, merge, out_bf16, rda_three_pass)
     avg = sum(per_launch_ms) / len(per_launch_ms)
     achieved = alg / (avg * 1e-3) / 1e9
     peak, peak_kind = hbm_peak()
@@ -670,7 +687,7 @@ def roofline_of(w, merge, out_bf16, per_launch_ms, ceilings, traffic_table, work
         "peak_source": f"of {peak_kind}",
         "traffic": None if tpp is None else tpp * w.total_params,
         "algorithmic_bytes_per_launch": alg, "bytes_per_param": alg / w.total_params,
-        "write_share": write_share(w, merge, out_bf16),
+        "write_share": write_share(w, merge, out_bf16, rda_three_pass),
         "kernel_ms": {"avg": avg, "median": statistics.median(per_launch_ms), "min": min(per_launch_ms),
                       "max": max(per_launch_ms)},
         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
@@ -707,7 +724,7 @@ def config_row(dd, ctx, device, name, merge, args, ceilings, probes, traffic_tab
         # that the parity windows below are again those of a FIRST merge
         merger.merge = "avg" if merge == "push" else merge
         merger.push_mask = merger.frags[0]["quorum_mask"] if merge == "push" else 0
-        merger.launches_per_step = 3 if merge == "rda" else 1
+        merger.launches_per_step = rda_launches(w) if merge == "rda" else 1
         for p, f in enumerate(merger.frags):
             synth.fill_fragment_gpu(f["global_"], f["momentum"], f["learners"], seed=w.seed * 1000 + p)
         if merge == "int4":
@@ -1016,7 +1033,7 @@ def cpu_baseline_leg(merger, args):
 
 
 def wanted_configs(args, headline, headline_merge):
-    names = ["tiny", "dense150m", "dense1b3", "moe4b", "rda", "int4", "push", "broadcast", "tape24"]
+    names = ["tiny", "dense150m", "dense1b3", "moe4b", "rda", "rda_dense150m", "int4", "push", "broadcast", "tape24"]
     if args.configs == "none":
         return []
     if args.configs != "all":
@@ -1081,6 +1098,10 @@ def run_ours(args):
     ctx = dd.Context(local_rank)
     merger = Merger(dd, ctx, w, device, merge=args.merge, out_bf16=args.out_bf16, resident=args.resident,
                     rank_seed=rank, range_sharded_rda=args.merge == "rda" and args.sharding == "range" and world > 1)
+    three_pass = args.merge == "rda" and (args.rda_three_pass or (args.sharding == "range" and world > 1))
+    if args.rda_three_pass:
+        merger.flags |= dd.RDA_THREE_PASS
+        merger.launches_per_step = 3
     grid, block, tile = ctx.launch_geometry(merger.ldtype)
 
     parity = None
@@ -1090,7 +1111,8 @@ def run_ours(args):
     total_ms, per_launch_ms, clocks = merger.timed(args.steps, args.warmup, world)
     max_ms = ddist.max_over_ranks(total_ms, device=device)
     value = ddist.whole_job_rate(job_params, args.steps, 1, max_ms)
-    roofline = roofline_of(w, args.merge, args.out_bf16, per_launch_ms, ceilings, traffic_table, args.workload)
+    roofline = roofline_of(w, args.merge, args.out_bf16, per_launch_ms, ceilings, traffic_table, args.workload,
+                           three_pass)
     roofline["kernel_ms"]["slowest_steps"] = sorted(range(len(per_launch_ms)), key=lambda k: -per_launch_ms[k])[:3]
     alg_bytes = roofline["algorithmic_bytes_per_launch"]
     fits_l2 = alg_bytes < 4 * L2_BYTES
@@ -1150,6 +1172,10 @@ def run_ours(args):
         merger.free()
         merger = None
         for name in [x for x in todo if x not in ("rda", "int4", "push", "broadcast", "tape24")]:
+            if name == "rda_dense150m":
+                # six participants: the radial-directional merge in its two-launch form
+                rows.append(config_row(dd, ctx, device, "dense150m", "rda", args, ceilings, probes, traffic_table))
+                continue
             rows.append(config_row(dd, ctx, device, name, "avg", args, ceilings, probes, traffic_table,
                                    resident="participants" if name == "moe4b" else "all"))
         if probes is not None:

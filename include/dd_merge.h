@@ -71,6 +71,7 @@ enum {
     DD_HEAVY_BALL = 1u << 0,        /* Theta' = Theta - lr v' instead of the Nesterov form */
     DD_DIAG_PER_LEARNER = 1u << 1,  /* also ||Theta - theta_m||^2 for every participant */
     DD_DIAG_STATE = 1u << 2,        /* also ||Theta'||^2 and ||v'||^2 */
+    DD_RDA_THREE_PASS = 1u << 3,    /* radial-directional merges: always the three-launch form (see dd_merge_fragment_rda) */
     /* Test hook for the error path.  Production callers must never set it: every warp's
      * first bulk copy is made to wait for bytes that never come, so its bounded wait
      * expires (about a second, up to three for the launch), every fragment the launch
@@ -213,11 +214,21 @@ int dd_merge_fragments_batched_push(dd_ctx *ctx, const dd_fragment_desc *descs,
  * A participant with D_m = 0 adds its (zero) norm to the radial mean and nothing
  * to the direction; if the mean direction vanishes, Delta = 0.
  *
- * Three launches on cuda_stream: norms, mean direction (kept in `scratch`), outer
- * step.  Learner copies are read twice; bytes per parameter = 2 (s b_theta + 4) + 24.
+ * Learner copies are read twice, in one of two forms:
+ *   - at most 8 participants: two launches on cuda_stream.  The first accumulates the
+ *     Gram matrix G_jk = <D_j, D_k> of the outer gradients (||D_j||^2 = G_jj, and the
+ *     mean direction's squared length is a^T G a with a_j = w^_j / ||D_j||); the second
+ *     is the ordinary fused merge with the weights c a_j, c = (sum_j w^_j ||D_j||) /
+ *     sqrt(a^T G a).  Nothing is stored in between but the matrix; bytes per parameter
+ *     = 2 s b_theta + 20.  `scratch` is not used.
+ *   - more participants, or DD_RDA_THREE_PASS: three launches -- norms, mean direction
+ *     (kept in `scratch`), outer step; bytes per parameter = 2 (s b_theta + 4) + 24.
+ * In a batch every fragment takes the same form: two launches only if no
+ * radial-directional fragment has more than 8 participants.
  *
  *   scratch   [device] n floats (16-byte aligned), or NULL: the context allocates
- *             and keeps one (growing it synchronises the device)
+ *             and keeps one when the three-launch form needs it (growing it
+ *             synchronises the device)
  *   record    as for dd_merge_fragment; delta_m_sq is always filled, delta_sq is
  *             ||Delta||^2 of the RDA result.  DD_DIAG_PER_LEARNER is implied.
  * Everything else is as in dd_merge_fragment.

@@ -37,6 +37,9 @@ struct dd_ctx {
     size_t rda_scratch_cap = 0;               // floats
     dd_merge_record *rda_records = nullptr;   // hand-over records when the caller passes none
     size_t rda_records_cap = 0;
+    double *gram = nullptr;                   // Gram matrices of two-launch radial-directional merges
+    size_t gram_cap = 0;                      // fragments
+    int gram_grid[2] = {0, 0};                // [bf16] persistent grid of the Gram launch
     ddm::HostPipe *pipe = nullptr;
     char cuda_err[256] = {0};
 };

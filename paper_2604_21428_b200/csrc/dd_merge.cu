@@ -8,6 +8,7 @@
 #include <cuda_runtime.h>
 
 #include "dd_merge_tma.cuh"
+#include "dd_rda_gram.cuh"
 
 namespace ddm {
 
@@ -36,6 +37,15 @@ __global__ void __launch_bounds__(kThreads, 2)
 rda_pass_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ Common c)
 {
     merge_body_tma<BF16, MODE, MODE == kModeNorms>(frags, c);
+}
+
+// Second launch of the two-launch radial-directional merge: the ordinary merge with the
+// weights the header derives from the Gram matrix (direct averaging for DD_MERGE_AVG fragments).
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads, 2)
+rda_gram_merge_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ Common c)
+{
+    merge_body_tma<BF16, kModeMergeGram, false>(frags, c);
 }
 
 }  // namespace ddm
@@ -80,7 +90,21 @@ static cudaError_t occupancy(int *blocks)
         if (e == cudaSuccess) e = prepare_kernel(rda_pass_kernel<BF16, kModeNorms>, blocks);
         if (e == cudaSuccess) e = prepare_kernel(rda_pass_kernel<BF16, kModeDir>, blocks);
         if (e == cudaSuccess) e = prepare_kernel(rda_pass_kernel<BF16, kModeApply>, blocks);
+        if (e == cudaSuccess) e = prepare_kernel(rda_gram_merge_kernel<BF16>, blocks);
     }
+    return e;
+}
+
+// The Gram launch has its own shape (nine warps, CTA-wide stages): resident CTAs per SM, at most 2.
+template <bool BF16>
+static cudaError_t gram_occupancy(int *blocks)
+{
+    cudaError_t e = cudaFuncSetAttribute(rda_gram_kernel<BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)kGramRingBytes);
+    int b = 0;
+    if (e == cudaSuccess)
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, rda_gram_kernel<BF16>, kGramThreads, kGramRingBytes);
+    *blocks = b > 2 ? 2 : b;
     return e;
 }
 
@@ -178,7 +202,8 @@ int check_common(const dd_ctx *ctx, int M, dd_dtype dtype, float lr, float mu, u
     if (M < 1) return DD_ERR_INVALID_ARG;
     if (dtype != DD_F32 && dtype != DD_BF16) return DD_ERR_INVALID_ARG;
     if (!std::isfinite(lr) || !std::isfinite(mu)) return DD_ERR_INVALID_ARG;
-    if (flags & ~(uint32_t)(DD_HEAVY_BALL | DD_DIAG_PER_LEARNER | DD_DIAG_STATE | DD_DEBUG_EXPIRE_WAIT))
+    if (flags & ~(uint32_t)(DD_HEAVY_BALL | DD_DIAG_PER_LEARNER | DD_DIAG_STATE | DD_RDA_THREE_PASS |
+                            DD_DEBUG_EXPIRE_WAIT))
         return DD_ERR_INVALID_ARG;
     return DD_OK;
 }
@@ -284,6 +309,13 @@ extern "C" int dd_create(dd_ctx **out, int device)
     }
     for (int a = 0; a < 2; ++a)
         for (int b = 0; b < 2; ++b) ctx->grid[a][b] = ctx->sm_count * (occ[a][b] > 0 ? occ[a][b] : 1);
+    int gocc[2] = {0, 0};
+    if (gram_occupancy<false>(&gocc[0]) != cudaSuccess || gram_occupancy<true>(&gocc[1]) != cudaSuccess) {
+        (void)cudaGetLastError();
+        delete ctx;
+        return DD_ERR_CUDA;
+    }
+    for (int a = 0; a < 2; ++a) ctx->gram_grid[a] = ctx->sm_count * (gocc[a] > 0 ? gocc[a] : 1);
     *out = ctx;
     return rc;
 }
@@ -297,6 +329,7 @@ extern "C" int dd_destroy(dd_ctx *ctx)
     if (ctx->tickets) cudaFree(ctx->tickets);
     if (ctx->rda_scratch) cudaFree(ctx->rda_scratch);
     if (ctx->rda_records) cudaFree(ctx->rda_records);
+    if (ctx->gram) cudaFree(ctx->gram);
     host_pipe_destroy(ctx);
     for (Slot &s : ctx->slots) {
         if (s.host) cudaFreeHost(s.host);
@@ -507,21 +540,8 @@ static int rda_batched_impl(dd_ctx *ctx, const dd_fragment_desc *descs, const ui
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice, "cudaSetDevice");
 
-    // Scratch for the mean direction: n floats per radial-directional fragment.
-    size_t need = 0;
     for (int p = 0; p < P; ++p)
-        if (!merge_kinds || merge_kinds[p] == DD_MERGE_RDA) need += round_up8((size_t)descs[p].n);
-        else if (merge_kinds[p] != DD_MERGE_AVG) return DD_ERR_INVALID_ARG;
-    if (scratch) {
-        if (scratch_elems < need) return DD_ERR_INVALID_ARG;
-    } else if (need > ctx->rda_scratch_cap) {
-        DD_CUDA(ctx, cudaDeviceSynchronize());
-        if (ctx->rda_scratch) cudaFree(ctx->rda_scratch);
-        ctx->rda_scratch = nullptr;
-        ctx->rda_scratch_cap = 0;
-        DD_CUDA(ctx, cudaMalloc(&ctx->rda_scratch, need * sizeof(float)));
-        ctx->rda_scratch_cap = need;
-    }
+        if (merge_kinds && merge_kinds[p] != DD_MERGE_RDA && merge_kinds[p] != DD_MERGE_AVG) return DD_ERR_INVALID_ARG;
     // The passes hand norms to one another through the records: use the context's
     // own when the caller wants none.
     if (!records) {
@@ -539,20 +559,52 @@ static int rda_batched_impl(dd_ctx *ctx, const dd_fragment_desc *descs, const ui
     rc = acquire_slot(ctx, P);
     if (rc != DD_OK) return rc;
     Slot &slot = ctx->slots[ctx->next_slot];
-    float *next_scratch = scratch ? scratch : ctx->rda_scratch;
     unsigned long long tile = 0;
+    // With few participants everywhere the merge takes two launches (Gram matrix, then the ordinary
+    // merge with weights derived from it) and needs no scratch for the mean direction.
+    bool use_gram = only_pass < 0 && !(flags & DD_RDA_THREE_PASS);
+    bool any_rda = false;
     for (int p = 0; p < P; ++p) {
         const dd_fragment_desc &d = descs[p];
         DevFrag &f = slot.host[p];
         rc = fill_fragment(f, d.global, d.momentum, d.out_bf16, d.learner_ptrs, d.tokens, d.steps,
                            d.quorum_mask, d.K, d.n, M, learner_bytes_of(learner_dtype, d.n));
         if (rc != DD_OK) return rc;
-        if (push_masks && push_masks[p]) {      // written by the apply pass, after the passes that read
+        if (push_masks && push_masks[p]) {      // written by the last launch, after every launch that reads
             rc = set_push(f, d.learner_ptrs, push_masks[p], M, d.n, learner_bytes_of(learner_dtype, d.n));
             if (rc != DD_OK) return rc;
         }
         f.kind = (!merge_kinds || merge_kinds[p] == DD_MERGE_RDA) ? DD_MERGE_RDA : DD_MERGE_AVG;
         if (f.kind == DD_MERGE_RDA) {
+            any_rda = true;
+            if (f.n_part_host > kGramMaxPart) use_gram = false;
+        }
+        f.tile_begin = tile;
+        tile += tiles_of(d.n);
+        f.tile_end = tile;
+    }
+    use_gram = use_gram && any_rda;
+
+    if (!use_gram) {
+        // Scratch for the mean direction: n floats per radial-directional fragment.
+        size_t need = 0;
+        for (int p = 0; p < P; ++p)
+            if (slot.host[p].kind == DD_MERGE_RDA) need += round_up8((size_t)descs[p].n);
+        if (scratch) {
+            if (scratch_elems < need) return DD_ERR_INVALID_ARG;
+        } else if (need > ctx->rda_scratch_cap) {
+            DD_CUDA(ctx, cudaDeviceSynchronize());
+            if (ctx->rda_scratch) cudaFree(ctx->rda_scratch);
+            ctx->rda_scratch = nullptr;
+            ctx->rda_scratch_cap = 0;
+            DD_CUDA(ctx, cudaMalloc(&ctx->rda_scratch, need * sizeof(float)));
+            ctx->rda_scratch_cap = need;
+        }
+        float *next_scratch = scratch ? scratch : ctx->rda_scratch;
+        for (int p = 0; p < P; ++p) {
+            const dd_fragment_desc &d = descs[p];
+            DevFrag &f = slot.host[p];
+            if (f.kind != DD_MERGE_RDA) continue;
             f.scratch = next_scratch;
             next_scratch += round_up8((size_t)d.n);
             const size_t n = (size_t)d.n;
@@ -560,34 +612,56 @@ static int rda_batched_impl(dd_ctx *ctx, const dd_fragment_desc *descs, const ui
                 overlaps(f.scratch, 4 * n, d.out_bf16, 2 * n))
                 return DD_ERR_ALIAS;
         }
-        f.tile_begin = tile;
-        tile += tiles_of(d.n);
-        f.tile_end = tile;
+    } else if ((size_t)P > ctx->gram_cap) {
+        DD_CUDA(ctx, cudaDeviceSynchronize());
+        if (ctx->gram) cudaFree(ctx->gram);
+        ctx->gram = nullptr;
+        ctx->gram_cap = 0;
+        const size_t cap = P < 64 ? 64 : (size_t)P;
+        DD_CUDA(ctx, cudaMalloc(&ctx->gram, cap * kGramPairs * sizeof(double)));
+        ctx->gram_cap = cap;
     }
 
     const bool bf16 = learner_dtype == DD_BF16;
     unsigned long long g = (unsigned long long)ctx->grid[bf16][1];
     if (g > tile) g = tile;
+    unsigned long long gg = (unsigned long long)ctx->gram_grid[bf16];
+    if (gg > tile) gg = tile;
     Common c;
     c.eta = outer_lr;
     c.mu = outer_mu;
-    c.flags = flags;
+    c.flags = flags & ~(uint32_t)DD_RDA_THREE_PASS;
     c.M = M;
     c.P = P;
     c.total_tiles = tile;
     c.records = records;
     c.nq = kNumScalarDiag + M;
-    c.pl_cap = pl_capacity(slot.host, P, true);
-    rc = ensure_workspace(ctx, (size_t)P, (size_t)c.nq, (size_t)ctx->grid[bf16][1]);
+    if (use_gram && c.nq < kGramPairs) c.nq = kGramPairs;
+    c.pl_cap = use_gram ? 0 : pl_capacity(slot.host, P, true);
+    const size_t widest = ctx->grid[bf16][1] > ctx->gram_grid[bf16] ? ctx->grid[bf16][1] : ctx->gram_grid[bf16];
+    rc = ensure_workspace(ctx, (size_t)P, (size_t)c.nq, widest);
     if (rc != DD_OK) return rc;
     c.partials = ctx->partials;
     c.tickets = ctx->tickets;
+    c.gram = ctx->gram;
 
     DD_CUDA(ctx, cudaMemcpyAsync(slot.dev, slot.host, (size_t)P * sizeof(DevFrag),
                                  cudaMemcpyHostToDevice, stream));
-    cudaError_t e = bf16 ? launch_rda_passes<true>(slot.dev, c, (unsigned)g, stream, only_pass)
-                         : launch_rda_passes<false>(slot.dev, c, (unsigned)g, stream, only_pass);
-    if (e != cudaSuccess) return cuda_fail(ctx, e, "rda_pass_kernel launch");
+    cudaError_t e;
+    if (use_gram) {
+        if (bf16) {
+            rda_gram_kernel<true><<<(unsigned)gg, kGramThreads, kGramRingBytes, stream>>>(slot.dev, c);
+            rda_gram_merge_kernel<true><<<(unsigned)g, kThreads, kTmaRingBytes, stream>>>(slot.dev, c);
+        } else {
+            rda_gram_kernel<false><<<(unsigned)gg, kGramThreads, kGramRingBytes, stream>>>(slot.dev, c);
+            rda_gram_merge_kernel<false><<<(unsigned)g, kThreads, kTmaRingBytes, stream>>>(slot.dev, c);
+        }
+        e = cudaGetLastError();
+    } else {
+        e = bf16 ? launch_rda_passes<true>(slot.dev, c, (unsigned)g, stream, only_pass)
+                 : launch_rda_passes<false>(slot.dev, c, (unsigned)g, stream, only_pass);
+    }
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "radial-directional merge launch");
     DD_CUDA(ctx, cudaEventRecord(slot.done, stream));
     slot.used = true;
     ctx->next_slot = (ctx->next_slot + 1) % kSlots;

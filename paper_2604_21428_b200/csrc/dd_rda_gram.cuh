@@ -14,24 +14,23 @@
 // same time, so the staging is CTA-wide here: a stage holds one sub-tile (1024 elements of
 // bf16 copies, 512 of fp32 ones) of Theta and of every participant, filled by a producer
 // warp with bulk asynchronous copies (one 2 KB piece per participant) and consumed by the
-// eight other warps, a thread owning four (two) consecutive elements.  Full / empty
-// mbarriers per stage; every wait has an iteration limit.
+// eight other warps.  The ring is cut into as many stages as fit (three at 8 participants,
+// eight at 2).  Full / empty mbarriers per stage; every wait has an iteration limit.
 #pragma once
 
 #include "dd_merge_tma.cuh"
 
-#ifndef DD_GRAM_STAGES
-#define DD_GRAM_STAGES 3
+#ifndef DD_GRAM_RING_KB
+#define DD_GRAM_RING_KB 64
 #endif
 
 namespace ddm {
 
 constexpr int kGramMaxPart = DD_RDA_GRAM_MAX_PARTICIPANTS;
 constexpr int kGramPairs = kGramMaxPart * (kGramMaxPart + 1) / 2;
-constexpr int kGramStages = DD_GRAM_STAGES;
+constexpr int kGramMaxStages = 8;                                 // stages the ring is cut into at most
 constexpr int kGramThreads = kThreads + 32;                       // eight consumer warps and the producer warp
-constexpr int kGramStageBytes = 4096 + kGramMaxPart * kTmaChunk;  // Theta sub-tile + one piece per participant
-constexpr size_t kGramRingBytes = (size_t)kGramStages * kGramStageBytes;
+constexpr size_t kGramRingBytes = (size_t)DD_GRAM_RING_KB * 1024; // stages of Theta sub-tile + one piece per participant
 constexpr int kGramFlushTiles = 128;                              // tiles a thread sums in fp32 before the fp64 hand-over
 
 __device__ __forceinline__ void mbar_arrive(unsigned bar)
@@ -94,23 +93,122 @@ __device__ __forceinline__ void flush_gram(Smem &sm, GramShared &gs, const Commo
     }
 }
 
+// One consumer warp's share of a fragment: every stage of this CTA's tiles.  A thread owns four
+// (bf16) or two (fp32) consecutive elements of every sub-tile and accumulates every pair's product.
+template <bool BF16>
+__device__ __forceinline__ void gram_consume(Smem &sm, GramShared &gs, unsigned long long tile,
+                                             unsigned long long mine, const unsigned char *stage_base,
+                                             unsigned full_s, unsigned empty_s, int nst, unsigned stage_bytes,
+                                             unsigned &phase_bits, bool &failed)
+{
+    constexpr int E = BF16 ? 1024 : 512;               // elements per sub-tile: 2 KB of every copy
+    constexpr int EPT = E / kThreads;                  // elements per consumer thread: 4 or 2
+    const unsigned G = gridDim.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int s = sm.n_part;
+    const unsigned long long nelems = (sm.n / kVec) * kVec;
+    const unsigned long long tile_end = sm.tile_end;
+    const unsigned my = (unsigned)threadIdx.x * EPT;   // first element of this thread within a sub-tile
+    float acc[kGramPairs];
+#pragma unroll
+    for (int q = 0; q < kGramPairs; ++q) acc[q] = 0.0f;
+    auto hand_over = [&]() {                           // per-thread fp32 sums -> per-warp fp64 sums
+#pragma unroll
+        for (int j = 0; j < kGramMaxPart; ++j)
+#pragma unroll
+            for (int k = 0; k <= j; ++k) {
+                const int q = gram_index(j, k);
+                if (j < s) {
+                    const float t = warp_sum(acc[q]);
+                    if (lane == 0) gs.acc[warp][q] += (double)t;
+                }
+                acc[q] = 0.0f;
+            }
+    };
+    int slot = 0, tiles_summed = 0;
+    for (unsigned long long t = tile; t < tile_end && !failed; t += G) {
+        // elements of this tile that go through the stages (the fragment's last tile may be short)
+        const unsigned long long e0 = (t - sm.tile_begin) * (unsigned long long)kTileElems;
+        const unsigned in_tile = (unsigned)(nelems - e0 < (unsigned long long)kTileElems ? nelems - e0 : kTileElems);
+        for (unsigned first = 0; first < in_tile; first += E) {
+            const unsigned cnt = in_tile - first < (unsigned)E ? in_tile - first : (unsigned)E;
+            const bool ok = mbar_wait_bounded(full_s + 8u * slot, (phase_bits >> slot) & 1u);
+            if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+            const unsigned char *st = stage_base + (size_t)slot * stage_bytes;
+            if (my < cnt) {
+                float T[EPT], D[kGramMaxPart][EPT];
+                if (BF16) {
+                    const float4 t4 = *reinterpret_cast<const float4 *>(st + threadIdx.x * 16);
+                    T[0] = t4.x; T[1] = t4.y; T[2] = t4.z; T[3] = t4.w;
+                } else {
+                    const float2 t2 = *reinterpret_cast<const float2 *>(st + threadIdx.x * 8);
+                    T[0] = t2.x; T[1] = t2.y;
+                }
+#pragma unroll
+                for (int j = 0; j < kGramMaxPart; ++j) {
+                    if (j < s) {
+                        const uint2 x = *reinterpret_cast<const uint2 *>(st + E * 4 + j * kTmaChunk + threadIdx.x * 8);
+                        if (BF16) {
+                            D[j][0] = __uint_as_float(x.x << 16) - T[0];
+                            D[j][1] = __uint_as_float(x.x & 0xffff0000u) - T[1];
+                            D[j][2] = __uint_as_float(x.y << 16) - T[2];
+                            D[j][3] = __uint_as_float(x.y & 0xffff0000u) - T[3];
+                        } else {
+                            D[j][0] = __uint_as_float(x.x) - T[0];
+                            D[j][1] = __uint_as_float(x.y) - T[1];
+                        }
+#pragma unroll
+                        for (int k = 0; k <= j; ++k) {
+                            float a = acc[gram_index(j, k)];
+#pragma unroll
+                            for (int e = 0; e < EPT; ++e) a = fmaf(D[j][e], D[k][e], a);
+                            acc[gram_index(j, k)] = a;
+                        }
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty_s + 8u * slot);
+            phase_bits ^= 1u << slot;
+            if (++slot == nst) slot = 0;
+        }
+        if (++tiles_summed == kGramFlushTiles) { hand_over(); tiles_summed = 0; }
+    }
+    // the ragged end of the fragment (n mod 8 elements): one element per lane of warp 0 of the CTA
+    // that owns the last tile
+    const int rem = (int)(sm.n % kVec);
+    if (rem != 0 && warp == 0 && tile + (mine - 1) * G == tile_end - 1 && lane < rem && !failed) {
+        const unsigned long long e = nelems + lane;
+        const float T = sm.theta[e];
+        float D[kGramMaxPart];
+#pragma unroll
+        for (int j = 0; j < kGramMaxPart; ++j) {
+            if (j < s) {
+                D[j] = (BF16 ? __uint_as_float((unsigned)reinterpret_cast<const uint16_t *>(sm.ptr[j])[e] << 16)
+                             : reinterpret_cast<const float *>(sm.ptr[j])[e]) - T;
+#pragma unroll
+                for (int k = 0; k <= j; ++k) acc[gram_index(j, k)] = fmaf(D[j], D[k], acc[gram_index(j, k)]);
+            }
+        }
+    }
+    hand_over();
+}
+
 template <bool BF16>
 __global__ void __launch_bounds__(kGramThreads, 2)
 rda_gram_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ Common c)
 {
     constexpr int E = BF16 ? 1024 : 512;               // elements per sub-tile: 2 KB of every copy
-    constexpr int EPT = E / kThreads;                  // elements per consumer thread: 4 or 2
-    constexpr int kSubs = kTileElems / E;              // sub-tiles per tile
     constexpr int kEsz = BF16 ? 2 : 4;
     __shared__ Smem sm;
     __shared__ GramShared gs;
-    __shared__ unsigned long long full_bar[kGramStages], empty_bar[kGramStages];
+    __shared__ unsigned long long full_bar[kGramMaxStages], empty_bar[kGramMaxStages];
     extern __shared__ __align__(128) unsigned char stage_base[];
     const unsigned G = gridDim.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const bool producer = warp == kWarps;
     if (threadIdx.x == 0) {
-        for (int d = 0; d < kGramStages; ++d) {
+        for (int d = 0; d < kGramMaxStages; ++d) {
             mbar_init(full_bar + d, 1);                // the producer's arrival (plus the bytes it announces)
             mbar_init(empty_bar + d, kWarps);          // one arrival per consumer warp
         }
@@ -120,9 +218,10 @@ rda_gram_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ Commo
     __syncthreads();
     const unsigned full_s = smem_addr(full_bar), empty_s = smem_addr(empty_bar), stage_s = smem_addr(stage_base);
 
-    // position in the ring: producer and consumers walk the same sequence of stages
-    int slot = 0;
-    unsigned phase = 0;                                // parity of the slot's current use
+    // Every stage barrier completes one phase per use, whatever the number of stages a fragment
+    // cuts the ring into: bit d is the parity of barrier d's next use (producer and consumers count
+    // alike, each for itself).
+    unsigned phase_bits = 0;
     bool failed = false;                               // this warp gave up a bounded wait
     int cur = -1;
     unsigned long long tile = blockIdx.x;
@@ -140,118 +239,43 @@ rda_gram_kernel(const DevFrag *__restrict__ frags, const __grid_constant__ Commo
         const int s = sm.n_part;
         const bool worked_on = sm.status == DD_STATUS_OK && sm.kind == DD_MERGE_RDA && s <= kGramMaxPart;
         if (worked_on) {
+            // a stage: the Theta sub-tile, then one 2 KB piece per participant; as many stages as fit
+            const unsigned stage_bytes = (unsigned)(E * 4 + s * kTmaChunk);
+            int nst = (int)(kGramRingBytes / stage_bytes);
+            nst = nst > kGramMaxStages ? kGramMaxStages : nst;
             const unsigned long long nelems = (sm.n / kVec) * kVec;       // whole 8-element steps go through the stages
             const bool dead = gs.dead != 0;
             if (dead && threadIdx.x == 0) sm.any_failed = 1;               // an earlier failure leaves this fragment undone
             if (producer) {
                 if (lane == 0 && !dead) {
                     const bool expire_hook = (c.flags & DD_DEBUG_EXPIRE_WAIT) != 0;
+                    int slot = 0;
                     for (unsigned long long t = tile; t < tile_end && !failed; t += G) {
                         const unsigned long long e0 = (t - sm.tile_begin) * (unsigned long long)kTileElems;
-                        for (int sub = 0; sub < kSubs && !failed; ++sub) {
-                            const unsigned long long first = e0 + (unsigned long long)sub * E;
-                            if (first >= nelems) break;
-                            const unsigned cnt = (unsigned)(nelems - first < (unsigned long long)E ? nelems - first : E);
+                        const unsigned in_tile = (unsigned)(nelems - e0 < (unsigned long long)kTileElems ? nelems - e0 : kTileElems);
+                        const char *theta_t = reinterpret_cast<const char *>(sm.theta + e0);
+                        for (unsigned first = 0; first < in_tile && !failed; first += E) {
+                            const unsigned cnt = in_tile - first < (unsigned)E ? in_tile - first : (unsigned)E;
                             // the slot is free once every consumer warp has left its previous use
-                            if (!mbar_wait_bounded(empty_s + 8u * slot, phase ^ 1u)) { failed = true; break; }
+                            if (!mbar_wait_bounded(empty_s + 8u * slot, ((phase_bits >> slot) & 1u) ^ 1u)) { failed = true; break; }
                             const unsigned fb = full_s + 8u * slot;
-                            const unsigned dst = stage_s + (unsigned)slot * kGramStageBytes;
+                            const unsigned dst = stage_s + (unsigned)slot * stage_bytes;
                             // (test hook) announce 16 bytes that no copy delivers: the consumers' wait must expire
-                            const unsigned phantom = expire_hook && t == tile && sub == 0 ? 16u : 0u;
+                            const unsigned phantom = expire_hook && t == tile && first == 0 ? 16u : 0u;
                             mbar_arrive_expect_tx(fb, cnt * 4u + (unsigned)s * cnt * kEsz + phantom);
-                            bulk_copy_g2s(dst, sm.theta + first, cnt * 4u, fb);
+                            bulk_copy_g2s(dst, theta_t + first * 4u, cnt * 4u, fb);
                             for (int j = 0; j < s; ++j)
-                                bulk_copy_g2s(dst + 4096u + (unsigned)j * kTmaChunk,
-                                              reinterpret_cast<const char *>(sm.ptr[j]) + first * kEsz, cnt * kEsz, fb);
-                            if (++slot == kGramStages) { slot = 0; phase ^= 1u; }
+                                bulk_copy_g2s(dst + E * 4u + (unsigned)j * kTmaChunk,
+                                              reinterpret_cast<const char *>(sm.ptr[j]) + (e0 + first) * kEsz, cnt * kEsz, fb);
+                            phase_bits ^= 1u << slot;
+                            if (++slot == nst) slot = 0;
                         }
                     }
                     if (failed) { gs.dead = 1; sm.any_failed = 1; }
                 }
+                __syncwarp();                            // the producer warp reconverges before the CTA-wide barriers
             } else if (!dead) {
-                float acc[kGramPairs];
-#pragma unroll
-                for (int q = 0; q < kGramPairs; ++q) acc[q] = 0.0f;
-                auto hand_over = [&]() {              // per-thread fp32 sums -> per-warp fp64 sums
-#pragma unroll
-                    for (int j = 0; j < kGramMaxPart; ++j)
-#pragma unroll
-                        for (int k = 0; k <= j; ++k) {
-                            const int q = gram_index(j, k);
-                            if (j < s) {
-                                const float t = warp_sum(acc[q]);
-                                if (lane == 0) gs.acc[warp][q] += (double)t;
-                            }
-                            acc[q] = 0.0f;
-                        }
-                };
-                int tiles_summed = 0;
-                for (unsigned long long t = tile; t < tile_end && !failed; t += G) {
-                    const unsigned long long e0 = (t - sm.tile_begin) * (unsigned long long)kTileElems;
-                    for (int sub = 0; sub < kSubs; ++sub) {
-                        const unsigned long long first = e0 + (unsigned long long)sub * E;
-                        if (first >= nelems) break;
-                        const unsigned cnt = (unsigned)(nelems - first < (unsigned long long)E ? nelems - first : E);
-                        const bool ok = mbar_wait_bounded(full_s + 8u * slot, phase);
-                        if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
-                        const unsigned char *st = stage_base + (size_t)slot * kGramStageBytes;
-                        const unsigned my = (unsigned)threadIdx.x * EPT;
-                        if (my < cnt) {
-                            float T[EPT], D[kGramMaxPart][EPT];
-                            if (BF16) {
-                                const float4 t4 = *reinterpret_cast<const float4 *>(st + threadIdx.x * 16);
-                                T[0] = t4.x; T[1] = t4.y; T[2] = t4.z; T[3] = t4.w;
-                            } else {
-                                const float2 t2 = *reinterpret_cast<const float2 *>(st + threadIdx.x * 8);
-                                T[0] = t2.x; T[1] = t2.y;
-                            }
-#pragma unroll
-                            for (int j = 0; j < kGramMaxPart; ++j) {
-                                if (j < s) {
-                                    const uint2 x = *reinterpret_cast<const uint2 *>(st + 4096 + j * kTmaChunk + threadIdx.x * 8);
-                                    if (BF16) {
-                                        D[j][0] = __uint_as_float(x.x << 16) - T[0];
-                                        D[j][1] = __uint_as_float(x.x & 0xffff0000u) - T[1];
-                                        D[j][2] = __uint_as_float(x.y << 16) - T[2];
-                                        D[j][3] = __uint_as_float(x.y & 0xffff0000u) - T[3];
-                                    } else {
-                                        D[j][0] = __uint_as_float(x.x) - T[0];
-                                        D[j][1] = __uint_as_float(x.y) - T[1];
-                                    }
-#pragma unroll
-                                    for (int k = 0; k <= j; ++k) {
-                                        float a = acc[gram_index(j, k)];
-#pragma unroll
-                                        for (int e = 0; e < EPT; ++e) a = fmaf(D[j][e], D[k][e], a);
-                                        acc[gram_index(j, k)] = a;
-                                    }
-                                }
-                            }
-                        }
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(empty_s + 8u * slot);
-                        if (++slot == kGramStages) { slot = 0; phase ^= 1u; }
-                    }
-                    if (++tiles_summed == kGramFlushTiles) { hand_over(); tiles_summed = 0; }
-                }
-                // the ragged end of the fragment (n mod 8 elements): one element per lane of warp 0 of
-                // the CTA that owns the last tile
-                const int rem = (int)(sm.n % kVec);
-                if (rem != 0 && warp == 0 && tile + (mine - 1) * G == tile_end - 1 && lane < rem && !failed) {
-                    const unsigned long long e = nelems + lane;
-                    const float T = sm.theta[e];
-                    float D[kGramMaxPart];
-#pragma unroll
-                    for (int j = 0; j < kGramMaxPart; ++j) {
-                        if (j < s) {
-                            D[j] = (BF16 ? __uint_as_float((unsigned)reinterpret_cast<const uint16_t *>(sm.ptr[j])[e] << 16)
-                                         : reinterpret_cast<const float *>(sm.ptr[j])[e]) - T;
-#pragma unroll
-                            for (int k = 0; k <= j; ++k) acc[gram_index(j, k)] = fmaf(D[j], D[k], acc[gram_index(j, k)]);
-                        }
-                    }
-                }
-                hand_over();
+                gram_consume<BF16>(sm, gs, tile, mine, stage_base, full_s, empty_s, nst, stage_bytes, phase_bits, failed);
                 if (failed && lane == 0) { gs.dead = 1; sm.any_failed = 1; }
             }
             if (c.records != nullptr) flush_gram(sm, gs, c);

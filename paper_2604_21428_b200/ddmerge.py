@@ -17,7 +17,7 @@ OK = 0
 ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_ALIAS, ERR_TOO_MANY_LEARNERS, ERR_CUDA, ERR_TOO_LARGE = \
     -1, -2, -3, -4, -5, -6
 STATUS_OK, STATUS_QUORUM_NOT_MET, STATUS_ZERO_WEIGHT, STATUS_WAIT_LIMIT = 0, 1, 2, 3
-HEAVY_BALL, DIAG_PER_LEARNER, DIAG_STATE = 1, 2, 4
+HEAVY_BALL, DIAG_PER_LEARNER, DIAG_STATE, RDA_THREE_PASS = 1, 2, 4, 8
 DEBUG_EXPIRE_WAIT = 1 << 30
 MERGE_AVG, MERGE_RDA = 0, 1
 RDA_PASS_NORMS, RDA_PASS_DIRECTION, RDA_PASS_APPLY = 0, 1, 2

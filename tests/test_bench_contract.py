@@ -76,6 +76,11 @@ def test_byte_accounting_follows_the_stated_formulas():
     assert bench.algorithmic_bytes(w, out_bf16=True) == 500_000_000 * (24 * 2 + 18)
     assert bench.algorithmic_bytes(w, "int4") == int(500_000_000 * (24 * (0.5 + 4 / 128) + 16))
     assert abs(bench.write_share(w) - 8 / 64) < 1e-12
+    # radial-directional: three launches above 8 participants, two (through the Gram matrix) up to 8
+    assert bench.algorithmic_bytes(w, "rda") == 500_000_000 * (2 * (24 * 2 + 4) + 24) and bench.rda_launches(w) == 3
+    d6 = synth.workload("dense150m")
+    assert bench.algorithmic_bytes(d6, "rda") == d6.total_params * (2 * 6 * 2 + 20) and bench.rda_launches(d6) == 2
+    assert bench.algorithmic_bytes(d6, "rda", rda_three_pass=True) == d6.total_params * (2 * (6 * 2 + 4) + 24)
     t = synth.workload("tiny")
     assert bench.algorithmic_bytes(t) == (1 << 20) * (2 * 4 + 16)
     d = synth.workload("dense150m")

@@ -38,7 +38,7 @@ def _check_record(got, ref):
 
 
 def _case(dd, ctx, n, M, dtype, tokens, mask, K, *, seed, steps=None, merges=2, own_scratch=False,
-          heavy=False, zero_learner=None):
+          heavy=False, zero_learner=None, three_pass=False):
     theta, v, learners = synth.fragment_cpu(n, M, dtype, seed)
     if zero_learner is not None:                    # this participant's outer gradient is exactly 0
         if dtype == "bf16":
@@ -51,7 +51,7 @@ def _case(dd, ctx, n, M, dtype, tokens, mask, K, *, seed, steps=None, merges=2, 
     out_dev = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
     rec_buf = dd.new_records(1)
     scratch = torch.empty((n + 7) // 8 * 8, dtype=torch.float32, device="cuda") if own_scratch else None
-    flags = dd.DIAG_STATE | (dd.HEAVY_BALL if heavy else 0)
+    flags = dd.DIAG_STATE | (dd.HEAVY_BALL if heavy else 0) | (dd.RDA_THREE_PASS if three_pass else 0)
     for k in range(merges):
         o_out = np.zeros(n, dtype=np.uint16)
         ref = oracle.merge_fragment(theta, v, learners, tokens, mask, K, ETA, MU, steps=steps,
@@ -201,3 +201,82 @@ def test_range_sharded_rda_equals_unsharded(dd, ctx, shards):
     assert floor_rel_err(v_dev.cpu().numpy(), o_v) <= TOL_STATE
     for rec in recs:
         _check_record(dd.read_records(rec)[0], ref)
+
+
+# With at most eight participants the merge takes two launches (Gram matrix of the outer gradients,
+# then the ordinary merge with weights derived from it); the cases above with up to eight
+# participants ran that form.  The same cases in the three-launch form, which larger participant
+# counts and range-sharded fragments use:
+@pytest.mark.parametrize("n", [5, 1023, 8192 * 2 + 3, 200_001])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_rda_three_launch_form(dd, ctx, n, dtype):
+    _case(dd, ctx, n, 5, dtype, [100, 200, 0, 400, 500], 0b11101, 2, seed=n % 89, three_pass=True)
+
+
+def test_rda_three_launch_form_special_cases(dd, ctx):
+    _case(dd, ctx, 30_000, 4, "f32", [4000, 9000, 100, 2500], 0b1111, 4, seed=5, steps=[4, 3, 1, 5],
+          heavy=True, three_pass=True)
+    _case(dd, ctx, 30_000, 4, "bf16", [5, 5, 5, 5], 0b1111, 1, seed=6, zero_learner=0, merges=1,
+          three_pass=True)
+    _case(dd, ctx, 2 * 296 * 8192 + 8192 + 3, 3, "bf16", [700, 0, 900], 0b111, 2, seed=31, merges=1,
+          three_pass=True)
+
+
+def test_rda_two_launch_form_exactly_eight_and_nine_participants(dd, ctx):
+    # eight participants: the largest Gram matrix (36 products); nine: the three-launch form takes over
+    tokens = [10 * (m + 1) for m in range(12)]
+    rec = _case(dd, ctx, 70_001, 12, "bf16", tokens, 0b000011111111, 3, seed=41)
+    assert rec.n_part == 8
+    rec = _case(dd, ctx, 70_001, 12, "f32", tokens, 0b000011111111, 3, seed=42, merges=1)
+    assert rec.n_part == 8
+    rec = _case(dd, ctx, 70_001, 12, "bf16", tokens, 0b000111111111, 3, seed=43, merges=1)
+    assert rec.n_part == 9
+    # one participant: Delta is its own outer gradient
+    rec = _case(dd, ctx, 9_001, 3, "bf16", [1, 2, 3], 0b010, 1, seed=44, merges=1)
+    assert rec.n_part == 1
+
+
+def test_rda_two_launch_form_collinear_gradients(dd, ctx):
+    # every learner moved along the same direction by a different amount: the Gram matrix has rank
+    # one, a^T G a = (sum a_j k_j)^2 |d|^2, and RDA equals the weighted mean of the gradients
+    n, M = 50_000, 4
+    rng = np.random.default_rng(5)
+    theta = rng.normal(0, 0.02, n).astype(np.float32)
+    d = rng.normal(0, 1e-3, n).astype(np.float32)
+    learners = [(theta - np.float32(k) * d).astype(np.float32) for k in (1.0, 2.0, 0.5, 4.0)]
+    v = np.zeros(n, dtype=np.float32)
+    tokens, mask = [3, 1, 4, 1], 0b1111
+    o_t, o_v = theta.copy(), v.copy()
+    ref = oracle.merge_fragment(o_t, o_v, learners, tokens, mask, 1, ETA, MU, merge=oracle.MERGE_RDA)
+    t_dev, v_dev = torch.from_numpy(theta).cuda(), torch.from_numpy(v).cuda()
+    rec_buf = dd.new_records(1)
+    ctx.merge_fragment_rda(t_dev, v_dev, [torch.from_numpy(a).cuda() for a in learners], tokens, mask, 1,
+                           ETA, MU, flags=dd.DIAG_STATE, record=rec_buf)
+    torch.cuda.synchronize()
+    _check_record(dd.read_records(rec_buf)[0], ref)
+    assert floor_rel_err(t_dev.cpu().numpy(), o_t) <= TOL_STATE
+    assert floor_rel_err(v_dev.cpu().numpy(), o_v) <= TOL_STATE
+
+
+def test_rda_two_launch_bounded_wait_expiry(dd, ctx):
+    # the Gram launch stages through CTA-wide barriers of its own: the test hook makes the first
+    # stage of every CTA wait for bytes that never come; every wait runs out, the record says so,
+    # and the context works normally afterwards
+    n, M = 300_000, 3
+    theta, v, learners = synth.fragment_cpu(n, M, "bf16", 77)
+    t_dev, v_dev = torch.from_numpy(theta).cuda(), torch.from_numpy(v).cuda()
+    L = [to_torch_learner(a, "cuda") for a in learners]
+    rec_buf = dd.new_records(1)
+    ctx.merge_fragment_rda(t_dev, v_dev, L, [1, 2, 3], 0b111, 1, ETA, MU, flags=dd.DEBUG_EXPIRE_WAIT,
+                           record=rec_buf)
+    torch.cuda.synchronize()
+    rec = dd.read_records(rec_buf)[0]
+    assert rec.status == dd.STATUS_WAIT_LIMIT and rec.idx == [0, 1, 2]
+    t_dev.copy_(torch.from_numpy(theta))
+    v_dev.copy_(torch.from_numpy(v))
+    ref = oracle.merge_fragment(theta, v, learners, [1, 2, 3], 0b111, 1, ETA, MU, merge=oracle.MERGE_RDA)
+    ctx.merge_fragment_rda(t_dev, v_dev, L, [1, 2, 3], 0b111, 1, ETA, MU, flags=dd.DIAG_STATE, record=rec_buf)
+    torch.cuda.synchronize()
+    _check_record(dd.read_records(rec_buf)[0], ref)
+    assert floor_rel_err(t_dev.cpu().numpy(), theta) <= TOL_STATE
+    assert floor_rel_err(v_dev.cpu().numpy(), v) <= TOL_STATE
