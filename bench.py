@@ -760,6 +760,9 @@ def config_row(dd, ctx, device, name, merge, args, ceilings, probes, traffic_tab
                 row["ms_cuda_graph_replay"] = merger.timed_graph()
         else:
             row["l2"] = "inputs larger than L2 (no flush)"
+        if not args.no_e2e and merge in ("avg", "int4") and not (merge == "avg" and not own):
+            # end to end from pinned host memory; the large workloads stream a bounded slice
+            row["e2e"] = e2e_leg(dd, ctx, merger, args, 1, pinned_cap_bytes=12 << 30, steps=2)
         if probes is not None and merge == "push" and w.learner_dtype == "bf16":
             s_all = row["participants"][0]
             row["pattern_probe_gbs"] = probes.run(rd2=s_all, rd4=2, wr4=2, wr2=s_all, push_in_place=True, reps=5)
@@ -934,60 +937,101 @@ def run_replay(args, ceilings=None):
     return line
 
 
-def e2e_leg(dd, ctx, merger, args, world):
-    """End to end through the public host-buffer call: pinned host buffers in, results in host
-    memory, host<->device copies inside the timed region."""
+def e2e_leg(dd, ctx, merger, args, world, pinned_cap_bytes=None, steps=None):
+    """End to end through the public host-buffer calls: pinned host buffers in, results in host
+    memory, host<->device copies inside the timed region.  One fragment of learner copies goes
+    through dd_merge_fragment_host, several through dd_merge_fragments_batched_host, int4 payloads
+    through dd_merge_fragment_int4_host."""
     import torch
     import torch.distributed as dist
 
     from paper_2604_21428_b200 import dist as ddist
-    w, f = merger.w, merger.frags[0]
-    n = f["n"]
-    part = [m for m in range(w.M) if (f["quorum_mask"] >> m) & 1 and f["tokens"][m] > 0]
-    # Page-locked host memory is bounded: every rank of the node pins its own buffers, so
-    # with several ranks (or little free host memory) the end-to-end leg streams a leading
-    # slice of the fragment instead of all of it.
+    w = merger.w
+    steps = steps or args.e2e_steps
+    int4 = merger.merge == "int4"
     esz = 2 if w.learner_dtype == "bf16" else 4
-    per_elem = len(part) * esz + 8
+    parts = [[m for m in range(w.M) if (f["quorum_mask"] >> m) & 1 and f["tokens"][m] > 0] for f in merger.frags]
+
+    def in_bytes(p, n):       # host-to-device bytes of n elements of fragment p
+        if int4:
+            return len(parts[p]) * ((n + 1) // 2 + (n + 127) // 128 * 4) + 8 * n
+        return n * (len(parts[p]) * esz + 8)
+
+    # Page-locked host memory is bounded: every rank of the node pins its own buffers, so with
+    # several ranks (or little free host memory, or a cap given by the caller) the end-to-end leg
+    # streams a leading slice of every fragment instead of all of it.
     try:
         avail = next(int(l.split()[1]) * 1024 for l in open("/proc/meminfo") if l.startswith("MemAvailable"))
     except Exception:
         avail = 64 << 30
     local_world = int(os.environ.get("LOCAL_WORLD_SIZE", str(world)))
     budget = int(0.4 * avail / max(local_world, 1))
-    n = max(8, min(n, budget // per_elem) // 8 * 8)
-    h_theta = torch.empty(n, dtype=torch.float32, pin_memory=True)
-    h_mom = torch.empty(n, dtype=torch.float32, pin_memory=True)
-    h_theta.copy_(f["global_"][:n])
-    h_mom.copy_(f["momentum"][:n])
-    h_learners = [None] * w.M
-    for m in part:
-        h_learners[m] = torch.empty(n, dtype=f["learners"][m].dtype, pin_memory=True)
-        h_learners[m].copy_(f["learners"][m][:n])
-    h2d = n * (len(part) * esz + 8)
-    d2h = n * 8 + dd.RECORD_BYTES
-    ctx.merge_fragment_host(h_theta, h_mom, h_learners, f["tokens"], f["quorum_mask"], f["K"],
-                            merger.eta, merger.mu, n=n, learner_dtype=merger.ldtype, flags=merger.flags)  # warm-up
+    if pinned_cap_bytes:
+        budget = min(budget, pinned_cap_bytes)
+    full = sum(in_bytes(p, f["n"]) for p, f in enumerate(merger.frags))
+    share = min(1.0, budget / max(full, 1))
+    align = 128 if int4 else 8
+    sizes = [max(align, int(f["n"] * share) // align * align) if share < 1.0 else f["n"] for f in merger.frags]
+    host_frags, h2d, d2h = [], 0, 0
+    for p, (f, n) in enumerate(zip(merger.frags, sizes)):
+        h_theta = torch.empty(n, dtype=torch.float32, pin_memory=True)
+        h_mom = torch.empty(n, dtype=torch.float32, pin_memory=True)
+        h_theta.copy_(f["global_"][:n])
+        h_mom.copy_(f["momentum"][:n])
+        hf = dict(global_=h_theta, momentum=h_mom, tokens=f["tokens"], quorum_mask=f["quorum_mask"], K=f["K"], n=n)
+        if int4:
+            hf["codes"], hf["scales"] = [None] * w.M, [None] * w.M
+            for m in parts[p]:
+                hf["codes"][m] = torch.empty((n + 1) // 2, dtype=torch.uint8, pin_memory=True)
+                hf["codes"][m].copy_(merger.int4_codes[m][:(n + 1) // 2])
+                hf["scales"][m] = torch.empty((n + 127) // 128, dtype=torch.float32, pin_memory=True)
+                hf["scales"][m].copy_(merger.int4_scales[m][:(n + 127) // 128])
+        else:
+            hf["learners"] = [None] * w.M
+            for m in parts[p]:
+                hf["learners"][m] = torch.empty(n, dtype=f["learners"][m].dtype, pin_memory=True)
+                hf["learners"][m].copy_(f["learners"][m][:n])
+        host_frags.append(hf)
+        h2d += in_bytes(p, n)
+        d2h += n * 8 + dd.RECORD_BYTES
+
+    def one_step():
+        if int4:
+            hf = host_frags[0]
+            return [ctx.merge_fragment_int4_host(hf["global_"], hf["momentum"], hf["codes"], hf["scales"],
+                                                 hf["tokens"], hf["quorum_mask"], hf["K"], merger.eta, merger.mu,
+                                                 n=hf["n"], flags=merger.flags)]
+        if w.P == 1:
+            hf = host_frags[0]
+            return [ctx.merge_fragment_host(hf["global_"], hf["momentum"], hf["learners"], hf["tokens"],
+                                            hf["quorum_mask"], hf["K"], merger.eta, merger.mu, n=hf["n"],
+                                            learner_dtype=merger.ldtype, flags=merger.flags)]
+        return ctx.merge_fragments_batched_host(host_frags, w.M, merger.ldtype, merger.eta, merger.mu,
+                                                flags=merger.flags)
+
+    one_step()                                           # warm-up: staging buffers, streams
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
     t0 = time.perf_counter()
-    for _ in range(args.e2e_steps):
-        rec = ctx.merge_fragment_host(h_theta, h_mom, h_learners, f["tokens"], f["quorum_mask"], f["K"],
-                                      merger.eta, merger.mu, n=n, learner_dtype=merger.ldtype,
-                                      flags=merger.flags)
+    for _ in range(steps):
+        recs = one_step()
     torch.cuda.synchronize()
     dt = time.perf_counter() - t0
-    assert rec.status == 0
+    assert all(r.status == 0 for r in recs)
     dt_max = ddist.max_over_ranks(dt, device=merger.device)
-    # every rank streams its own copy (or its own range) of n elements per step
-    out = {"value": n * world * args.e2e_steps / dt_max, "unit": UNIT,
+    n_total = sum(sizes)
+    call = ("dd_merge_fragment_int4_host" if int4 else
+            "dd_merge_fragment_host" if w.P == 1 else "dd_merge_fragments_batched_host")
+    # every rank streams its own copy (or its own range) of the elements per step
+    out = {"value": n_total * world * steps / dt_max, "unit": UNIT,
            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-           "steps": args.e2e_steps, "elements_per_rank_step": n,
-           "h2d_gbs": h2d * args.e2e_steps / dt_max / 1e9,
-           "path": "dd_merge_fragment_host: pinned host buffers, chunked H2D -> kernel -> D2H "
-                   "pipeline, blocking"}
-    del h_learners, h_theta, h_mom
+           "steps": steps, "elements_per_rank_step": n_total,
+           "h2d_gbs": h2d * steps / dt_max / 1e9,
+           "path": f"{call}: pinned host buffers, chunked H2D -> kernel -> D2H pipeline, blocking"}
+    if share < 1.0:
+        out["note"] = f"leading {share:.3f} of every fragment (page-locked host memory is bounded)"
+    del host_frags
     return out
 
 
@@ -1146,7 +1190,7 @@ def run_ours(args):
         "roofline": roofline,
     }
 
-    if not args.no_e2e and w.P == 1 and args.merge == "avg":
+    if not args.no_e2e and args.merge in ("avg", "int4"):
         line["e2e"] = e2e_leg(dd, ctx, merger, args, world)
     else:
         line["e2e"] = None

@@ -354,6 +354,36 @@ int dd_merge_fragment_host(dd_ctx *ctx, float *global, float *momentum,
                            dd_merge_record *record, size_t chunk_elems, void *cuda_stream);
 
 /*
+ * Host-buffer variants of the batched merge and of the int4 merge (Section 4, system overview:
+ * the syncer pulls the fragments from the learners' host RAM; Appendix "Outer gradients
+ * compression": 4 bits per value on the wire).  Same pipeline as dd_merge_fragment_host; the
+ * chunks of successive fragments follow one another without a pause.
+ *
+ * dd_merge_fragments_batched_host: descs[p].global, .momentum, .out_bf16 and every
+ *   descs[p].learner_ptrs[m] are HOST pointers here; records is a HOST array of P records
+ *   (or NULL).  Per fragment the semantics are those of dd_merge_fragment_host.
+ *
+ * dd_merge_fragment_int4_host: code_ptrs[m] / scale_ptrs[m] are HOST pointers to the codes
+ *   ((n + 1) / 2 bytes) and scales (ceil(n / 128) floats) that dd_quantize_outer_gradient_int4
+ *   defines; global, momentum, out_bf16, record are host memory.  chunk_elems (0 = library
+ *   default) must be a multiple of 128 so that no chunk splits a quantisation block.  Only
+ *   s (1/2 + 4/128) + 8 bytes per parameter cross the bus on the way in, against 2 s + 8 for
+ *   bf16 copies.  DD_DIAG_PER_LEARNER is not offered.
+ *
+ * Both block the calling thread until the results are in host memory.
+ */
+int dd_merge_fragments_batched_host(dd_ctx *ctx, const dd_fragment_desc *descs, int P, int M,
+                                    dd_dtype learner_dtype, float outer_lr, float outer_mu,
+                                    uint32_t flags, dd_merge_record *records /* [host] P records or NULL */,
+                                    size_t chunk_elems, void *cuda_stream);
+int dd_merge_fragment_int4_host(dd_ctx *ctx, float *global, float *momentum,
+                                const uint8_t *const *code_ptrs, const float *const *scale_ptrs, int M,
+                                const uint64_t *tokens, const uint64_t *steps, uint64_t quorum_mask,
+                                int K, float outer_lr, float outer_mu, uint32_t flags, size_t n,
+                                void *out_bf16, dd_merge_record *record, size_t chunk_elems,
+                                void *cuda_stream);
+
+/*
  * The batched merge for callers that cannot allocate device memory.  (The paper
  * has no counterpart to this entry point; it exists for deployment reasons only.)
  *

@@ -28,7 +28,8 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libddmerge
 EXPORTS = (
     "dd_create", "dd_destroy", "dd_merge_fragment", "dd_merge_fragments_batched",
     "dd_merge_fragment_push", "dd_merge_fragments_batched_push", "dd_merge_fragments_batched_rda_push", "dd_merge_fragments_batched_rda_pass",
-    "dd_merge_fragment_host", "dd_merge_fragments_batched_noalloc",
+    "dd_merge_fragment_host", "dd_merge_fragments_batched_host", "dd_merge_fragment_int4_host",
+    "dd_merge_fragments_batched_noalloc",
     "dd_merge_fragment_rda", "dd_merge_fragments_batched_rda",
     "dd_quantize_outer_gradient_int4", "dd_merge_fragment_int4",
     "dd_broadcast_fragment", "dd_grace_controller_init", "dd_grace_controller_observe",
@@ -133,6 +134,15 @@ def _load() -> ctypes.CDLL:
     lib.dd_merge_fragment_host.restype = ctypes.c_int
     lib.dd_merge_fragment_host.argtypes = [
         vp, vp, vp, ctypes.POINTER(vp), ctypes.c_int, ctypes.c_int, u64p, u64p, ctypes.c_uint64,
+        ctypes.c_int, ctypes.c_float, ctypes.c_float, ctypes.c_uint32, ctypes.c_size_t, vp,
+        ctypes.POINTER(CRecord), ctypes.c_size_t, vp]
+    lib.dd_merge_fragments_batched_host.restype = ctypes.c_int
+    lib.dd_merge_fragments_batched_host.argtypes = [
+        vp, ctypes.POINTER(CFragmentDesc), ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_float,
+        ctypes.c_float, ctypes.c_uint32, ctypes.POINTER(CRecord), ctypes.c_size_t, vp]
+    lib.dd_merge_fragment_int4_host.restype = ctypes.c_int
+    lib.dd_merge_fragment_int4_host.argtypes = [
+        vp, vp, vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.c_int, u64p, u64p, ctypes.c_uint64,
         ctypes.c_int, ctypes.c_float, ctypes.c_float, ctypes.c_uint32, ctypes.c_size_t, vp,
         ctypes.POINTER(CRecord), ctypes.c_size_t, vp]
     lib.dd_merge_fragments_batched_noalloc.restype = ctypes.c_int
@@ -457,6 +467,42 @@ class Context:
         rec = CRecord()
         self._check(lib.dd_merge_fragment_host(
             self._h, _ptr(global_), _ptr(momentum), ptrs, M, learner_dtype, _u64_array(tokens),
+            None if steps is None else _u64_array(steps),
+            ctypes.c_uint64(quorum_mask & (2**64 - 1)), int(K), ctypes.c_float(outer_lr),
+            ctypes.c_float(outer_mu), ctypes.c_uint32(flags), ctypes.c_size_t(n), _ptr(out_bf16),
+            ctypes.byref(rec) if want_record else None, ctypes.c_size_t(chunk_elems),
+            _stream_handle(stream)))
+        return _parse_record(rec) if want_record else None
+
+    def merge_fragments_batched_host(self, fragments, M: int, learner_dtype: int, outer_lr: float,
+                                     outer_mu: float, *, flags: int = 0, want_records: bool = True,
+                                     chunk_elems: int = 0, stream=None):
+        """``dd_merge_fragments_batched_host``: like ``merge_fragments_batched`` with every tensor
+        of every fragment in HOST memory (ideally pinned).  Blocks until the results are in host
+        memory; returns the fragments' Records (or None)."""
+        P = len(fragments)
+        descs, _keep = _pack_descs(fragments, M)
+        recs = (CRecord * max(P, 1))() if want_records else None
+        self._check(lib.dd_merge_fragments_batched_host(
+            self._h, descs, P, M, learner_dtype, ctypes.c_float(outer_lr), ctypes.c_float(outer_mu),
+            ctypes.c_uint32(flags), recs, ctypes.c_size_t(chunk_elems), _stream_handle(stream)))
+        return [_parse_record(recs[p]) for p in range(P)] if want_records else None
+
+    def merge_fragment_int4_host(self, global_, momentum, codes, scales, tokens, quorum_mask: int, K: int,
+                                 outer_lr: float, outer_mu: float, *, n: int | None = None, steps=None,
+                                 flags: int = 0, out_bf16=None, want_record: bool = True,
+                                 chunk_elems: int = 0, stream=None):
+        """``dd_merge_fragment_int4_host``: ``codes`` / ``scales`` are lists of M HOST tensors (or
+        None for absent learners); ``global_`` and ``momentum`` host tensors updated in place.
+        Blocks until the results are in host memory; returns the fragment's Record."""
+        M = len(codes)
+        if n is None:
+            n = int(global_.numel())
+        cp = (ctypes.c_void_p * M)(*[_ptr(t) for t in codes])
+        sp = (ctypes.c_void_p * M)(*[_ptr(t) for t in scales])
+        rec = CRecord()
+        self._check(lib.dd_merge_fragment_int4_host(
+            self._h, _ptr(global_), _ptr(momentum), cp, sp, M, _u64_array(tokens),
             None if steps is None else _u64_array(steps),
             ctypes.c_uint64(quorum_mask & (2**64 - 1)), int(K), ctypes.c_float(outer_lr),
             ctypes.c_float(outer_mu), ctypes.c_uint32(flags), ctypes.c_size_t(n), _ptr(out_bf16),
