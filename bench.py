@@ -387,6 +387,11 @@ def spawn_ranks(args, argv) -> int:
     """``python bench.py --gpus N`` outside a launcher: starts the N ranks itself (what
     ``python -m torch.distributed.run --nproc-per-node N`` would do) and waits for them.  Rank 0
     prints the JSON line; the exit code is the first non-zero one."""
+    import torch
+    have = torch.cuda.device_count()
+    if have < args.gpus:
+        sys.stderr.write(f"bench.py: --gpus {args.gpus} asks for more GPUs than this node has ({have})\n")
+        return 2
     plan = launch_plan(args.gpus, argv)
     procs = []
     for item in plan:
@@ -816,6 +821,7 @@ def broadcast_row(dd, ctx, merger, args, ceilings, probes):
            "frac_of_nominal_8TBs": alg / (avg * 1e-3) / 1e9 / NOMINAL_HBM_GBS, "launches_per_merge": 1,
            "steps": args.config_steps, "l2": "inputs larger than L2 (no flush)",
            "note": "dd_broadcast_fragment, alpha = 0: the learner side of a syncer update on its own"}
+    row["traffic_bytes_per_param_ncu"] = ncu_traffic_table().get(("broadcast", w.name))
     if ceilings:
         blend = blend_ceiling(ceilings["read_gbs"], ceilings["write_gbs"], row["write_share"])
         row["blend_ceiling_gbs"] = blend
@@ -1202,9 +1208,11 @@ def run_ours(args):
         line["cpu_baseline"] = None
 
     # ---- one row per other workload and merge kind (N = 1 only) ------------------------------
-    if rank == 0 and world == 1 and args.scale == 1.0:
+    if rank == 0 and world == 1:
         rows = []
         todo = wanted_configs(args, args.workload, args.merge)
+        if args.scale != 1.0:        # a shrunk run (profiling): only the rows that reuse the resident buffers
+            todo = [x for x in todo if x in ("rda", "int4", "push", "broadcast")]
         for name in [x for x in todo if x in ("rda", "int4", "push", "broadcast")]:
             # the other merge kinds of the headline workload, on the buffers that are already resident
             if w.P == 1 and args.merge == "avg" and w.learner_dtype == "bf16":

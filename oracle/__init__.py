@@ -89,6 +89,12 @@ def _load():
             ctypes.c_int, u64p, u64p, ctypes.c_uint64, ctypes.c_int, ctypes.c_float,
             ctypes.c_float, ctypes.c_int, ctypes.c_int, ctypes.c_size_t, ctypes.c_void_p,
             ctypes.POINTER(_Record)]
+        lib.ddo_merge_fragment_rda_stage.restype = ctypes.c_int
+        lib.ddo_merge_fragment_rda_stage.argtypes = [
+            ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.c_int,
+            ctypes.c_int, u64p, u64p, ctypes.c_uint64, ctypes.c_int, ctypes.c_float, ctypes.c_float,
+            ctypes.c_int, ctypes.c_size_t, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
+            ctypes.c_void_p, ctypes.POINTER(_Record)]
         lib.ddo_apply_to_learner.restype = None
         lib.ddo_apply_to_learner.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p,
                                              ctypes.c_float, ctypes.c_size_t]
@@ -216,6 +222,40 @@ def select_quorum(arrival, K: int, grace: float):
     if st == INVALID:
         raise ValueError("oracle: invalid quorum arguments")
     return st, int(mask.value), int(n_adm.value)
+
+
+def merge_fragment_rda_stage(stage: int, theta: np.ndarray, v: np.ndarray, learners, tokens, mask: int,
+                             K: int, eta: float, mu: float, *, norms_sq=None, dir_sq: float = 0.0,
+                             steps=None, nesterov: bool = True, out_bf16: np.ndarray | None = None):
+    """One stage (0 norms, 1 direction, 2 outer step) of the radial-directional merge on ONE element
+    range of a sharded fragment; the caller sums each stage's output over the ranges before the next
+    stage.  ``norms_sq``: the summed stage-0 output (participant order); ``dir_sq``: the summed
+    stage-1 output.  Stage 2 updates ``theta`` and ``v`` in place.  Returns (Record, dir_sq of this
+    range for stage 1)."""
+    lib = _load()
+    assert theta.dtype == np.float32 and v.dtype == np.float32 and theta.shape == v.shape
+    n, M = theta.size, len(learners)
+    present = [a for a in learners if a is not None]
+    is_bf16 = bool(present) and present[0].dtype == np.uint16
+    ptrs = (ctypes.c_void_p * M)(*[None if a is None else a.ctypes.data for a in learners])
+    for a in present:
+        assert a.flags.c_contiguous and a.size == n
+    norms = None if norms_sq is None else (ctypes.c_double * MAX_LEARNERS)(*[float(x) for x in norms_sq])
+    dsq = ctypes.c_double(float(dir_sq))
+    rec = _Record()
+    rc = lib.ddo_merge_fragment_rda_stage(
+        int(stage), theta.ctypes.data, v.ctypes.data, ptrs, M, int(is_bf16), _u64(tokens),
+        None if steps is None else _u64(steps), ctypes.c_uint64(mask & (2**64 - 1)), K, ctypes.c_float(eta),
+        ctypes.c_float(mu), int(nesterov), n, norms, ctypes.byref(dsq),
+        None if out_bf16 is None else out_bf16.ctypes.data, ctypes.byref(rec))
+    if rc != 0:
+        raise ValueError("oracle: invalid arguments of a radial-directional stage")
+    s = rec.n_part
+    out = Record(status=rec.status, n_part=s, idx=[int(rec.idx[j]) for j in range(s)],
+                 w_hat=[float(rec.w_hat[j]) for j in range(s)], w_total=float(rec.w_total),
+                 delta_sq=float(rec.delta_sq), theta_sq=float(rec.theta_sq), mom_sq=float(rec.mom_sq),
+                 delta_m_sq=[float(rec.delta_m_sq[j]) for j in range(s)])
+    return out, float(dsq.value)
 
 
 def apply_to_learner(learner: np.ndarray, theta: np.ndarray, alpha: float) -> None:

@@ -255,6 +255,96 @@ int ddo_merge_fragment(float *Theta, float *v, const void *const *learners, int 
     return 0;
 }
 
+/*
+ * Radial-directional averaging of a fragment that is cut by element range over several syncer
+ * shards.  The paper's sharded syncer all-reduces the norms first and the directions second
+ * (appendix "Merging methods"); so one call does ONE stage on this shard's n elements and the
+ * caller sums the stage's output over the shards before the next stage:
+ *
+ *   stage 0  rec->delta_m_sq[j] = sum_i (Theta_i - theta_{j,i})^2 over the shard    -> sum over shards
+ *   stage 1  *dir_sq = sum_i u_i^2,  u = sum_j (w_hat_j / ||D_j||) D_j, with ||D_j||
+ *            from norms_sq (the summed stage-0 output)                               -> sum over shards
+ *   stage 2  Delta = (sum_j w_hat_j ||D_j||) u / sqrt(*dir_sq) with the summed *dir_sq, then the
+ *            outer step on the shard; rec->delta_sq, theta_sq, mom_sq are the shard's -> sum over shards
+ *
+ * Participation and weights are recomputed in every stage (they depend on the counters only).
+ * With a single shard the three stages are ddo_merge_fragment(..., DDO_MERGE_RDA).
+ */
+int ddo_merge_fragment_rda_stage(int stage, float *Theta, float *v, const void *const *learners, int M,
+                                 int learner_is_bf16, const uint64_t *tokens, const uint64_t *steps,
+                                 uint64_t mask, int K, float eta, float mu, int nesterov, size_t n,
+                                 const double *norms_sq, double *dir_sq, uint16_t *out_bf16,
+                                 ddo_record *rec)
+{
+    double w_hat[DDO_MAX_LEARNERS], dir_coef[DDO_MAX_LEARNERS];
+    double radial = 0.0, scale;
+    const double eta_d = (double)eta, mu_d = (double)mu;
+    size_t i;
+    int j, s, st;
+
+    memset(rec, 0, sizeof *rec);
+    st = ddo_participants(mask, tokens, M, K, rec->idx, &rec->n_part);
+    if (st == DDO_INVALID) return DDO_INVALID;
+    s = rec->n_part;
+    if (st != DDO_STATUS_OK) { rec->status = st; return 0; }
+    st = ddo_weights(tokens, steps, rec->idx, s, w_hat, &rec->w_total);
+    if (st == DDO_INVALID) return DDO_INVALID;
+    if (st != DDO_STATUS_OK) { rec->status = st; return 0; }
+    for (j = 0; j < s; ++j) {
+        rec->w_hat[j] = w_hat[j];
+        if (learners[rec->idx[j]] == NULL) return DDO_INVALID;
+    }
+    rec->status = DDO_STATUS_OK;
+
+    if (stage == 0) {
+        for (j = 0; j < s; ++j) {
+            double acc = 0.0;
+            for (i = 0; i < n; ++i) {
+                double d = (double)Theta[i] - learner_at(learners[rec->idx[j]], learner_is_bf16, i);
+                acc += d * d;
+            }
+            rec->delta_m_sq[j] = acc;
+        }
+        return 0;
+    }
+    if (norms_sq == NULL || dir_sq == NULL) return DDO_INVALID;
+    for (j = 0; j < s; ++j) {
+        double nm = sqrt(norms_sq[j]);
+        rec->delta_m_sq[j] = norms_sq[j];
+        radial += w_hat[j] * nm;
+        dir_coef[j] = nm > 0.0 ? w_hat[j] / nm : 0.0;
+    }
+    if (stage == 1) {
+        double acc = 0.0;
+        for (i = 0; i < n; ++i) {
+            double T = (double)Theta[i], u = 0.0;
+            for (j = 0; j < s; ++j)
+                u += dir_coef[j] * (T - learner_at(learners[rec->idx[j]], learner_is_bf16, i));
+            acc += u * u;
+        }
+        *dir_sq = acc;
+        return 0;
+    }
+    if (stage != 2) return DDO_INVALID;
+    scale = *dir_sq > 0.0 ? radial / sqrt(*dir_sq) : 0.0;
+    for (i = 0; i < n; ++i) {
+        double T = (double)Theta[i], d = 0.0, vn, u, Tn;
+        for (j = 0; j < s; ++j)
+            d += dir_coef[j] * (T - learner_at(learners[rec->idx[j]], learner_is_bf16, i));
+        d *= scale;
+        vn = mu_d * (double)v[i] + d;
+        u = nesterov ? d + mu_d * vn : vn;
+        Tn = T - eta_d * u;
+        v[i] = (float)vn;
+        Theta[i] = (float)Tn;
+        if (out_bf16 != NULL) out_bf16[i] = ddo_bf16_rne((float)Tn);
+        rec->delta_sq += d * d;
+        rec->theta_sq += (double)Theta[i] * (double)Theta[i];
+        rec->mom_sq += (double)v[i] * (double)v[i];
+    }
+    return 0;
+}
+
 /* ---- learner side of an update (Algorithm 1 step 3; appendix "Mixing learner and syncer params") */
 
 /* theta_m <- alpha theta_m + (1 - alpha) Theta, rounded to the learner dtype. */

@@ -56,7 +56,9 @@ def test_spawned_ranks_run_with_their_environment(tmp_path):
     args = bench.parse_args(["--gpus", "3", "--impl", "reference", "--steps", "1", "--warmup", "0",
                              "--workload", "tiny"])
     script = tmp_path / "run.py"
-    script.write_text("import sys\nsys.path.insert(0, %r)\nimport bench\n"
+    # (the launcher refuses to start more ranks than there are GPUs: none are needed for this arm)
+    script.write_text("import sys\nsys.path.insert(0, %r)\nimport bench, torch\n"
+                      "torch.cuda.device_count = lambda: 3\n"
                       "sys.exit(bench.spawn_ranks(bench.parse_args(%r), %r))\n"
                       % (ROOT, ["--gpus", "3"], ["--gpus", "3", "--impl", "reference", "--steps", "1",
                                                  "--warmup", "0", "--workload", "tiny"]))

@@ -131,7 +131,7 @@ def _run(name, n_windows, merges):
             assert abs(rec.theta_sq - _sq(f["global_"])) <= TOL_NORM * rec.theta_sq
             assert abs(rec.mom_sq - _sq(f["momentum"])) <= TOL_NORM * rec.mom_sq
         if expect_dsq is not None:
-            assert abs(recs[0].delta_sq - expect_dsq) <= 1e-4 * expect_dsq, (recs[0].delta_sq, expect_dsq)
+            assert abs(recs[0].delta_sq - expect_dsq) <= TOL_NORM * expect_dsq, (recs[0].delta_sq, expect_dsq)
     ctx.close()
 
 
@@ -266,7 +266,7 @@ def test_scale500m_full_size_rda_properties():
         u = sum(wf[j] / norms[j] * (t0 - ls[j]) for j in range(len(part)))
         delta = mom[lo:hi].double().cpu().numpy() - MU * v0           # v' = mu v + Delta
         # Delta = c u with one factor for the whole fragment, fixed by the norms
-        assert floor_rel_err(delta, c_expected * u) <= 1e-4
+        assert floor_rel_err(delta, c_expected * u) <= TOL_STATE
     assert abs(rec.theta_sq - _sq(theta)) <= TOL_NORM * rec.theta_sq
     assert abs(rec.mom_sq - _sq(mom)) <= TOL_NORM * rec.mom_sq
     ctx.close()

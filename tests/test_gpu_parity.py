@@ -690,3 +690,43 @@ def test_per_learner_norms_around_the_shared_memory_limit(dd, ctx, s):
     tokens = [100 + 3 * m for m in range(M)]
     run_case(dd, ctx, 3 * 8192 + 70_001, M, "bf16", tokens, (1 << s) - 1, s, seed=300 + s,
              flags=dd.DIAG_STATE | dd.DIAG_PER_LEARNER, merges=1)
+
+
+@pytest.mark.parametrize("shards", [2, 3])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_range_sharded_direct_average_equals_unsharded(dd, ctx, shards, dtype):
+    """A fragment cut into contiguous element ranges, as a multi-GPU job holds it (one range per
+    rank, no data-path collective): every range is merged by its own call -- here all on one GPU --
+    and the ranges' squared norms are added up, which is what the job's one small all-reduce does.
+    Result: the oracle's merge of the whole fragment."""
+    from paper_2604_21428_b200 import dist as ddist
+
+    n, M = 200_003, 5
+    tokens, mask, K = [100, 200, 0, 400, 500], 0b11101, 3
+    theta, v, learners = synth.fragment_cpu(n, M, dtype, 4242)
+    t_dev, v_dev = torch.from_numpy(theta).cuda(), torch.from_numpy(v).cuda()
+    l_dev = [to_torch_learner(a, "cuda") for a in learners]
+    out_dev = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+    o_out = np.zeros(n, dtype=np.uint16)
+    ref = oracle.merge_fragment(theta, v, learners, tokens, mask, K, ETA, MU, out_bf16=o_out)
+    ranges = [ddist.shard_range(n, r, shards) for r in range(shards)]
+    assert ranges[0][0] == 0 and ranges[-1][1] == n and all(a[1] == b[0] for a, b in zip(ranges, ranges[1:]))
+    recs = [dd.new_records(1) for _ in range(shards)]
+    for (lo, hi), rec in zip(ranges, recs):
+        ctx.merge_fragment(t_dev[lo:hi], v_dev[lo:hi], [t[lo:hi] for t in l_dev], tokens, mask, K, ETA, MU,
+                           n=hi - lo, learner_dtype=dd.BF16 if dtype == "bf16" else dd.F32,
+                           flags=dd.DIAG_STATE | dd.DIAG_PER_LEARNER, out_bf16=out_dev[lo:hi], record=rec)
+    torch.cuda.synchronize()
+    per_rank = [dd.read_records(rec)[0] for rec in recs]
+    # what dist.allreduce_record leaves on every rank: identical participation and weights, summed norms
+    total = per_rank[0]
+    for r in per_rank[1:]:
+        assert (r.status, r.n_part, r.idx, r.w_hat) == (total.status, total.n_part, total.idx, total.w_hat)
+    import dataclasses
+    total = dataclasses.replace(total, delta_sq=sum(r.delta_sq for r in per_rank),
+                                theta_sq=sum(r.theta_sq for r in per_rank), mom_sq=sum(r.mom_sq for r in per_rank),
+                                delta_m_sq=[sum(r.delta_m_sq[j] for r in per_rank) for j in range(total.n_part)])
+    assert_record_matches(total, ref)
+    assert floor_rel_err(t_dev.cpu().numpy(), theta) <= TOL_STATE
+    assert floor_rel_err(v_dev.cpu().numpy(), v) <= TOL_STATE
+    assert floor_rel_err(bf16_bits_to_f32(out_dev), oracle.bf16_to_f32(o_out)) <= TOL_BF16

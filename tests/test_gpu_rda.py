@@ -32,7 +32,7 @@ def _check_record(got, ref):
     assert got.w_hat == [float(np.float32(w)) for w in ref.w_hat]
     for name in ("delta_sq", "theta_sq", "mom_sq"):
         a, b = getattr(got, name), getattr(ref, name)
-        assert abs(a - b) <= 4 * TOL_NORM * abs(b) + 1e-300, (name, a, b)
+        assert abs(a - b) <= TOL_NORM * abs(b) + 1e-300, (name, a, b)
     for a, b in zip(got.delta_m_sq, ref.delta_m_sq):
         assert abs(a - b) <= TOL_NORM * abs(b) + 1e-300
 
@@ -150,7 +150,7 @@ def test_batched_mixed_avg_and_rda(dd, ctx):
             ref = oracle.merge_fragment(theta, v, learners, dev[p]["tokens"], masks[p], K, ETA, MU,
                                         merge=oracle.MERGE_RDA if kinds[p] else oracle.MERGE_AVG)
             assert (recs[p].status, recs[p].idx) == (ref.status, ref.idx)
-            assert abs(recs[p].delta_sq - ref.delta_sq) <= 4 * TOL_NORM * ref.delta_sq
+            assert abs(recs[p].delta_sq - ref.delta_sq) <= TOL_NORM * ref.delta_sq
             assert abs(recs[p].theta_sq - ref.theta_sq) <= TOL_NORM * ref.theta_sq
             assert floor_rel_err(dev[p]["global_"].cpu().numpy(), theta) <= TOL_STATE, (k, p)
             assert floor_rel_err(dev[p]["momentum"].cpu().numpy(), v) <= TOL_STATE, (k, p)

@@ -150,3 +150,95 @@ def test_range_sharded_rda_hands_over_between_passes(world):
     out = mgr.dict()
     mp.spawn(_rda_worker, args=(world, _free_port(), out), nprocs=world, join=True)
     assert all(out[r] for r in range(world)) and len(out) == world
+
+
+class _OraclePassCtx:
+    """The three passes of a range-sharded radial-directional merge done by the ORACLE on this rank's
+    element range, behind the interface of the library's per-pass call: each pass reads the hand-over
+    fields that the previous all-reduce left in the records buffer and writes its own share."""
+
+    def __init__(self, dd, shards):
+        self.dd, self.shards = dd, shards          # shards[p] = (theta, v, learners) of this rank's range
+
+    def _table(self, records):
+        return records.view(torch.float64).view(-1, self.dd.RECORD_BYTES // 8)
+
+    def merge_fragments_batched_rda_pass(self, fragments, M, learner_dtype, lr, mu, pass_index, *, records,
+                                         scratch, merge_kinds=None, flags=0, push_masks=None, stream=None):
+        dd, t = self.dd, self._table(records)
+        a, _ = dd.record_field_columns("delta_m_sq")
+        c, _ = dd.record_field_columns("delta_sq")
+        for p, f in enumerate(fragments):
+            theta, v, learners = self.shards[p]
+            st, idx = oracle.participants(f["quorum_mask"], f["tokens"], f["K"])
+            s = len(idx)
+            norms = [float(x) for x in t[p, a:a + s]]
+            rec, dsq = oracle.merge_fragment_rda_stage(pass_index, theta, v, learners, f["tokens"],
+                                                       f["quorum_mask"], f["K"], lr, mu,
+                                                       norms_sq=norms if pass_index > 0 else None,
+                                                       dir_sq=float(t[p, c]) if pass_index == 2 else 0.0)
+            if pass_index == 0:
+                t[p, a:a + s] = torch.tensor(rec.delta_m_sq, dtype=torch.float64)
+            elif pass_index == 1:
+                t[p, c] = dsq
+            else:
+                for name in ("delta_sq", "theta_sq", "mom_sq"):
+                    t[p, dd.record_field_columns(name)[0]] = getattr(rec, name)
+
+
+def _rda_oracle_worker(rank, world, port, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        from paper_2604_21428_b200 import ddmerge as dd
+        M, K = 5, 2
+        sizes = [10_007, 4_099]
+        tokens = [[100, 0, 300, 400, 500], [7, 9, 11, 0, 13]]
+        masks = [0b11101, 0b10111]
+        whole, shards, frags, ranges = [], [], [], []
+        for p, n in enumerate(sizes):
+            theta, v, learners = synth.fragment_cpu(n, M, "bf16", seed=900 + p)     # same on every rank
+            v[:] = np.random.default_rng(p).normal(0, 1e-4, n).astype(np.float32)
+            whole.append((theta, v, learners))
+            lo, hi = ddist.shard_range(n, rank, world)
+            ranges.append((lo, hi))
+            shards.append((theta[lo:hi].copy(), v[lo:hi].copy(), [a[lo:hi].copy() for a in learners]))
+            frags.append(dict(tokens=tokens[p], quorum_mask=masks[p], K=K, n=hi - lo))
+        records = torch.zeros(len(sizes) * dd.RECORD_BYTES, dtype=torch.uint8)
+        ddist.rda_merge_range_sharded(_OraclePassCtx(dd, shards), frags, M, dd.BF16, 0.7, 0.9,
+                                      records=records, scratch=torch.zeros(8))
+        parts = [None] * world
+        dist.all_gather_object(parts, [(ranges[p], shards[p][0], shards[p][1]) for p in range(len(sizes))])
+        ok = True
+        t = records.view(torch.float64).view(len(sizes), dd.RECORD_BYTES // 8)
+        for p, n in enumerate(sizes):
+            theta, v, learners = whole[p]
+            ref = oracle.merge_fragment(theta, v, learners, tokens[p], masks[p], K, 0.7, 0.9,
+                                        merge=oracle.MERGE_RDA)
+            t_full, v_full = np.empty(n, np.float32), np.empty(n, np.float32)
+            for per_rank in parts:
+                (lo, hi), ts, vs = per_rank[p]
+                t_full[lo:hi], v_full[lo:hi] = ts, vs
+            # the shards' sums are taken in another order than the whole fragment's: a few ulps of
+            # the norms, hence of Delta, hence at most an ulp or two of the float32 state
+            ok = ok and float(np.max(np.abs(t_full - theta))) <= 2e-9 and float(np.max(np.abs(v_full - v))) <= 1e-9
+            for name in ("delta_sq", "theta_sq", "mom_sq"):
+                got = float(t[p, dd.record_field_columns(name)[0]])
+                ok = ok and abs(got - getattr(ref, name)) <= 1e-10 * getattr(ref, name)
+            a, _ = dd.record_field_columns("delta_m_sq")
+            ok = ok and all(abs(float(t[p, a + j]) - x) <= 1e-12 * x for j, x in enumerate(ref.delta_m_sq))
+        out[rank] = bool(ok)
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_range_sharded_rda_with_oracle_shards_equals_whole_fragment(world):
+    """dist.rda_merge_range_sharded on gloo ranks, every rank's passes computed by the oracle on
+    its own element range: after the two all-reduces the gathered fragment equals the oracle's
+    radial-directional merge of the whole fragment, and every rank holds whole-fragment norms."""
+    mgr = mp.Manager()
+    out = mgr.dict()
+    mp.spawn(_rda_oracle_worker, args=(world, _free_port(), out), nprocs=world, join=True)
+    assert all(out[r] for r in range(world)) and len(out) == world

@@ -511,6 +511,39 @@ def test_huge_token_counts():
         oracle.weights([2**63, 2**63], None, [0, 1])        # the exact sum would wrap
 
 
+def test_rda_stages_equal_the_whole_merge_and_add_up_over_ranges():
+    # one range: the three stages ARE the merge, bit for bit; three ranges with the stage outputs
+    # summed in between: the same merge up to the order of the sums
+    n, M = 3001, 4
+    theta, v, learners = _frag(n=n, M=M, dtype="bf16", seed=55)
+    v[:] = np.random.default_rng(3).normal(0, 1e-3, n).astype(np.float32)
+    tokens, mask, K = [5, 0, 2, 9], 0b1101, 2
+    t_ref, v_ref = theta.copy(), v.copy()
+    ref = oracle.merge_fragment(t_ref, v_ref, learners, tokens, mask, K, 0.7, 0.9, merge=oracle.MERGE_RDA)
+    t1, v1 = theta.copy(), v.copy()
+    r0, _ = oracle.merge_fragment_rda_stage(0, t1, v1, learners, tokens, mask, K, 0.7, 0.9)
+    _, d = oracle.merge_fragment_rda_stage(1, t1, v1, learners, tokens, mask, K, 0.7, 0.9, norms_sq=r0.delta_m_sq)
+    r2, _ = oracle.merge_fragment_rda_stage(2, t1, v1, learners, tokens, mask, K, 0.7, 0.9,
+                                            norms_sq=r0.delta_m_sq, dir_sq=d)
+    np.testing.assert_array_equal(t1, t_ref)
+    np.testing.assert_array_equal(v1, v_ref)
+    assert (r2.delta_sq, r2.theta_sq, r2.mom_sq, r0.delta_m_sq) == (ref.delta_sq, ref.theta_sq, ref.mom_sq, ref.delta_m_sq)
+    cuts = [(0, 1000), (1000, 1008), (1008, n)]
+    shard = [(theta[a:b].copy(), v[a:b].copy(), [x[a:b].copy() for x in learners]) for a, b in cuts]
+    norms = np.sum([oracle.merge_fragment_rda_stage(0, t, m, l, tokens, mask, K, 0.7, 0.9)[0].delta_m_sq
+                    for t, m, l in shard], axis=0)
+    dsq = sum(oracle.merge_fragment_rda_stage(1, t, m, l, tokens, mask, K, 0.7, 0.9, norms_sq=norms)[1]
+              for t, m, l in shard)
+    recs = [oracle.merge_fragment_rda_stage(2, t, m, l, tokens, mask, K, 0.7, 0.9, norms_sq=norms, dir_sq=dsq)[0]
+            for t, m, l in shard]
+    np.testing.assert_allclose(np.concatenate([t for t, _, _ in shard]), t_ref, rtol=0, atol=2e-9)
+    np.testing.assert_allclose(np.concatenate([m for _, m, _ in shard]), v_ref, rtol=0, atol=1e-9)
+    assert abs(sum(r.delta_sq for r in recs) - ref.delta_sq) <= 1e-12 * ref.delta_sq
+    # the stage interface refuses a later stage without the summed output of the earlier one
+    with pytest.raises(ValueError):
+        oracle.merge_fragment_rda_stage(1, t1, v1, learners, tokens, mask, K, 0.7, 0.9)
+
+
 # ---- int4 compression of outer gradients (reading of this build; the paper gives no quantiser) ----
 
 def test_int4_quantiser_properties():
