@@ -210,7 +210,7 @@ int dd_merge_fragments_batched_push(dd_ctx *ctx, const dd_fragment_desc *descs,
  * so that ||Delta|| does not shrink like 1/sqrt(M) when the D_m are nearly
  * orthogonal; the outer step is the same as for dd_merge_fragment.  (The printed
  * weighted formula shows the mean vector in the first factor; it is read as the
- * weighted mean of the norms, "completely analogously" to the unweighted one.)
+ * weighted mean of the norms, by analogy with the unweighted one.)
  * A participant with D_m = 0 adds its (zero) norm to the radial mean and nothing
  * to the direction; if the mean direction vanishes, Delta = 0.
  *

@@ -209,7 +209,7 @@ int ddo_merge_fragment(float *Theta, float *v, const void *const *learners, int 
         /*
          * RDA({v_m, w_m}) = (sum w_m ||v_m|| / sum w_m) * phi(sum w_m phi(v_m) / sum w_m),
          * phi(x) = x / ||x||.  The printed weighted display shows a vector in
-         * the first factor; by "completely analogously" to the unweighted
+         * the first factor; by analogy with the unweighted
          * definition it is read as the weighted mean of the NORMS.  phi is
          * undefined at 0: a participant whose outer gradient is exactly zero
          * contributes its (zero) norm to the radial mean and nothing to the
