@@ -270,7 +270,7 @@ class Probes:
         self.lib.ddp_stream_probe.restype = ctypes.c_double
         self.lib.ddp_stream_probe.argtypes = [
             ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
-            ctypes.c_size_t, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
+            ctypes.c_size_t, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
             ctypes.POINTER(ctypes.c_double)]
         free = torch.cuda.mem_get_info(device)[0]
         self.bytes = int(min(scratch_bytes, max(1 << 30, free // 2)))
@@ -278,7 +278,7 @@ class Probes:
         self.buf.fill_(0x3c)
         self.stream = int(torch.cuda.current_stream().cuda_stream)
 
-    def run(self, rd2=0, rd4=0, wr4=0, wr2=0, push_in_place=False, ctas_per_sm=2, reps=10):
+    def run(self, rd2=0, rd4=0, wr4=0, wr2=0, push_in_place=False, ctas_per_sm=2, ring_depth=3, reps=10):
         """GB/s of the shape (best of ``reps``), streams sized to fill the scratch buffer."""
         row_bytes = 2048 * (rd2 + (0 if push_in_place else wr2)) + 4096 * max(rd4, wr4)
         if push_in_place:
@@ -286,7 +286,7 @@ class Probes:
         rows = (self.bytes - (1 << 20)) // row_bytes
         ms = ctypes.c_double(0.0)
         gbs = self.lib.ddp_stream_probe(self.buf.data_ptr(), self.bytes, rd2, rd4, wr4, wr2,
-                                        rows * 1024, int(push_in_place), ctas_per_sm, reps, self.stream,
+                                        rows * 1024, int(push_in_place), ctas_per_sm, ring_depth, reps, self.stream,
                                         ctypes.byref(ms))
         if gbs < 0:
             raise RuntimeError(f"bandwidth probe failed (code {gbs})")
@@ -312,6 +312,13 @@ def measure_ceilings(device):
                "24 participants, 87.5 % reads (mix); about 9 GB each, best of 10, CUDA events",
     }
     return out, pr
+
+
+def merge_ring_depth(s: int, learner_dtype: str) -> int:
+    """Ring slots the fused merge uses per warp at s participants (the kernel's own rule, so that a
+    pattern probe moves data exactly as the kernel does): one copy in flight for fp32 copies and for
+    up to 7 bf16 copies, two above."""
+    return 2 if learner_dtype != "bf16" or s <= 7 else 3
 
 
 def blend_ceiling(read_gbs: float, write_gbs: float, wshare: float) -> float:
@@ -770,13 +777,15 @@ def config_row(dd, ctx, device, name, merge, args, ceilings, probes, traffic_tab
             row["e2e"] = e2e_leg(dd, ctx, merger, args, 1, pinned_cap_bytes=12 << 30, steps=2)
         if probes is not None and merge == "push" and w.learner_dtype == "bf16":
             s_all = row["participants"][0]
-            row["pattern_probe_gbs"] = probes.run(rd2=s_all, rd4=2, wr4=2, wr2=s_all, push_in_place=True, reps=5)
+            row["pattern_probe_gbs"] = probes.run(rd2=s_all, rd4=2, wr4=2, wr2=s_all, push_in_place=True,
+                                                  ring_depth=merge_ring_depth(s_all, "bf16"), reps=5)
             row["frac_of_pattern_probe"] = row["achieved_gbs"] / row["pattern_probe_gbs"]
         if probes is not None and merge == "avg":
             # the same access pattern with the arithmetic left out, at this workload's mean participant count
             s_mean = max(1, round(sum(row["participants"]) / w.P))
             if w.learner_dtype == "bf16":
-                row["pattern_probe_gbs"] = probes.run(rd2=s_mean, rd4=2, wr4=2, reps=5)
+                row["pattern_probe_gbs"] = probes.run(rd2=s_mean, rd4=2, wr4=2,
+                                                      ring_depth=merge_ring_depth(s_mean, "bf16"), reps=5)
                 row["frac_of_pattern_probe"] = row["achieved_gbs"] / row["pattern_probe_gbs"]
     finally:
         if own:
@@ -1015,6 +1024,7 @@ def e2e_leg(dd, ctx, merger, args, world, pinned_cap_bytes=None, steps=None):
         return ctx.merge_fragments_batched_host(host_frags, w.M, merger.ldtype, merger.eta, merger.mu,
                                                 flags=merger.flags)
 
+    steps = max(1, steps)
     one_step()                                           # warm-up: staging buffers, streams
     if world > 1:
         dist.barrier()

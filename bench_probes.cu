@@ -48,6 +48,7 @@ struct Args {
     char *wr4[2];
     int n_rd2, n_rd4, n_wr4, n_wr2;
     unsigned long long rows;            // rows of 1024 elements per stream
+    int depth;                          // ring slots in use (2 .. kStages): depth - 1 copies in flight per warp
     int *err;
 };
 
@@ -92,9 +93,9 @@ __global__ void __launch_bounds__(kThreads, 2) stream_probe_kernel(const __grid_
                          :: "r"(ring_s + 2048u * islot), "l"(src), "r"(2048u), "r"(bar) : "memory");
         }
         if (++ipiece == npieces) { ipiece = 0; irow += stride; }
-        if (++islot == kStages) islot = 0;
+        if (++islot == a.depth) islot = 0;
     };
-    for (int p = 0; p < kStages - 1; ++p) issue();
+    for (int p = 0; p < a.depth - 1; ++p) issue();
 
     unsigned keep = 0;
     for (unsigned long long row = first; row < a.rows && !failed; row += stride) {
@@ -112,7 +113,7 @@ __global__ void __launch_bounds__(kThreads, 2) stream_probe_kernel(const __grid_
                 const uint4 x = *reinterpret_cast<const uint4 *>(slot + r * 512 + lane * 16);
                 acc[r].x ^= x.x; acc[r].y += x.y; acc[r].z ^= x.z; acc[r].w += x.w;
             }
-            if (++cslot == kStages) { cslot = 0; cphase ^= 1u; }
+            if (++cslot == a.depth) { cslot = 0; cphase ^= 1u; }
         }
         if (failed) break;
         for (int q = 0; q < a.n_wr4; ++q)
@@ -145,21 +146,23 @@ extern "C" {
 // of 4 bytes per element, `elems` elements each (rounded down to a multiple of 1024).  As in
 // the merge, the four-byte outputs are the four-byte inputs (in place) when both exist;
 // two-byte outputs overwrite the two-byte inputs when `push_in_place` is set, else they are
-// streams of their own.  ctas_per_sm sizes the persistent grid (2 is the merge's shape).
+// streams of their own.  ctas_per_sm sizes the persistent grid (2 is the merge's shape);
+// ring_depth is the number of ring slots a warp uses (2 or 3: one or two copies in flight, the
+// merge's two settings).
 // Returns -1 for bad arguments or a buffer that is too small, -2 for a CUDA error, -3 when a
 // bounded wait ran out on the device.
 double ddp_stream_probe(void *buffer, size_t buffer_bytes, int n_rd2, int n_rd4, int n_wr4, int n_wr2,
-                        size_t elems, int push_in_place, int ctas_per_sm, int reps, void *cuda_stream,
-                        double *best_ms)
+                        size_t elems, int push_in_place, int ctas_per_sm, int ring_depth, int reps,
+                        void *cuda_stream, double *best_ms)
 {
     if (!buffer || n_rd2 < 0 || n_rd2 > kMaxStreams || n_wr2 < 0 || n_wr2 > kMaxStreams || n_rd4 < 0 ||
-        n_rd4 > 2 || n_wr4 < 0 || n_wr4 > 2 || ctas_per_sm < 1 || reps < 1 || ((uintptr_t)buffer & 255u))
+        n_rd4 > 2 || n_wr4 < 0 || n_wr4 > 2 || ctas_per_sm < 1 || reps < 1 || ring_depth < 2 || ring_depth > kStages || ((uintptr_t)buffer & 255u))
         return -1.0;
     const unsigned long long rows = elems / 1024;
     if (rows == 0) return -1.0;
     Args a;
     std::memset(&a, 0, sizeof a);
-    a.n_rd2 = n_rd2; a.n_rd4 = n_rd4; a.n_wr4 = n_wr4; a.n_wr2 = n_wr2; a.rows = rows;
+    a.n_rd2 = n_rd2; a.n_rd4 = n_rd4; a.n_wr4 = n_wr4; a.n_wr2 = n_wr2; a.rows = rows; a.depth = ring_depth;
     char *base = static_cast<char *>(buffer);
     size_t used = 256;                                   // the error words live in the first 256 bytes
     a.err = reinterpret_cast<int *>(base);

@@ -101,9 +101,24 @@ constexpr int kEvictFirstMaxParticipants = 7;
 struct TmaRing {
     int islot = 0;           // next slot to fill
     int cslot = 0;           // next slot to consume
-    unsigned cphase = 0;     // parity of the phase the consumer waits for
+    unsigned phase_bits = 0; // bit d: parity of the phase the consumer waits for on slot d
     bool failed = false;     // a bounded wait gave up
 };
+
+// Slots of the ring a fragment uses (one fewer is in flight ahead of the consumer).  Measured on
+// B200 at 2 CTAs per SM.  bf16 copies: with one piece in flight per warp (32 KB per SM) the launch
+// is 3-7 % faster up to 7 participants, within 1.5 % either way from 8 to 16, and 2-4 % slower
+// from 18 on.  fp32 copies: one piece in flight is 1-4 % faster at every count up to 24.  The
+// passes of the three-launch radial-directional merge keep the full ring.  Every slot's barrier
+// has its own phase parity, so the depth may change from one fragment to the next (the ring is
+// drained in between).
+constexpr int kShallowMaxParticipantsBf16 = 7;
+template <bool BF16, int MODE>
+__device__ __forceinline__ int ring_depth(int s)
+{
+    if (kTmaStages < 3 || (MODE != kModeMerge && MODE != kModeMergeGram)) return kTmaStages;
+    return (!BF16 || s <= kShallowMaxParticipantsBf16) ? 2 : kTmaStages;
+}
 
 // All tiles of the current fragment that belong to this CTA (tile, tile+G, ...):
 // warp w merges super-row w of each of them.  Pieces per super-row, in order:
@@ -155,6 +170,8 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
     const unsigned row_stride = G * (unsigned)(kTileElems / kVec);
     const unsigned v_first = ((unsigned)(tile - tile_begin) * kWarps + (unsigned)warp) * kRowSteps;
 
+    const int nst = ring_depth<BF16, MODE>(s);
+    rs.islot = rs.cslot = 0;                   // drained: both may restart at slot 0 whatever the depth was
     const bool evict_first = MODE == kModeMerge && s <= kEvictFirstMaxParticipants;
     const unsigned long long policy = l2_policy_evict_first();
 
@@ -191,7 +208,7 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
             }
         }
         if (++ipiece == npieces) { ipiece = 0; iv0 += row_stride; }
-        if (++rs.islot == kTmaStages) rs.islot = 0;
+        if (++rs.islot == nst) rs.islot = 0;
         ++outstanding;
     };
     // ---- consumer: the next piece is in rs.cslot once its barrier flips -----------------
@@ -199,19 +216,20 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
         __syncwarp();                                              // the slot consumed last is free again
         if (!rs.failed) {
             issue();
-            const bool ok = mbar_wait_bounded(bar_s + 8u * rs.cslot, rs.cphase);
+            const bool ok = mbar_wait_bounded(bar_s + 8u * rs.cslot, (rs.phase_bits >> rs.cslot) & 1u);
             if (!__all_sync(0xffffffffu, ok)) rs.failed = true;    // the whole warp gives up together
         }
         return ring + rs.cslot * kTmaChunk;
     };
     auto release = [&]() {
         if (rs.failed) return;
-        if (++rs.cslot == kTmaStages) { rs.cslot = 0; rs.cphase ^= 1u; }
+        rs.phase_bits ^= 1u << rs.cslot;
+        if (++rs.cslot == nst) rs.cslot = 0;
         --outstanding;
     };
 
 #pragma unroll 1
-    for (int p = 0; p < kTmaStages - 1; ++p) issue();
+    for (int p = 0; p < nst - 1; ++p) issue();
 
     const float eta = c.eta, mu = c.mu;
     const bool heavy = (c.flags & DD_HEAVY_BALL) != 0;
@@ -403,8 +421,9 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
         // Give the copies still in flight a bounded chance to land before this
         // warp's slots can be reused or the CTA exits, and say what happened.
         for (int k = 0; k < outstanding; ++k) {
-            (void)mbar_wait_bounded(bar_s + 8u * rs.cslot, rs.cphase);
-            if (++rs.cslot == kTmaStages) { rs.cslot = 0; rs.cphase ^= 1u; }
+            (void)mbar_wait_bounded(bar_s + 8u * rs.cslot, (rs.phase_bits >> rs.cslot) & 1u);
+            rs.phase_bits ^= 1u << rs.cslot;
+            if (++rs.cslot == nst) rs.cslot = 0;
         }
         rs.islot = rs.cslot;
         if (lane == 0) sm.any_failed = 1;       // reported through the fragment's ticket (flush_fragment)
