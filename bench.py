@@ -321,6 +321,14 @@ def merge_ring_depth(s: int, learner_dtype: str) -> int:
     return 2 if learner_dtype != "bf16" or s <= 7 else 3
 
 
+def push_launch_shape(s: int, k: int) -> tuple[int, int]:
+    """(CTAs per SM, ring slots) of a merge of s bf16 copies fused with a push to k of them: the
+    launcher's own rule (one CTA per SM with the full ring when writes are 45 % or more of the
+    bytes moved, else two with a shallow ring)."""
+    wr, rd = 8 + 2 * k, 8 + 2 * s
+    return (1, 3) if wr >= 0.45 * (rd + wr) else (2, 2)
+
+
 def blend_ceiling(read_gbs: float, write_gbs: float, wshare: float) -> float:
     """Bandwidth of a stream with the given share of writes if reads and writes each ran at
     their own ceiling and did not disturb one another (an upper bound, not a measurement)."""
@@ -777,8 +785,9 @@ def config_row(dd, ctx, device, name, merge, args, ceilings, probes, traffic_tab
             row["e2e"] = e2e_leg(dd, ctx, merger, args, 1, pinned_cap_bytes=12 << 30, steps=2)
         if probes is not None and merge == "push" and w.learner_dtype == "bf16":
             s_all = row["participants"][0]
+            ctas, depth = push_launch_shape(s_all, s_all)
             row["pattern_probe_gbs"] = probes.run(rd2=s_all, rd4=2, wr4=2, wr2=s_all, push_in_place=True,
-                                                  ring_depth=merge_ring_depth(s_all, "bf16"), reps=5)
+                                                  ctas_per_sm=ctas, ring_depth=depth, reps=5)
             row["frac_of_pattern_probe"] = row["achieved_gbs"] / row["pattern_probe_gbs"]
         if probes is not None and merge == "avg":
             # the same access pattern with the arithmetic left out, at this workload's mean participant count

@@ -55,6 +55,7 @@ struct Common {
     int nq;                              // quantities per fragment in `partials`
     double *gram = nullptr;              // [P][kGramPairsMax] Gram matrices (lower triangle) of the two-launch RDA
     int pl_cap = 0;                      // participants the per-lane norm area holds (0: none)
+    int push_depth = 2;                  // ring slots a fragment with a fused push uses (3 when the launch runs 1 CTA per SM)
 };
 
 }  // namespace ddm

@@ -108,15 +108,17 @@ struct TmaRing {
 // Slots of the ring a fragment uses (one fewer is in flight ahead of the consumer).  Measured on
 // B200 at 2 CTAs per SM.  bf16 copies: with one piece in flight per warp (32 KB per SM) the launch
 // is 3-7 % faster up to 7 participants, within 1.5 % either way from 8 to 16, and 2-4 % slower
-// from 18 on.  fp32 copies: one piece in flight is 1-4 % faster at every count up to 24.  The
-// passes of the three-launch radial-directional merge keep the full ring.  Every slot's barrier
-// has its own phase parity, so the depth may change from one fragment to the next (the ring is
-// drained in between).
+// from 18 on.  fp32 copies: one piece in flight is 1-4 % faster at every count up to 24.  With a
+// fused push the host picks the depth together with the grid (push_ring_depth in the launcher).
+// The passes of the three-launch radial-directional merge keep the full ring.  Every slot's
+// barrier has its own phase parity, so the depth may change from one fragment to the next (the
+// ring is drained in between).
 constexpr int kShallowMaxParticipantsBf16 = 7;
 template <bool BF16, int MODE>
-__device__ __forceinline__ int ring_depth(int s)
+__device__ __forceinline__ int ring_depth(int s, int n_push, int push_depth)
 {
     if (kTmaStages < 3 || (MODE != kModeMerge && MODE != kModeMergeGram)) return kTmaStages;
+    if (n_push > 0) return push_depth;
     return (!BF16 || s <= kShallowMaxParticipantsBf16) ? 2 : kTmaStages;
 }
 
@@ -170,7 +172,7 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
     const unsigned row_stride = G * (unsigned)(kTileElems / kVec);
     const unsigned v_first = ((unsigned)(tile - tile_begin) * kWarps + (unsigned)warp) * kRowSteps;
 
-    const int nst = ring_depth<BF16, MODE>(s);
+    const int nst = ring_depth<BF16, MODE>(s, sm.n_push, c.push_depth);
     rs.islot = rs.cslot = 0;                   // drained: both may restart at slot 0 whatever the depth was
     const bool evict_first = MODE == kModeMerge && s <= kEvictFirstMaxParticipants;
     const unsigned long long policy = l2_policy_evict_first();

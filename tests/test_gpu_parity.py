@@ -178,6 +178,23 @@ def test_batched_large_fragments_element_by_element(dd, ctx):
                   flags=dd.DIAG_STATE | dd.DIAG_PER_LEARNER, merges=1)
 
 
+def test_batched_ring_depth_changes_between_fragments(dd, ctx):
+    # the staging ring runs shallower below 8 bf16 participants: fragments on either side of that
+    # count alternate, about 100 tiles each, so that most CTAs switch depth between their tiles
+    M = 12
+    counts = [3, 9, 7, 8, 12, 1, 10, 5]
+    sizes = [8192 * 100 + 17 * (p + 1) for p in range(len(counts))]
+    rng = np.random.default_rng(33)
+    tokens = rng.integers(1, 1000, size=(len(sizes), M))
+    masks = []
+    for c in counts:
+        chosen = rng.choice(M, size=c, replace=False)
+        masks.append(int(sum(1 << int(m) for m in chosen)))
+    recs = _batched_case(dd, ctx, sizes, M, "bf16", tokens, masks, 1, seed=34,
+                         flags=dd.DIAG_STATE | dd.DIAG_PER_LEARNER)
+    assert [r.n_part for r in recs] == counts
+
+
 def test_masked_learners_are_never_read(dd, ctx):
     # absent learners: NaN payloads, then null pointers
     run_case(dd, ctx, 20_001, 6, "bf16", [9, 9, 0, 9, 9, 9], 0b101011, 2, seed=8, poison_absent=True)

@@ -130,6 +130,74 @@ def test_batched_merge_and_push(dd, ctx):
                 assert torch.equal(frags[p]["learners"][m], before[p][m])
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_push_to_one_of_many(dd, ctx, dtype):
+    # few bytes written per byte read (9 merged, 1 pushed): the launch keeps the ordinary grid and a
+    # shallower ring than the write-heavy pushes above; several tiles per CTA and a ragged tail
+    n, M = 2 * 296 * 8192 + 4099, 10
+    tokens = [50 + 7 * m for m in range(M)]
+    mask, K, push = 0b1110111111, 4, 0b0001000000            # learner 6 is pushed to and not merged
+    theta, v, learners = synth.fragment_cpu(n, M, dtype, 611)
+    t_dev, v_dev = torch.from_numpy(theta).cuda(), torch.from_numpy(v).cuda()
+    l_dev = [to_torch_learner(a, "cuda") for a in learners]
+    before = [t.clone() for t in l_dev]
+    rec = dd.new_records(1)
+    ref = oracle.merge_fragment(theta, v, learners, tokens, mask, K, ETA, MU)
+    ctx.merge_fragment_push(t_dev, v_dev, l_dev, tokens, mask, K, ETA, MU, push, n=n,
+                            learner_dtype=dd.BF16 if dtype == "bf16" else dd.F32,
+                            flags=dd.DIAG_STATE, record=rec)
+    torch.cuda.synchronize()
+    got = dd.read_records(rec)[0]
+    assert (got.status, got.n_part, got.idx) == (ref.status, ref.n_part, ref.idx) and got.n_part == 9
+    assert floor_rel_err(t_dev.cpu().numpy(), theta) <= TOL_STATE
+    assert floor_rel_err(v_dev.cpu().numpy(), v) <= TOL_STATE
+    for m in range(M):
+        if (push >> m) & 1:
+            want = learners[m].copy()
+            oracle.apply_to_learner(want, theta, 0.0)
+            _check_pushed(l_dev[m], want, dtype)
+        else:
+            assert torch.equal(l_dev[m], before[m]), f"learner {m} was not to be written"
+
+
+def test_batched_push_mixes_pushed_and_plain_fragments(dd, ctx):
+    # one launch: fragments with and without a push, above and below 8 participants, about 60 tiles
+    # each (CTAs change ring depth between their tiles)
+    M = 10
+    counts = [9, 4, 10, 8, 2, 9]
+    pushes = [0, 0b0000000001, 0b1111111111, 0, 0b0000000110, 0b1000000000]
+    sizes = [8192 * 60 + 11 * (p + 1) for p in range(len(counts))]
+    rng = np.random.default_rng(41)
+    tokens = rng.integers(1, 500, size=(len(sizes), M))
+    masks = [(1 << c) - 1 for c in counts]
+    host, frags = [], []
+    for p, n in enumerate(sizes):
+        theta, v, learners = synth.fragment_cpu(n, M, "bf16", 900 + p)
+        host.append((theta, v, learners))
+        frags.append(dict(global_=torch.from_numpy(theta).cuda(), momentum=torch.from_numpy(v).cuda(),
+                          learners=[to_torch_learner(a, "cuda") for a in learners],
+                          tokens=[int(x) for x in tokens[p]], quorum_mask=masks[p], K=2, n=n))
+    before = [[t.clone() for t in f["learners"]] for f in frags]
+    recs = dd.new_records(len(sizes))
+    ctx.merge_fragments_batched_push(frags, pushes, M, dd.BF16, ETA, MU, flags=dd.DIAG_STATE, records=recs)
+    torch.cuda.synchronize()
+    got = dd.read_records(recs)
+    for p, n in enumerate(sizes):
+        theta, v, learners = host[p]
+        ref = oracle.merge_fragment(theta, v, learners, frags[p]["tokens"], masks[p], 2, ETA, MU)
+        assert (got[p].status, got[p].n_part, got[p].idx) == (ref.status, ref.n_part, ref.idx)
+        assert got[p].n_part == counts[p]
+        assert floor_rel_err(frags[p]["global_"].cpu().numpy(), theta) <= TOL_STATE
+        assert floor_rel_err(frags[p]["momentum"].cpu().numpy(), v) <= TOL_STATE
+        for m in range(M):
+            if (pushes[p] >> m) & 1:
+                want = learners[m].copy()
+                oracle.apply_to_learner(want, theta, 0.0)
+                _check_pushed(frags[p]["learners"][m], want, "bf16")
+            else:
+                assert torch.equal(frags[p]["learners"][m], before[p][m])
+
+
 def test_push_argument_validation(dd, ctx):
     n, M = 1024, 3
     theta, v, learners = synth.fragment_cpu(n, M, "bf16", 5)
