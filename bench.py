@@ -1034,6 +1034,19 @@ def e2e_leg(dd, ctx, merger, args, world, pinned_cap_bytes=None, steps=None):
                                                 flags=merger.flags)
 
     steps = max(1, steps)
+    # what the bus gives to a plain copy from page-locked memory in this run (256 MB, best of 3):
+    # the end-to-end rate can at most be this divided by the bytes that cross per element
+    probe_h = torch.empty(256 << 20, dtype=torch.uint8, pin_memory=True)
+    probe_d = torch.empty(256 << 20, dtype=torch.uint8, device=merger.device)
+    h2d_probe = 0.0
+    for _ in range(4):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        probe_d.copy_(probe_h, non_blocking=True)
+        torch.cuda.synchronize()
+        h2d_probe = max(h2d_probe, probe_h.numel() / (time.perf_counter() - t0) / 1e9)
+    del probe_h, probe_d
+
     one_step()                                           # warm-up: staging buffers, streams
     if world > 1:
         dist.barrier()
@@ -1053,6 +1066,8 @@ def e2e_leg(dd, ctx, merger, args, world, pinned_cap_bytes=None, steps=None):
            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
            "steps": steps, "elements_per_rank_step": n_total,
            "h2d_gbs": h2d * steps / dt_max / 1e9,
+           "h2d_copy_probe_gbs": h2d_probe,
+           "frac_of_h2d_copy_probe": h2d * steps / dt_max / 1e9 / h2d_probe,
            "path": f"{call}: pinned host buffers, chunked H2D -> kernel -> D2H pipeline, blocking"}
     if share < 1.0:
         out["note"] = f"leading {share:.3f} of every fragment (page-locked host memory is bounded)"

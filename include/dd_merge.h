@@ -332,9 +332,11 @@ int dd_merge_fragment_int4(dd_ctx *ctx, float *global, float *momentum,
  * The same update for a fragment whose operands live in HOST memory -- the
  * paper's syncer pulls each learner's fragment from that learner's host RAM and
  * keeps the global state off the accelerators (Section 4, system overview).
- * The fragment is cut into chunks of chunk_elems elements (0 = library default,
- * else a multiple of 8) that are pipelined through device staging buffers owned
- * by the context: host-to-device copies, the fused kernel and device-to-host
+ * The fragment is cut into chunks of chunk_elems elements (0 = library default:
+ * an eighth of the fragment in whole 2^20 elements, between 2^20 and 2^24; else a
+ * multiple of 8) that are pipelined through three sets of device staging buffers
+ * owned by the context (each holds one chunk of every operand: 8 + 2 + the
+ * participants' payload bytes per element): host-to-device copies, the fused kernel and device-to-host
  * copies of successive chunks overlap.  Only copies of participating learners
  * are transferred.
  *
