@@ -23,6 +23,19 @@ namespace ddm {
 // (dd_rda_gram.cuh), then the ordinary merge with weights derived from it (kModeMergeGram).
 enum : int { kModeMerge = 0, kModeNorms = 1, kModeDir = 2, kModeApply = 3, kModeMergeGram = 4 };
 
+// One 2 KB piece of a warp round as the producer lane needs it: where the piece of the row that
+// starts at step 0 begins, how many bytes one 8-element step of it takes, which steps of the row it
+// covers.  The piece of the row that starts at step v covers steps [first, first + cap) of that row
+// and begins at src0 + v * step_bytes.
+struct alignas(16) Piece {
+    const char *src0;
+    unsigned short step_bytes;           // 16 (bf16) or 32 (fp32)
+    unsigned short first;                // first step of the row in this piece (0 or 64)
+    unsigned short cap;                  // steps of the row in this piece (128 or 64)
+    unsigned short pad_;
+};
+constexpr int kMaxPieces = 2 * DD_MAX_LEARNERS + 4;
+
 struct Smem {
     const void *ptr[DD_MAX_LEARNERS];    // participant j's buffer (compacted)
     double wraw[DD_MAX_LEARNERS];        // raw weights, participant order
@@ -47,6 +60,7 @@ struct Smem {
     int any_failed;                      // a warp of this CTA gave up a bounded wait in (or before) this fragment
     double red[kWarps][kNumScalarDiag];  // per-warp ||Delta||^2, ||Theta'||^2, ||v'||^2 of this fragment
     double dm[kWarps][DD_MAX_LEARNERS];  // per-warp per-participant ||Theta-theta_m||^2
+    Piece piece[kMaxPieces];             // the pieces of one warp round, in the order they are consumed
 };
 
 // ---- memory access helpers ---------------------------------------------------

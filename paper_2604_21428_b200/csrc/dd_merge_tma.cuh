@@ -113,13 +113,52 @@ struct TmaRing {
 // The passes of the three-launch radial-directional merge keep the full ring.  Every slot's
 // barrier has its own phase parity, so the depth may change from one fragment to the next (the
 // ring is drained in between).
-constexpr int kShallowMaxParticipantsBf16 = 7;
+#ifndef DD_SHALLOW_MAX_BF16
+#define DD_SHALLOW_MAX_BF16 7
+#endif
+constexpr int kShallowMaxParticipantsBf16 = DD_SHALLOW_MAX_BF16;
 template <bool BF16, int MODE>
 __device__ __forceinline__ int ring_depth(int s, int n_push, int push_depth)
 {
     if (kTmaStages < 3 || (MODE != kModeMerge && MODE != kModeMergeGram)) return kTmaStages;
     if (n_push > 0) return push_depth;
+#ifdef DD_SHALLOW_EXCEPT
+    if (BF16 && s == DD_SHALLOW_EXCEPT) return kTmaStages;
+#endif
     return (!BF16 || s <= kShallowMaxParticipantsBf16) ? 2 : kTmaStages;
+}
+
+// Fills sm.piece for the current fragment (all threads of the CTA; a CTA barrier must follow).
+// MODE is the mode the fragment is processed in.  The order is the order of consumption:
+//   Theta[0:512) Theta[512:1024) | learner pieces (1 per bf16 copy, 2 per fp32 copy) | v[0:512) v[512:1024)
+template <bool BF16, int MODE>
+__device__ __forceinline__ void build_piece_table(Smem &sm)
+{
+    constexpr int LB = BF16 ? 1 : 2;
+    constexpr bool kHasV = MODE == kModeMerge || MODE == kModeApply;
+    const int nmid = MODE == kModeApply ? 2 : sm.n_part * LB;
+    const int npieces = 2 + nmid + (kHasV ? 2 : 0);
+    for (int i = threadIdx.x; i < npieces; i += kThreads) {
+        Piece pc;
+        pc.pad_ = 0;
+        if (BF16 && MODE != kModeApply && i >= 2 && i < 2 + nmid) {
+            pc.src0 = reinterpret_cast<const char *>(sm.ptr[i - 2]);
+            pc.step_bytes = 16;
+            pc.first = 0;
+            pc.cap = (unsigned short)(kSuperRow / kVec);
+        } else {
+            // float32 operand (Theta, fp32 learner copy, stored direction, v): two halves of 64 steps
+            const int q = i < 2 ? i : (i < 2 + nmid ? i - 2 : i - 2 - nmid);
+            const void *base = i < 2 ? (const void *)sm.theta
+                             : i >= 2 + nmid ? (const void *)sm.mom
+                             : MODE == kModeApply ? (const void *)sm.scratch : sm.ptr[q >> 1];
+            pc.first = (unsigned short)(64 * (q & 1));
+            pc.src0 = reinterpret_cast<const char *>(base) + 32u * pc.first;
+            pc.step_bytes = 32;
+            pc.cap = 64;
+        }
+        sm.piece[i] = pc;
+    }
 }
 
 // All tiles of the current fragment that belong to this CTA (tile, tile+G, ...):
@@ -184,23 +223,11 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
     auto issue = [&]() {
         if (rs.failed || iv0 >= nfull) return;
         if (lane == 0) {
+            const Piece pc = sm.piece[ipiece];
             const unsigned cnt = min(kRowSteps, nfull - iv0);      // steps in this super-row
-            const char *src;
-            unsigned bytes;
-            if (BF16 && MODE != kModeApply && ipiece >= 2 && ipiece < 2 + nmid) {
-                src = reinterpret_cast<const char *>(sm.ptr[ipiece - 2]) + 16ull * iv0;
-                bytes = cnt * 16u;
-            } else {
-                // float32 operand (Theta, fp32 learner copy, stored direction, v): two halves of 64 steps
-                const int q = ipiece < 2 ? ipiece : (ipiece < 2 + nmid ? ipiece - 2 : ipiece - 2 - nmid);
-                const void *base = ipiece < 2 ? (const void *)theta
-                                 : ipiece >= 2 + nmid ? (const void *)mom
-                                 : MODE == kModeApply ? (const void *)sm.scratch : sm.ptr[q >> 1];
-                const unsigned first = 64u * (unsigned)(q & 1);
-                const unsigned nv = cnt > first ? min(64u, cnt - first) : 0u;
-                src = reinterpret_cast<const char *>(base) + 32ull * (iv0 + first);
-                bytes = nv * 32u;
-            }
+            const unsigned have = cnt > pc.first ? min(cnt - pc.first, (unsigned)pc.cap) : 0u;
+            const unsigned bytes = have * pc.step_bytes;
+            const char *src = pc.src0 + (unsigned long long)iv0 * pc.step_bytes;
             // (test hook) announce 16 bytes that no copy will deliver: the wait must expire
             const unsigned phantom = expire_hook && iv0 == v_first && ipiece == 0 ? 16u : 0u;
             mbar_arrive_expect_tx(bar_s + 8u * rs.islot, bytes + phantom);
@@ -472,6 +499,9 @@ __device__ __forceinline__ void merge_body_tma(const DevFrag *frags, const Commo
                            (MODE == kModeApply && sm.kind == DD_MERGE_AVG);
         const bool worked_on = sm.status == DD_STATUS_OK && (plain || sm.kind == DD_MERGE_RDA);
         if (worked_on) {
+            if (plain) build_piece_table<BF16, kModeMerge>(sm);
+            else build_piece_table<BF16, MODE>(sm);
+            __syncthreads();
             // A warp whose ring failed in an earlier fragment skips its rows of this one too: the
             // fragment is incomplete and must say so.
             if (rs.failed && lane == 0 &&
