@@ -16,7 +16,10 @@ namespace ddm {
 
 constexpr int kInt4Block = DD_INT4_BLOCK;     // elements per scale
 constexpr int kQuantUnroll = 4;               // blocks a warp of the quantiser loads before it reduces
-constexpr int kInt4Batch = 8;                 // participants whose loads a thread keeps in flight
+#ifndef DD_INT4_BATCH
+#define DD_INT4_BATCH 8
+#endif
+constexpr int kInt4Batch = DD_INT4_BATCH;                 // participants whose loads a thread keeps in flight
 
 // ---- learner side: quantise Theta - theta ---------------------------------------------
 //
