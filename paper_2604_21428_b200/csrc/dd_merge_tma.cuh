@@ -109,10 +109,11 @@ struct TmaRing {
 // B200 at 2 CTAs per SM.  bf16 copies: with one piece in flight per warp (32 KB per SM) the launch
 // is 3-7 % faster up to 7 participants, within 1.5 % either way from 8 to 16, and 2-4 % slower
 // from 18 on.  fp32 copies: one piece in flight is 1-4 % faster at every count up to 24.  With a
-// fused push the host picks the depth together with the grid (push_ring_depth in the launcher).
-// The passes of the three-launch radial-directional merge keep the full ring.  Every slot's
-// barrier has its own phase parity, so the depth may change from one fragment to the next (the
-// ring is drained in between).
+// fused push the host picks the depth together with the grid (push_shape in the launcher).  The
+// norms and direction passes of the three-launch radial-directional merge follow the same rule
+// (-2 % on three launches at 6 participants); its apply pass, 40 % writes, runs shallow.  Every
+// slot's barrier has its own phase parity, so the depth may change from one fragment to the next
+// (the ring is drained in between).
 #ifndef DD_SHALLOW_MAX_BF16
 #define DD_SHALLOW_MAX_BF16 7
 #endif
@@ -120,11 +121,9 @@ constexpr int kShallowMaxParticipantsBf16 = DD_SHALLOW_MAX_BF16;
 template <bool BF16, int MODE>
 __device__ __forceinline__ int ring_depth(int s, int n_push, int push_depth)
 {
-    if (kTmaStages < 3 || (MODE != kModeMerge && MODE != kModeMergeGram)) return kTmaStages;
+    if (kTmaStages < 3) return kTmaStages;
+    if (MODE == kModeApply) return 2;
     if (n_push > 0) return push_depth;
-#ifdef DD_SHALLOW_EXCEPT
-    if (BF16 && s == DD_SHALLOW_EXCEPT) return kTmaStages;
-#endif
     return (!BF16 || s <= kShallowMaxParticipantsBf16) ? 2 : kTmaStages;
 }
 
