@@ -789,6 +789,27 @@ def config_row(dd, ctx, device, name, merge, args, ceilings, probes, traffic_tab
             row["pattern_probe_gbs"] = probes.run(rd2=s_all, rd4=2, wr4=2, wr2=s_all, push_in_place=True,
                                                   ctas_per_sm=ctas, ring_depth=depth, reps=5)
             row["frac_of_pattern_probe"] = row["achieved_gbs"] / row["pattern_probe_gbs"]
+        if probes is not None and merge == "rda" and w.learner_dtype == "bf16":
+            # one probe per launch of the merge (the same streams, nothing computed), added up
+            s_mean = max(1, round(sum(row["participants"]) / w.P))
+            depth = merge_ring_depth(s_mean, "bf16")
+            if merger.launches_per_step == 2:
+                legs = [("gram", 2 * s_mean + 4, dict(rd2=s_mean, rd4=1)),
+                        ("merge", 2 * s_mean + 16, dict(rd2=s_mean, rd4=2, wr4=2, ring_depth=depth))]
+            else:
+                legs = [("norms", 2 * s_mean + 4, dict(rd2=s_mean, rd4=1, ring_depth=depth)),
+                        ("direction", 2 * s_mean + 8, dict(rd2=s_mean, rd4=1, wr4=1, ring_depth=depth)),
+                        # u, Theta, v read (u stands in as two two-byte streams), Theta', v' written
+                        ("apply", 20, dict(rd2=2, rd4=2, wr4=2, ring_depth=2))]
+            t_total, b_total, per_leg = 0.0, 0.0, {}
+            for leg, bpp, shape in legs:
+                gbs = probes.run(reps=5, **shape)
+                per_leg[leg] = gbs
+                t_total += bpp / gbs
+                b_total += bpp
+            row["pattern_probe_gbs"] = b_total / t_total
+            row["pattern_probe_per_launch_gbs"] = per_leg
+            row["frac_of_pattern_probe"] = row["achieved_gbs"] / row["pattern_probe_gbs"]
         if probes is not None and merge == "avg":
             # the same access pattern with the arithmetic left out, at this workload's mean participant count
             s_mean = max(1, round(sum(row["participants"]) / w.P))
