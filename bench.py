@@ -800,7 +800,8 @@ def config_row(dd, ctx, device, name, merge, args, ceilings, probes, traffic_tab
                 legs = [("norms", 2 * s_mean + 4, dict(rd2=s_mean, rd4=1, ring_depth=depth)),
                         ("direction", 2 * s_mean + 8, dict(rd2=s_mean, rd4=1, wr4=1, ring_depth=depth)),
                         # u, Theta, v read (u stands in as two two-byte streams), Theta', v' written
-                        ("apply", 20, dict(rd2=2, rd4=2, wr4=2, ring_depth=2))]
+                        # (one CTA per SM with the full ring: the launcher's shape for this pass)
+                        ("apply", 20, dict(rd2=2, rd4=2, wr4=2, ctas_per_sm=1, ring_depth=3))]
             t_total, b_total, per_leg = 0.0, 0.0, {}
             for leg, bpp, shape in legs:
                 gbs = probes.run(reps=5, **shape)

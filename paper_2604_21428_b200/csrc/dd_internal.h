@@ -56,6 +56,7 @@ struct Common {
     double *gram = nullptr;              // [P][kGramPairsMax] Gram matrices (lower triangle) of the two-launch RDA
     int pl_cap = 0;                      // participants the per-lane norm area holds (0: none)
     int push_depth = 2;                  // ring slots a fragment with a fused push uses (3 when the launch runs 1 CTA per SM)
+    int apply_depth = 2;                 // ring slots of the radial-directional apply pass (3 when it runs 1 CTA per SM)
 };
 
 }  // namespace ddm

@@ -550,14 +550,19 @@ namespace ddm {
 
 template <bool BF16>
 static cudaError_t launch_rda_passes(const DevFrag *dev_frags, const Common &c, unsigned grid,
-                                     cudaStream_t stream, int only_pass)
+                                     unsigned apply_grid, cudaStream_t stream, int only_pass)
 {
     if (only_pass < 0 || only_pass == DD_RDA_PASS_NORMS)
         rda_pass_kernel<BF16, kModeNorms><<<grid, kThreads, kTmaRingBytes + pl_area_bytes(c.pl_cap), stream>>>(dev_frags, c);
     if (only_pass < 0 || only_pass == DD_RDA_PASS_DIRECTION)
         rda_pass_kernel<BF16, kModeDir><<<grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
-    if (only_pass < 0 || only_pass == DD_RDA_PASS_APPLY)
-        rda_pass_kernel<BF16, kModeApply><<<grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, c);
+    if (only_pass < 0 || only_pass == DD_RDA_PASS_APPLY) {
+        // The apply pass reads 12 bytes per element and writes 8: with so large a share of writes
+        // one CTA per SM with the full ring is the faster shape (as for a write-heavy fused push).
+        Common ca = c;
+        if (apply_grid != grid) ca.apply_depth = kTmaStages;
+        rda_pass_kernel<BF16, kModeApply><<<apply_grid, kThreads, kTmaRingBytes, stream>>>(dev_frags, ca);
+    }
     return cudaGetLastError();
 }
 
@@ -700,8 +705,14 @@ static int rda_batched_impl(dd_ctx *ctx, const dd_fragment_desc *descs, const ui
         }
         e = cudaGetLastError();
     } else {
-        e = bf16 ? launch_rda_passes<true>(slot.dev, c, (unsigned)g, stream, only_pass)
-                 : launch_rda_passes<false>(slot.dev, c, (unsigned)g, stream, only_pass);
+        // Fragments of kind DD_MERGE_AVG get the ordinary merge in the last launch, which wants the
+        // ordinary grid: the narrower one is taken only when every fragment is radial-directional.
+        bool all_rda = true;
+        for (int p = 0; p < P; ++p) all_rda = all_rda && slot.host[p].kind == DD_MERGE_RDA;
+        unsigned long long ga = g;
+        if (all_rda && (unsigned long long)ctx->sm_count < ga) ga = (unsigned long long)ctx->sm_count;
+        e = bf16 ? launch_rda_passes<true>(slot.dev, c, (unsigned)g, (unsigned)ga, stream, only_pass)
+                 : launch_rda_passes<false>(slot.dev, c, (unsigned)g, (unsigned)ga, stream, only_pass);
     }
     if (e != cudaSuccess) return cuda_fail(ctx, e, "radial-directional merge launch");
     DD_CUDA(ctx, cudaEventRecord(slot.done, stream));

@@ -111,19 +111,20 @@ struct TmaRing {
 // from 18 on.  fp32 copies: one piece in flight is 1-4 % faster at every count up to 24.  With a
 // fused push the host picks the depth together with the grid (push_shape in the launcher).  The
 // norms and direction passes of the three-launch radial-directional merge follow the same rule
-// (-2 % on three launches at 6 participants); its apply pass, 40 % writes, runs shallow.  Every
-// slot's barrier has its own phase parity, so the depth may change from one fragment to the next
-// (the ring is drained in between).
+// (-2 % on three launches at 6 participants); its apply pass, 40 % writes, runs shallow at two
+// CTAs per SM and with the full ring when the host launches it with one (a probe of its pattern:
+// 6.69 against 6.33 TB/s).  Every slot's barrier has its own phase parity, so the depth may change
+// from one fragment to the next (the ring is drained in between).
 #ifndef DD_SHALLOW_MAX_BF16
 #define DD_SHALLOW_MAX_BF16 7
 #endif
 constexpr int kShallowMaxParticipantsBf16 = DD_SHALLOW_MAX_BF16;
 template <bool BF16, int MODE>
-__device__ __forceinline__ int ring_depth(int s, int n_push, int push_depth)
+__device__ __forceinline__ int ring_depth(int s, int n_push, const Common &c)
 {
     if (kTmaStages < 3) return kTmaStages;
-    if (MODE == kModeApply) return 2;
-    if (n_push > 0) return push_depth;
+    if (MODE == kModeApply) return c.apply_depth;
+    if (n_push > 0) return c.push_depth;
     return (!BF16 || s <= kShallowMaxParticipantsBf16) ? 2 : kTmaStages;
 }
 
@@ -210,7 +211,7 @@ __device__ __forceinline__ void process_fragment_tma(Smem &sm, const Common &c,
     const unsigned row_stride = G * (unsigned)(kTileElems / kVec);
     const unsigned v_first = ((unsigned)(tile - tile_begin) * kWarps + (unsigned)warp) * kRowSteps;
 
-    const int nst = ring_depth<BF16, MODE>(s, sm.n_push, c.push_depth);
+    const int nst = ring_depth<BF16, MODE>(s, sm.n_push, c);
     rs.islot = rs.cslot = 0;                   // drained: both may restart at slot 0 whatever the depth was
     const bool evict_first = MODE == kModeMerge && s <= kEvictFirstMaxParticipants;
     const unsigned long long policy = l2_policy_evict_first();
