@@ -395,7 +395,8 @@ def test_argument_validation(dd, ctx):
     torch.cuda.synchronize()
 
 
-@pytest.mark.parametrize("n,chunk", [(100_003, 8192), (50_000, 0), (7, 8), (0, 0), (65_536, 16_384)])
+# (2_500_003, 0): the default chunk is 2^20 elements there, so three chunks with a ragged last one
+@pytest.mark.parametrize("n,chunk", [(100_003, 8192), (50_000, 0), (7, 8), (0, 0), (65_536, 16_384), (2_500_003, 0)])
 def test_host_buffers_entry_point(dd, ctx, n, chunk):
     # operands in (pinned) host memory, pipelined through the GPU in chunks
     M = 6
