@@ -99,12 +99,20 @@ static cudaError_t occupancy(int *blocks)
 template <bool BF16>
 static cudaError_t gram_occupancy(int *blocks)
 {
-    cudaError_t e = cudaFuncSetAttribute(rda_gram_kernel<BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)kGramRingBytes);
-    int b = 0;
-    if (e == cudaSuccess)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, rda_gram_kernel<BF16>, kGramThreads, kGramRingBytes);
-    *blocks = b > 2 ? 2 : b;
+    // both instances (with and without the packed consumer) get the shared-memory attribute; the
+    // grid is sized for the one that fits fewer CTAs
+    int b = 2;
+    cudaError_t e = cudaSuccess;
+    auto one = [&](auto kernel) {
+        if (e != cudaSuccess) return;
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGramRingBytes);
+        int x = 0;
+        if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&x, kernel, kGramThreads, kGramRingBytes);
+        if (x < b) b = x;
+    };
+    one(rda_gram_kernel<BF16, true>);
+    one(rda_gram_kernel<BF16, false>);
+    *blocks = b;
     return e;
 }
 
@@ -696,11 +704,17 @@ static int rda_batched_impl(dd_ctx *ctx, const dd_fragment_desc *descs, const ui
                                  cudaMemcpyHostToDevice, stream));
     cudaError_t e;
     if (use_gram) {
+        int most = 0;                         // participants of the largest radial-directional fragment
+        for (int p = 0; p < P; ++p)
+            if (slot.host[p].kind == DD_MERGE_RDA && slot.host[p].n_part_host > most) most = slot.host[p].n_part_host;
+        const bool packed = most <= kGramPackedMaxPart;
         if (bf16) {
-            rda_gram_kernel<true><<<(unsigned)gg, kGramThreads, kGramRingBytes, stream>>>(slot.dev, c);
+            if (packed) rda_gram_kernel<true, true><<<(unsigned)gg, kGramThreads, kGramRingBytes, stream>>>(slot.dev, c);
+            else rda_gram_kernel<true, false><<<(unsigned)gg, kGramThreads, kGramRingBytes, stream>>>(slot.dev, c);
             rda_gram_merge_kernel<true><<<(unsigned)g, kThreads, kTmaRingBytes, stream>>>(slot.dev, c);
         } else {
-            rda_gram_kernel<false><<<(unsigned)gg, kGramThreads, kGramRingBytes, stream>>>(slot.dev, c);
+            if (packed) rda_gram_kernel<false, true><<<(unsigned)gg, kGramThreads, kGramRingBytes, stream>>>(slot.dev, c);
+            else rda_gram_kernel<false, false><<<(unsigned)gg, kGramThreads, kGramRingBytes, stream>>>(slot.dev, c);
             rda_gram_merge_kernel<false><<<(unsigned)g, kThreads, kTmaRingBytes, stream>>>(slot.dev, c);
         }
         e = cudaGetLastError();
