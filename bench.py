@@ -315,18 +315,17 @@ def measure_ceilings(device):
 
 
 def merge_ring_depth(s: int, learner_dtype: str) -> int:
-    """Ring slots the fused merge uses per warp at s participants (the kernel's own rule, so that a
-    pattern probe moves data exactly as the kernel does): one copy in flight for fp32 copies and for
-    up to 7 bf16 copies, two above."""
-    return 2 if learner_dtype != "bf16" or s <= 7 else 3
+    """Ring slots the fused merge uses per warp at s participants, asked of the library
+    (``dd_launch_shape``), so that a pattern probe moves data exactly as the kernel does."""
+    from paper_2604_21428_b200 import ddmerge as dd
+    return dd.launch_shape(dd.BF16 if learner_dtype == "bf16" else dd.F32, s)[1]
 
 
 def push_launch_shape(s: int, k: int) -> tuple[int, int]:
-    """(CTAs per SM, ring slots) of a merge of s bf16 copies fused with a push to k of them: the
-    launcher's own rule (one CTA per SM with the full ring when writes are 45 % or more of the
-    bytes moved, else two with a shallow ring)."""
-    wr, rd = 8 + 2 * k, 8 + 2 * s
-    return (1, 3) if wr >= 0.45 * (rd + wr) else (2, 2)
+    """(CTAs per SM, ring slots) of a merge of s bf16 copies fused with a push to k of them, asked
+    of the library (``dd_launch_shape``)."""
+    from paper_2604_21428_b200 import ddmerge as dd
+    return dd.launch_shape(dd.BF16, s, k)
 
 
 def blend_ceiling(read_gbs: float, write_gbs: float, wshare: float) -> float:

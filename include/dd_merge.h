@@ -510,6 +510,19 @@ const char *dd_last_cuda_error(const dd_ctx *ctx);
 /* Launch geometry chosen by the context (for reporting): CTAs, threads per CTA, elements per tile. */
 int dd_launch_geometry(const dd_ctx *ctx, dd_dtype learner_dtype, int *grid, int *block, int *tile);
 
+/*
+ * How a merge of `participants` copies of learner_dtype, fused with a push to `pushed` copies
+ * (0 = plain merge) and with or without the bf16 copy of Theta', is launched on a B200: persistent
+ * CTAs per SM (2, or 1 for a push whose writes are 45 % or more of the bytes moved) and ring slots
+ * each warp uses (2 = one 2 KB copy in flight ahead of the consumer, 3 = two).  Pure host function
+ * (no context, no GPU); it reports the rule the launcher and the kernel apply, for benchmarks that
+ * want to reproduce the kernel's data movement.  The paper has no counterpart.
+ * Returns DD_OK or DD_ERR_INVALID_ARG (dtype, participants outside 1..DD_MAX_LEARNERS, pushed
+ * outside 0..DD_MAX_LEARNERS).
+ */
+int dd_launch_shape(dd_dtype learner_dtype, int participants, int pushed, int with_out_bf16,
+                    int *ctas_per_sm, int *ring_slots);
+
 #ifdef __cplusplus
 }
 #endif

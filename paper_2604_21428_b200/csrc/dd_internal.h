@@ -20,6 +20,28 @@ constexpr unsigned long long kMaxFragmentElems = 1ull << 34;   // 8-element step
 #define DD_RDA_GRAM_MAX_PARTICIPANTS 8
 constexpr int kGramPairsMax = DD_RDA_GRAM_MAX_PARTICIPANTS * (DD_RDA_GRAM_MAX_PARTICIPANTS + 1) / 2;
 
+// Ring slots a warp uses for a plain merge (one fewer copy is in flight ahead of the consumer):
+// the shallow ring for fp32 copies and for up to kShallowMaxParticipantsBf16 bf16 copies, the full
+// one above.  One definition for the kernel and for the host's dd_launch_shape.
+#ifndef DD_TMA_STAGES
+#define DD_TMA_STAGES 3
+#endif
+#ifndef DD_SHALLOW_MAX_BF16
+#define DD_SHALLOW_MAX_BF16 7
+#endif
+constexpr int kTmaStages = DD_TMA_STAGES;
+constexpr int kShallowMaxParticipantsBf16 = DD_SHALLOW_MAX_BF16;
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+constexpr int merge_ring_slots(bool bf16, int participants)
+{
+    return kTmaStages < 3 ? kTmaStages : ((!bf16 || participants <= kShallowMaxParticipantsBf16) ? 2 : kTmaStages);
+}
+// A merge with a fused push: from this share of writes in the bytes moved on, one CTA per SM with
+// the full ring; below, the ordinary grid with the shallow ring.
+constexpr double kPushHeavyWriteShare = 0.45;
+
 // One fragment as the kernel sees it.  Raw counters, mask and pointers travel to
 // the device; participation and weights are derived there.
 struct alignas(16) DevFrag {

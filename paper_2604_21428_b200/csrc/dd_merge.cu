@@ -360,7 +360,7 @@ struct PushShape {
 };
 static PushShape push_shape(double read_bytes, double write_bytes)
 {
-    const bool heavy = write_bytes >= 0.45 * (read_bytes + write_bytes);
+    const bool heavy = write_bytes >= kPushHeavyWriteShare * (read_bytes + write_bytes);
     return PushShape{heavy, heavy ? kTmaStages : 2};
 }
 static void add_fragment_bytes(const DevFrag &f, size_t esz, double &rd, double &wr)
@@ -800,6 +800,25 @@ extern "C" int dd_merge_fragment_rda(dd_ctx *ctx, float *global, float *momentum
 extern "C" const char *dd_last_cuda_error(const dd_ctx *ctx)
 {
     return ctx ? ctx->cuda_err : "";
+}
+
+extern "C" int dd_launch_shape(dd_dtype learner_dtype, int participants, int pushed, int with_out_bf16,
+                               int *ctas_per_sm, int *ring_slots)
+{
+    if ((learner_dtype != DD_F32 && learner_dtype != DD_BF16) || participants < 1 ||
+        participants > DD_MAX_LEARNERS || pushed < 0 || pushed > DD_MAX_LEARNERS)
+        return DD_ERR_INVALID_ARG;
+    const bool bf16 = learner_dtype == DD_BF16;
+    int ctas = 2, slots = merge_ring_slots(bf16, participants);
+    if (pushed > 0) {
+        const double esz = bf16 ? 2.0 : 4.0;
+        const PushShape shape = push_shape(8.0 + esz * participants, 8.0 + (with_out_bf16 ? 2.0 : 0.0) + esz * pushed);
+        ctas = shape.one_cta_per_sm ? 1 : 2;
+        slots = shape.ring_depth;
+    }
+    if (ctas_per_sm) *ctas_per_sm = ctas;
+    if (ring_slots) *ring_slots = slots;
+    return DD_OK;
 }
 
 extern "C" int dd_launch_geometry(const dd_ctx *ctx, dd_dtype learner_dtype, int *grid, int *block,

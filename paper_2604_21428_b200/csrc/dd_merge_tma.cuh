@@ -17,13 +17,9 @@
 
 #include "dd_merge_kernel.cuh"
 
-#ifndef DD_TMA_STAGES
-#define DD_TMA_STAGES 3
-#endif
 
 namespace ddm {
 
-constexpr int kTmaStages = DD_TMA_STAGES;
 constexpr int kTmaChunk = 2048;                           // bytes per slot / per bulk copy
 constexpr int kSuperRow = 1024;                           // elements a warp merges per round (4 steps per lane)
 constexpr size_t kTmaRingBytes = (size_t)kWarps * kTmaStages * kTmaChunk;
@@ -115,17 +111,13 @@ struct TmaRing {
 // CTAs per SM and with the full ring when the host launches it with one (a probe of its pattern:
 // 6.69 against 6.33 TB/s).  Every slot's barrier has its own phase parity, so the depth may change
 // from one fragment to the next (the ring is drained in between).
-#ifndef DD_SHALLOW_MAX_BF16
-#define DD_SHALLOW_MAX_BF16 7
-#endif
-constexpr int kShallowMaxParticipantsBf16 = DD_SHALLOW_MAX_BF16;
 template <bool BF16, int MODE>
 __device__ __forceinline__ int ring_depth(int s, int n_push, const Common &c)
 {
     if (kTmaStages < 3) return kTmaStages;
     if (MODE == kModeApply) return c.apply_depth;
     if (n_push > 0) return c.push_depth;
-    return (!BF16 || s <= kShallowMaxParticipantsBf16) ? 2 : kTmaStages;
+    return merge_ring_slots(BF16, s);
 }
 
 // Fills sm.piece for the current fragment (all threads of the CTA; a CTA barrier must follow).

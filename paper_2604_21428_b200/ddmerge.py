@@ -34,7 +34,7 @@ EXPORTS = (
     "dd_quantize_outer_gradient_int4", "dd_merge_fragment_int4",
     "dd_broadcast_fragment", "dd_grace_controller_init", "dd_grace_controller_observe",
     "dd_grace_controller_window", "dd_plan_fragments", "dd_select_quorum", "dd_grace_window", "dd_status_string", "dd_last_cuda_error",
-    "dd_launch_geometry",
+    "dd_launch_geometry", "dd_launch_shape",
 )
 
 
@@ -174,6 +174,8 @@ def _load() -> ctypes.CDLL:
     lib.dd_last_cuda_error.argtypes = [vp]
     lib.dd_launch_geometry.restype = ctypes.c_int
     lib.dd_launch_geometry.argtypes = [vp, ctypes.c_int] + [ctypes.POINTER(ctypes.c_int)] * 3
+    lib.dd_launch_shape.restype = ctypes.c_int
+    lib.dd_launch_shape.argtypes = [ctypes.c_int] * 4 + [ctypes.POINTER(ctypes.c_int)] * 2
     return lib
 
 
@@ -572,6 +574,16 @@ def _infer_dtype(learners) -> int:
         if t is not None and not isinstance(t, int):
             return BF16 if t.dtype == torch.bfloat16 else F32
     return BF16
+
+
+def launch_shape(learner_dtype: int, participants: int, pushed: int = 0, with_out_bf16: bool = False):
+    """``dd_launch_shape``: (persistent CTAs per SM, ring slots per warp) of such a merge."""
+    ctas, slots = ctypes.c_int(0), ctypes.c_int(0)
+    rc = lib.dd_launch_shape(int(learner_dtype), int(participants), int(pushed), int(bool(with_out_bf16)),
+                             ctypes.byref(ctas), ctypes.byref(slots))
+    if rc != OK:
+        raise DDMergeError(rc)
+    return ctas.value, slots.value
 
 
 def select_quorum(arrival_s, K: int, grace_s: float):

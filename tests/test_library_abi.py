@@ -110,6 +110,24 @@ def test_grace_controller_matches_oracle(dd):
         dd.GraceController(2.0, 0.5, 0.5).observe(-1.0, 0.0, 0.0)
 
 
+def test_launch_shape_reports_the_launchers_rule(dd):
+    """``dd_launch_shape`` is a pure host function: the shallow ring up to 7 bf16 participants and
+    for fp32 copies, the full one above; a push whose writes are 45 % or more of the bytes moved
+    runs one CTA per SM with the full ring, a lighter push two with the shallow ring."""
+    assert [dd.launch_shape(dd.BF16, s) for s in (1, 7, 8, 64)] == [(2, 2), (2, 2), (2, 3), (2, 3)]
+    assert [dd.launch_shape(dd.F32, s) for s in (1, 8, 24)] == [(2, 2)] * 3
+    # writes / bytes moved: (8 + 2k) / (2s + 16 + 2k)
+    for s, k in [(4, 8), (8, 8), (24, 24), (2, 2), (8, 4), (24, 12), (8, 1), (24, 1)]:
+        heavy = (8 + 2 * k) >= 0.45 * (2 * s + 16 + 2 * k)
+        assert dd.launch_shape(dd.BF16, s, k) == ((1, 3) if heavy else (2, 2)), (s, k)
+    # the bf16 copy of Theta' counts as written bytes: 9 participants, 6 pushed is heavy only with it
+    assert dd.launch_shape(dd.BF16, 9, 6) == (2, 2) and dd.launch_shape(dd.BF16, 9, 6, True) == (1, 3)
+    for bad in [(dd.BF16, 0), (dd.BF16, 65), (dd.BF16, 4, -1), (dd.BF16, 4, 65), (7, 4)]:
+        with pytest.raises(dd.DDMergeError) as e:
+            dd.launch_shape(*bad)
+        assert e.value.rc == dd.ERR_INVALID_ARG
+
+
 def test_header_is_plain_c_and_links(dd, tmp_path):
     import subprocess
     pkg = os.path.join(ROOT, "paper_2604_21428_b200")
