@@ -236,6 +236,46 @@ def test_rda_two_launch_form_exactly_eight_and_nine_participants(dd, ctx):
     assert rec.n_part == 1
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_rda_two_launch_form_around_the_packed_limit(dd, ctx, dtype):
+    # up to 6 participants the Gram launch keeps packed even / odd sums, at 7 and 8 scalar ones (another
+    # kernel instance): both sides of the limit, several sub-tiles per thread and a ragged end
+    tokens = [10 * (m + 1) for m in range(10)]
+    for s, seed in ((5, 51), (6, 52), (7, 53)):
+        rec = _case(dd, ctx, 3 * 8192 + 1029, 10, dtype, tokens, (1 << s) - 1, 2, seed=seed, merges=1)
+        assert rec.n_part == s
+
+
+def test_rda_two_launch_batch_mixing_participant_counts(dd, ctx):
+    # one launch holds fragments on both sides of the packed limit: the launcher takes the instance with
+    # the scalar sums for all of them; a second batch of small counts only takes the packed one
+    rng = np.random.default_rng(61)
+    M, K = 8, 1
+    for counts in ([3, 8, 6, 7, 1], [2, 6, 4, 5]):
+        sizes = [8192 * 5 + 7 * (p + 1) for p in range(len(counts))]
+        tokens = rng.integers(1, 1000, size=(len(sizes), M))
+        masks = [(1 << c) - 1 for c in counts]
+        host, dev = [], []
+        for p, n in enumerate(sizes):
+            theta, v, learners = synth.fragment_cpu(n, M, "bf16", 700 + 10 * len(counts) + p)
+            host.append((theta, v, learners))
+            dev.append(dict(global_=torch.from_numpy(theta).cuda(), momentum=torch.from_numpy(v).cuda(),
+                            learners=[to_torch_learner(a, "cuda") for a in learners],
+                            tokens=[int(t) for t in tokens[p]], quorum_mask=masks[p], K=K, n=n))
+        recs_buf = dd.new_records(len(sizes))
+        ctx.merge_fragments_batched_rda(dev, M, dd.BF16, ETA, MU, flags=dd.DIAG_STATE, records=recs_buf)
+        torch.cuda.synchronize()
+        recs = dd.read_records(recs_buf)
+        for p, n in enumerate(sizes):
+            theta, v, learners = host[p]
+            ref = oracle.merge_fragment(theta, v, learners, dev[p]["tokens"], masks[p], K, ETA, MU,
+                                        merge=oracle.MERGE_RDA)
+            _check_record(recs[p], ref)
+            assert recs[p].n_part == counts[p]
+            assert floor_rel_err(dev[p]["global_"].cpu().numpy(), theta) <= TOL_STATE, p
+            assert floor_rel_err(dev[p]["momentum"].cpu().numpy(), v) <= TOL_STATE, p
+
+
 def test_rda_two_launch_form_collinear_gradients(dd, ctx):
     # every learner moved along the same direction by a different amount: the Gram matrix has rank
     # one, a^T G a = (sum a_j k_j)^2 |d|^2, and RDA equals the weighted mean of the gradients
