@@ -687,6 +687,31 @@ class Merger:
         del graph
         return {"median": statistics.median(times[3:]), "min": min(times[3:]), "merges_per_graph": reps}
 
+    def timed_prepared(self, reps: int = 200):
+        """The same single-fragment merges issued through ``prepare_merge_fragment`` (arguments
+        marshalled once): what a host loop that calls the library directly pays per merge."""
+        import torch
+        f0 = self.frags[0]
+        stream = torch.cuda.current_stream()
+        call = self.ctx.prepare_merge_fragment(
+            f0["global_"], f0["momentum"], self.packed_ptrs, self.packed_tokens, f0["K"], self.eta, self.mu,
+            n=f0["n"], learner_dtype=self.ldtype, flags=self.flags, out_bf16=f0["out_bf16"],
+            record=self.records, stream=stream)
+        mask = f0["quorum_mask"]
+        for _ in range(20):
+            call(mask)
+        times = []
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(5):
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for _ in range(reps):
+                call(mask)
+            e1.record(stream)
+            e1.synchronize()
+            times.append(e0.elapsed_time(e1) / reps)
+        return {"median": statistics.median(times), "min": min(times), "merges_per_sample": reps}
+
     def free(self):
         import torch
         self.frags = self.int4_codes = self.int4_scales = self.rda_scratch = self.records = None
@@ -777,6 +802,7 @@ def config_row(dd, ctx, device, name, merge, args, ceilings, probes, traffic_tab
             row["achieved_gbs_l2_flushed"] = alg / (row["ms_l2_flushed"]["median"] * 1e-3) / 1e9
             if w.P == 1 and merge == "avg":
                 row["ms_cuda_graph_replay"] = merger.timed_graph()
+                row["ms_prepared_call"] = merger.timed_prepared()
         else:
             row["l2"] = "inputs larger than L2 (no flush)"
         if not args.no_e2e and merge in ("avg", "int4") and not (merge == "avg" and not own):

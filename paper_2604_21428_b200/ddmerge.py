@@ -323,6 +323,30 @@ class Context:
             ctypes.c_float(outer_mu), ctypes.c_uint32(flags), ctypes.c_size_t(n), _ptr(out_bf16),
             _ptr(record), _stream_handle(stream)))
 
+    def prepare_merge_fragment(self, global_, momentum, learners, tokens, K: int, outer_lr: float,
+                               outer_mu: float, *, n: int | None = None, learner_dtype: int | None = None,
+                               steps=None, flags: int = 0, out_bf16=None, record=None, stream=None):
+        """``dd_merge_fragment`` with every argument but the quorum mask marshalled once: returns
+        ``call(quorum_mask)``.  For a syncer that merges the same buffers step after step the
+        per-call cost is then the C call alone.  ``tokens`` (and ``steps``) may be ``pack_u64``
+        arrays that the caller updates in place between calls; the tensors must stay alive."""
+        M = len(learners)
+        if n is None:
+            n = int(global_.numel())
+        if learner_dtype is None:
+            learner_dtype = _infer_dtype(learners)
+        fixed_head = (self._h, _ptr(global_), _ptr(momentum), _pointer_array(learners), M, learner_dtype,
+                      _u64_array(tokens), None if steps is None else _u64_array(steps))
+        fixed_tail = (int(K), ctypes.c_float(outer_lr), ctypes.c_float(outer_mu), ctypes.c_uint32(flags),
+                      ctypes.c_size_t(n), _ptr(out_bf16), _ptr(record), _stream_handle(stream))
+        fn, check = lib.dd_merge_fragment, self._check
+
+        def call(quorum_mask: int) -> None:
+            rc = fn(*fixed_head, quorum_mask & 0xFFFFFFFFFFFFFFFF, *fixed_tail)
+            if rc != OK:
+                check(rc)
+        return call
+
     def merge_fragment_push(self, global_, momentum, learners, tokens, quorum_mask: int, K: int,
                             outer_lr: float, outer_mu: float, push_mask: int, *, n: int | None = None,
                             learner_dtype: int | None = None, steps=None, flags: int = 0,

@@ -654,6 +654,29 @@ def test_cuda_graph_capture_and_replay(dd, ctx):
         assert floor_rel_err(v_dev.cpu().numpy(), v) <= TOL_STATE
 
 
+def test_prepared_call_equals_plain_call(dd, ctx):
+    # arguments marshalled once, the mask given per call, token counts updated in place in between:
+    # bit-identical to the ordinary call on the same inputs
+    n, M = 50_003, 5
+    theta, v, learners = synth.fragment_cpu(n, M, "bf16", 123)
+    a = [torch.from_numpy(theta).cuda(), torch.from_numpy(v).cuda()]
+    b = [torch.from_numpy(theta).cuda(), torch.from_numpy(v).cuda()]
+    l_dev = [to_torch_learner(x, "cuda") for x in learners]
+    rec_a, rec_b = dd.new_records(1), dd.new_records(1)
+    tokens = dd.pack_u64([10, 20, 30, 40, 50])
+    call = ctx.prepare_merge_fragment(a[0], a[1], l_dev, tokens, 2, ETA, MU, flags=dd.DIAG_STATE, record=rec_a)
+    for mask, new_tokens in ((0b10111, [10, 20, 30, 40, 50]), (0b01110, [5, 0, 7, 9, 11]), (0b00001, [1, 1, 1, 1, 1])):
+        for m, t in enumerate(new_tokens):
+            tokens[m] = t
+        call(mask)
+        ctx.merge_fragment(b[0], b[1], l_dev, new_tokens, mask, 2, ETA, MU, flags=dd.DIAG_STATE, record=rec_b)
+        torch.cuda.synchronize()
+        ra, rb = dd.read_records(rec_a)[0], dd.read_records(rec_b)[0]
+        assert (ra.status, ra.idx, ra.w_hat, ra.delta_sq) == (rb.status, rb.idx, rb.w_hat, rb.delta_sq)
+        assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    assert dd.read_records(rec_a)[0].status == dd.STATUS_QUORUM_NOT_MET      # one participant, K = 2
+
+
 def test_packed_pointer_and_count_arrays(dd, ctx):
     """Pre-marshalled learner addresses and token counts give the same merge as lists."""
     n, M = 20_001, 5
