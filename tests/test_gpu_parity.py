@@ -723,6 +723,37 @@ def test_bitwise_reproducible_run_to_run(dd, ctx):
             assert all(torch.equal(a, b) for a, b in zip(first, got)), rep
 
 
+@pytest.mark.parametrize("kind,s,k", [("avg", 9, 0), ("push", 8, 8), ("push", 8, 1), ("rda", 6, 0), ("rda", 8, 0)])
+def test_bitwise_reproducible_over_repeated_merges(dd, ctx, kind, s, k):
+    """Twenty merges in a row from the same start, twice: the same bits at the end, for the launch
+    shapes that differ from the plain merge's (full ring at 9 participants, the two shapes of the fused
+    push, the two instances of the Gram launch).  A slot refilled before every lane had read it, or a
+    barrier phase out of step after a change of ring depth, would show here as a difference."""
+    n, M = 296 * 8192 * 2 + 12_345, 10
+    theta, v, learners = synth.fragment_cpu(n, M, "bf16", 505)
+    tokens = [100 + 3 * m for m in range(M)]
+    mask, push = (1 << s) - 1, (1 << k) - 1
+    ends = []
+    for rep in range(2):
+        t_dev, v_dev = torch.from_numpy(theta).cuda(), torch.from_numpy(v).cuda()
+        l_dev = [to_torch_learner(a, "cuda") for a in learners]
+        rec_buf = dd.new_records(1)
+        for _ in range(20):
+            if kind == "push":
+                ctx.merge_fragment_push(t_dev, v_dev, l_dev, tokens, mask, 2, ETA, MU, push,
+                                        flags=dd.DIAG_STATE, record=rec_buf)
+            elif kind == "rda":
+                ctx.merge_fragment_rda(t_dev, v_dev, l_dev, tokens, mask, 2, ETA, MU,
+                                       flags=dd.DIAG_STATE, record=rec_buf)
+            else:
+                ctx.merge_fragment(t_dev, v_dev, l_dev, tokens, mask, 2, ETA, MU,
+                                   flags=dd.DIAG_STATE, record=rec_buf)
+        torch.cuda.synchronize()
+        assert dd.read_records(rec_buf)[0].status == 0
+        ends.append([t_dev, v_dev, rec_buf.clone()] + [x.view(torch.int16) for x in l_dev])
+    assert all(torch.equal(a, b) for a, b in zip(*ends))
+
+
 @pytest.mark.parametrize("s", [47, 48, 49])
 def test_per_learner_norms_around_the_shared_memory_limit(dd, ctx, s):
     """Up to 48 participants the per-participant norms are summed per lane in shared memory and
